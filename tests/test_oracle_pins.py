@@ -1,0 +1,381 @@
+"""Pins of the fp64 oracle against things other than itself: library routines,
+closed forms, brute force on tiny inputs, and the invariants the paper states
+(order invariance, Eq. 4; the skip rule, Eq. 5; the HRM-first ordering, Eq. 13)."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cosa_oracle as O
+from synth.configs import tiny
+from synth.generator import bf16_bits_to_f64
+
+
+def _inputs(seed=7, hq=2, hkv=1, n=1024, needles=2):
+    q, k, v, planted = tiny(seed, hq, hkv, n, needles).make()
+    return bf16_bits_to_f64(q), bf16_bits_to_f64(k), bf16_bits_to_f64(v), planted
+
+
+@pytest.fixture(scope="module")
+def small():
+    return _inputs()
+
+
+# ---------------------------------------------------------------- dense / masked
+def test_dense_matches_library_sdpa(small):
+    q, k, v, _ = small
+    out, lse = O.dense_attention(q, k, v, causal=True)
+    tq, tk, tv = (torch.from_numpy(x) for x in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        tq[None], tk[None].repeat_interleave(2, dim=1), tv[None].repeat_interleave(2, dim=1), is_causal=True)[0]
+    assert np.abs(out - ref.numpy()).max() < 1e-12
+    # lse against a library logsumexp
+    logits = torch.einsum("hqd,hkd->hqk", tq, tk.repeat_interleave(2, dim=0)) / math.sqrt(q.shape[2])
+    mask = torch.ones(q.shape[1], q.shape[1], dtype=torch.bool).tril()
+    ref_lse = torch.logsumexp(logits.masked_fill(~mask, -float("inf")), dim=-1)
+    assert np.abs(lse - ref_lse.numpy()).max() < 1e-12
+
+
+def test_dense_noncausal_matches_library(small):
+    q, k, v, _ = small
+    out, _ = O.dense_attention(q, k, v, causal=False, query_blocks=[0, 3])
+    tq, tk, tv = (torch.from_numpy(x) for x in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq[:1, None][:, 0][None], tk[None], tv[None])[0, 0]
+    rows = np.r_[0:128, 384:512]
+    assert np.abs(out[0] - ref.numpy()[rows]).max() < 1e-12
+
+
+def test_dense_closed_forms(small):
+    q, k, v, _ = small
+    out, lse, probs = O.dense_attention(q, k, v, query_blocks=[0, 5], return_probs=True)
+    for p in probs:                                      # rows of probabilities sum to one
+        assert np.abs(p.sum(axis=1) - 1).max() < 1e-12
+    assert np.allclose(out[:, 0], v[0, 0], atol=0, rtol=0)   # the first token sees only key 0
+    vc = np.broadcast_to(np.linspace(-1, 1, v.shape[2]), v.shape).copy()
+    outc, _ = O.dense_attention(q, k, vc, query_blocks=[2])
+    assert np.abs(outc - vc[0, :128]).max() < 1e-12      # constant V rows come back unchanged
+
+
+def test_masked_reduces_to_dense(small):
+    q, k, v, _ = small
+    qbs = [0, 3, 7]
+    sets = [[list(range(i + 1)) for i in qbs] for _ in range(q.shape[0])]
+    mo, ml = O.masked_attention(q, k, v, sets, query_blocks=qbs)
+    do, dl = O.dense_attention(q, k, v, query_blocks=qbs)
+    assert np.abs(mo - do).max() < 1e-12 and np.abs(ml - dl).max() < 1e-12
+    # a strict prefix of key blocks = non-causal dense attention on physically truncated K/V
+    sets = [[[0, 1, 2]] for _ in range(q.shape[0])]
+    mo, ml = O.masked_attention(q, k, v, sets, query_blocks=[6])
+    do6, dl6 = O.dense_attention(np.ascontiguousarray(q[:, 768:896]), k[:, :384], v[:, :384], causal=False,
+                                 query_blocks=[0])
+    assert np.abs(mo - do6).max() < 1e-12 and np.abs(ml - dl6).max() < 1e-12
+
+
+# ---------------------------------------------------------------- OSK, skipping off
+def _full_lists(hq, nqb, rng=None):
+    order = np.full((hq, nqb, nqb), -1, np.int32)
+    count = np.zeros((hq, nqb), np.int32)
+    for h in range(hq):
+        for i in range(nqb):
+            ids = np.arange(i + 1)
+            if rng is not None:
+                ids = rng.permutation(ids)
+            order[h, i, :i + 1] = ids
+            count[h, i] = i + 1
+    return order, count
+
+
+def test_full_budget_osk_is_dense_in_any_order(small):
+    """Property 2 (Eq. 4): with every block listed and Stage 2 off the result is dense attention."""
+    q, k, v, _ = small
+    do, dl = O.dense_attention(q, k, v)
+    for rng in (None, np.random.default_rng(1), np.random.default_rng(2)):
+        order, count = _full_lists(q.shape[0], 8, rng)
+        r = O.osk_attention(q, k, v, order, count, skip_scale=2000.0, tightened_budget=1.0)
+        assert np.abs(r["out"] - do).max() < 1e-12 and np.abs(r["lse"] - dl).max() < 1e-12
+        assert (r["visited"] == count).all() and (r["scored"] == count).all()
+        r2 = O.osk_attention(q, k, v, order, count, skip_scale=-1.0, tightened_budget=1.0)
+        assert np.abs(r2["out"] - do).max() < 1e-12
+
+
+def test_ordered_traversal_of_a_mask_is_masked_attention(small):
+    q, k, v, _ = small
+    rng = np.random.default_rng(3)
+    hq, nqb = q.shape[0], 8
+    order = np.full((hq, nqb, nqb), -1, np.int32)
+    count = np.zeros((hq, nqb), np.int32)
+    sets = [[None] * nqb for _ in range(hq)]
+    for h in range(hq):
+        for i in range(nqb):
+            c = int(rng.integers(1, i + 2))
+            ids = rng.choice(i + 1, size=c, replace=False)
+            order[h, i, :c], count[h, i], sets[h][i] = ids, c, ids
+    r = O.osk_attention(q, k, v, order, count, tightened_budget=1.0)
+    mo, ml = O.masked_attention(q, k, v, sets)
+    assert np.abs(r["out"] - mo).max() < 1e-12 and np.abs(r["lse"] - ml).max() < 1e-12
+
+
+# ---------------------------------------------------------------- OSK, skip rule
+def _two_block_case(a, b, veto_row=None, block=4, d=4):
+    """Key block A has every logit a, key block B every logit b (non-causal, one head)."""
+    q = np.zeros((1, block, d)); q[0, :, 0] = math.sqrt(d)
+    if veto_row is not None:
+        q[0, veto_row, 0] = -math.sqrt(d)           # on this row block B lies ABOVE block A
+    k = np.zeros((1, 2 * block, d)); k[0, :block, 0] = a; k[0, block:, 0] = b
+    v = np.zeros((1, 2 * block, d)); v[0, :block] = 1.0; v[0, block:] = -2.0
+    return q, k, v
+
+
+def _run_two(q, k, v, first, delta, n_for_theta):
+    # N of the call is 2*block; choose delta so that ln(delta/N) = theta
+    order = np.array([[[first, 1 - first]]], np.int32)
+    count = np.array([[2]], np.int32)
+    return O.osk_attention(q, k, v, order, count, skip_scale=delta, tightened_budget=0.999999,
+                           causal=False, block=q.shape[1])
+
+
+def test_skip_rule_depends_on_order_running_max():
+    """Limitation 2.1: the test is against the RUNNING maximum, so (A,B) can skip B but (B,A) skips nothing."""
+    a, b = 3.0, 0.5
+    q, k, v = _two_block_case(a, b)
+    n = k.shape[1]
+    theta = -1.0                                     # b - a = -2.5 < theta  -> B negligible after A
+    delta = n * math.exp(theta)
+    r = _run_two(q, k, v, 0, delta, n)
+    assert r["decisions"][(0, 0)] == [True, False] and r["visited"][0, 0] == 1
+    assert np.allclose(r["out"], 1.0, atol=1e-15)                       # only A's values
+    assert np.allclose(r["lse"], a + math.log(4), atol=1e-14)
+    assert np.allclose(r["gaps"][(0, 0)], [0.0, b - a], atol=1e-15)
+    r = _run_two(q, k, v, 1, delta, n)               # B first: both raise the running max
+    assert r["decisions"][(0, 0)] == [True, True]
+    w = math.exp(b) / (math.exp(a) + math.exp(b))
+    assert np.allclose(r["out"], (1 - w) * 1.0 + w * -2.0, atol=1e-14)
+    # a milder threshold keeps B even after A (b - a >= theta)
+    r = _run_two(q, k, v, 0, n * math.exp(-3.0), n)
+    assert r["decisions"][(0, 0)] == [True, True]
+    assert np.allclose(r["out"], (1 - w) * 1.0 + w * -2.0, atol=1e-14)
+    # boundary: equality is NOT a skip (strict inequality in Eq. 5)
+    r = _run_two(q, k, v, 0, n * math.exp(-2.5), n)
+    gap = r["gaps"][(0, 0)][1]
+    assert r["decisions"][(0, 0)][1] == (not gap < math.log(n * math.exp(-2.5) / n))
+
+
+def test_skip_rule_single_row_veto():
+    """Limitation 2.2 (bucket effect): one row on which B is not negligible vetoes the skip."""
+    q, k, v = _two_block_case(3.0, 0.5, veto_row=2)
+    n = k.shape[1]
+    r = _run_two(q, k, v, 0, n * math.exp(-1.0), n)
+    assert r["decisions"][(0, 0)] == [True, True]
+    assert r["gaps"][(0, 0)][1] == 0.0               # B raised the maximum of the veto row
+
+
+@pytest.fixture(scope="module")
+def kap_lists(small):
+    q, k, v, _ = small
+    return O.kap_select(q, k, s=8, budget=1.0)
+
+
+def test_online_and_offline_gaps_agree_and_sets_are_nested(small, kap_lists):
+    q, k, v, _ = small
+    order, count = kap_lists
+    n = q.shape[1]
+    prev_sets = None
+    for delta in (1e-9, 50.0, 200.0, 600.0):
+        r = O.osk_attention(q, k, v, order, count, skip_scale=delta, tightened_budget=0.999999)
+        theta = math.log(delta / n)
+        sets = {}
+        for (h, i), dec in r["decisions"].items():
+            off = O.osk_gaps_offline(q, k, order, count, h, i)
+            assert np.array_equal(np.asarray(r["gaps"][(h, i)]), off)
+            assert dec == [not g < theta for g in off]
+            assert dec[0]                                   # the first listed block is always computed
+            sets[(h, i)] = {int(order[h, i, kk]) for kk, c in enumerate(dec) if c}
+        if delta == 1e-9:
+            assert all(len(s) == count[h, i] for (h, i), s in sets.items())   # Delta -> 0+ skips nothing
+        if prev_sets is not None:                           # larger Delta -> subset
+            assert all(sets[key] <= prev_sets[key] for key in sets)
+        prev_sets = sets
+        # the output is masked attention over the computed set
+        bs = [[sorted(sets[(h, i)]) for i in range(n // 128)] for h in range(q.shape[0])]
+        mo, ml = O.masked_attention(q, k, v, bs)
+        assert np.abs(r["out"] - mo).max() < 1e-12 and np.abs(r["lse"] - ml).max() < 1e-12
+    assert any(len(s) < count[h, i] for (h, i), s in prev_sets.items())       # something was skipped
+
+
+def test_hrm_first_order_makes_later_gaps_order_free(small, kap_lists):
+    """After the blocks holding a row maximum have been visited the running maximum is the
+    maximum over the whole list, so the statistic no longer depends on the order."""
+    q, k, v, _ = small
+    order, count = kap_lists
+    h, i = 1, 7
+    cnt = int(count[h, i])
+    mloc = np.stack([(q[h, i * 128:(i + 1) * 128] @ k[0, j * 128:(j + 1) * 128].T / math.sqrt(128))
+                     for j in order[h, i, :cnt]])
+    mloc[list(order[h, i, :cnt]).index(i)] = np.where(np.tri(128, dtype=bool), mloc[list(order[h, i, :cnt]).index(i)], -np.inf)
+    mloc = mloc.max(axis=2)
+    gstar = (mloc - mloc.max(axis=0)).max(axis=1)
+    gaps = O.osk_gaps_offline(q, k, order, count, h, i)
+    owners = set(np.argmax(mloc, axis=0))             # list positions that own some row's maximum
+    last = max(owners)
+    assert np.allclose(gaps[last:], gstar[last:], atol=0)
+    assert (gaps >= gstar - 1e-15).all()              # Eq. (6): running max <= global max
+
+
+def test_cap_on_computed_blocks(small, kap_lists):
+    q, k, v, _ = small
+    order, count = kap_lists
+    n = q.shape[1]
+    delta, tb = 200.0, 0.3
+    theta = math.log(delta / n)
+    r = O.osk_attention(q, k, v, order, count, skip_scale=delta, tightened_budget=tb)
+    for (h, i), dec in r["decisions"].items():
+        off = O.osk_gaps_offline(q, k, order, count, h, i)
+        cap = min(int(count[h, i]), O.budget_count(tb, i + 1))
+        want = [kk for kk, g in enumerate(off) if not g < theta][:cap]
+        got = [kk for kk, c in enumerate(dec) if c]
+        assert got == want and r["visited"][h, i // 1] == len(want)
+        if len(want) == cap:                            # the walk stops right after the cap-th computed block
+            assert len(dec) == want[-1] + 1
+    # a cap that cannot bind changes nothing
+    ra = O.osk_attention(q, k, v, order, count, skip_scale=delta, tightened_budget=0.999999)
+    assert all(ra["decisions"][key] == [not g < theta for g in O.osk_gaps_offline(q, k, order, count, *key)]
+               for key in ra["decisions"])
+    # threshold off, cap on: the first C_i listed blocks
+    rb = O.osk_attention(q, k, v, order, count, skip_scale=-1.0, tightened_budget=tb)
+    for (h, i), dec in rb["decisions"].items():
+        assert dec == [True] * min(int(count[h, i]), O.budget_count(tb, i + 1))
+
+
+def test_skip_scale_not_below_n_is_rejected(small, kap_lists):
+    q, k, v, _ = small
+    with pytest.raises(ValueError):
+        O.osk_attention(q, k, v, *kap_lists, skip_scale=float(q.shape[1]), tightened_budget=0.5)
+
+
+# ---------------------------------------------------------------- KAP scores and flags
+def test_literal_and_cancelled_forms_agree(small):
+    q, k, v, _ = small
+    for s in (4, 8, 16):
+        for h in range(q.shape[0]):
+            for i in (0, 1, 4, 7):
+                a, fa, _ = O.kap_scores(q, k, h, i, s)
+                b, fb = O.kap_scores_literal(q, k, h, i, s)
+                assert np.abs(a - b).max() <= 1e-12 * max(1.0, a.max())
+                assert np.array_equal(fa, fb)
+
+
+def test_score_and_flag_invariants(small):
+    q, k, v, _ = small
+    for s in (8, 32):
+        R = 128 // s
+        for h in range(q.shape[0]):
+            for i in range(8):
+                sc, fl, M = O.kap_scores(q, k, h, i, s)
+                assert (sc > 0).all() and (sc <= R).all()
+                assert (sc[fl] >= 1.0).all()
+                assert 1 <= fl.sum() <= R
+                # every sampled row's maximum lies in some flagged block
+                assert fl[np.argmax(M, axis=1)].all()
+
+
+def test_single_sample_per_block_reduces_to_argsort(small):
+    """s = b: one sampled row and key per block, so exactly one HRM block and the list is
+    that block followed by the others in descending order of the sampled logit."""
+    q, k, v, _ = small
+    order, count = O.kap_select(q, k, s=128, budget=1.0)
+    for h in range(q.shape[0]):
+        z = (q[h, ::128] @ k[0, ::128].T) / math.sqrt(128)
+        for i in range(8):
+            ref = np.argsort(-z[i, :i + 1], kind="stable")
+            assert list(order[h, i, :i + 1]) == list(ref)
+            _, fl, _ = O.kap_scores(q, k, h, i, 128)
+            assert fl.sum() == 1 and fl[ref[0]]
+
+
+def test_token_granularity_reduces_to_exact_logit_argsort():
+    """b = 1, s = 1: every block is one token, the list is the argsort of the true logits."""
+    rng = np.random.default_rng(5)
+    q = rng.standard_normal((1, 24, 8)); k = rng.standard_normal((1, 24, 8))
+    order, count = O.kap_select(q, k, s=1, budget=1.0, block=1)
+    z = (q[0] @ k[0].T) / math.sqrt(8)
+    for i in range(24):
+        assert list(order[0, i, :i + 1]) == list(np.argsort(-z[i, :i + 1], kind="stable"))
+
+
+# ---------------------------------------------------------------- KAP lists
+def test_lists_against_bruteforce_lexsort(small):
+    q, k, v, _ = small
+    for budget in (0.2, 0.5, 1.0):
+        order, count = O.kap_select(q, k, s=8, budget=budget)
+        for h in range(q.shape[0]):
+            for i in range(8):
+                sc, fl, _ = O.kap_scores(q, k, h, i, 8)
+                ref = np.lexsort((np.arange(i + 1), -sc, ~fl))      # last key is the primary one
+                K = math.ceil(Fraction(budget).limit_denominator(1000) * (i + 1))
+                K = max(1, min(i + 1, K))
+                assert count[h, i] == K
+                assert list(order[h, i, :K]) == list(ref[:K])
+                assert (order[h, i, K:] == -1).all()
+
+
+def test_list_structure_and_prefix_property(small):
+    q, k, v, _ = small
+    full, cfull = O.kap_select(q, k, s=8, budget=1.0)
+    for budget in (0.1, 0.25, 0.5):
+        order, count = O.kap_select(q, k, s=8, budget=budget)
+        for h in range(q.shape[0]):
+            for i in range(8):
+                c = count[h, i]
+                ids = order[h, i, :c]
+                assert len(set(ids)) == c and ids.min() >= 0 and ids.max() <= i
+                assert list(ids) == list(full[h, i, :c])            # lists are nested across budgets
+                sc, fl, _ = O.kap_scores(q, k, h, i, 8)
+                f = fl[ids]
+                assert not (np.diff(f.astype(int)) > 0).any()       # flagged blocks first
+                for grp in (ids[f], ids[~f]):
+                    assert (np.diff(sc[grp]) <= 0).all()
+    for h in range(q.shape[0]):
+        for i in range(8):
+            assert sorted(full[h, i, :i + 1]) == list(range(i + 1))
+
+
+def test_ties_break_by_ascending_block_id():
+    sc = np.array([0.5, 2.0, 0.5, 2.0, 0.5])
+    fl = np.array([False, True, True, False, False])
+    assert O.flag_grouped_order(sc, fl) == [1, 2, 3, 0, 4]
+
+
+def test_budget_count_is_exact_ceiling():
+    for b in (0.5, 0.25, 0.125, 0.2, 0.1, 0.08, 0.04, 0.0625, 1.0, 0.05, 0.025, 0.03125):
+        for J in list(range(1, 300)) + [511, 512, 1000, 1024]:
+            want = max(1, min(J, math.ceil(Fraction(str(b)) * J)))
+            assert O.budget_count(b, J) == want, (b, J)
+
+
+def test_planted_structure_is_recalled():
+    q, k, v, planted = _inputs(seed=11, hq=4, hkv=1, n=2048, needles=3)
+    order, count = O.kap_select(q, k, s=8, budget=0.35)
+    for h in range(4):
+        for i in range(8, 16):
+            ids = set(order[h, i, :count[h, i]])
+            assert 0 in ids and i - 1 in ids                        # sink and local band
+        for j, t in zip(planted["needle_key_blocks"][0], planted["needle_targets"][0]):
+            if t >= 3:
+                assert j in set(order[h, t, :count[h, t]])          # the needle, at its target block
+
+
+def test_frozen_oracle_outputs():
+    """The stored values were written by tests/golden/make_golden.py from the oracle alone."""
+    import json
+    import os
+    with open(os.path.join(os.path.dirname(__file__), "golden", "oracle_tiny.json")) as f:
+        doc = json.load(f)
+    q, k, v, _ = _inputs()
+    order, count = O.kap_select(q, k, s=8, budget=0.5)
+    assert order.tolist() == doc["order"] and count.tolist() == doc["count"]
+    r = O.osk_attention(q, k, v, order, count, skip_scale=200.0, tightened_budget=0.3)
+    assert r["visited"].tolist() == doc["visited"] and r["scored"].tolist() == doc["scored"]
+    assert np.allclose(r["out"][1, 1000, :4], doc["out_sample"], atol=1e-13)
+    assert np.allclose(r["lse"][0, ::128], doc["lse_sample"], atol=1e-13)
