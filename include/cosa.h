@@ -1,0 +1,186 @@
+/*
+ * cosa.h -- C ABI of the CoSA prefill hot path on NVIDIA B200 (sm_100a).
+ *
+ * Two stages (paper Sec. 4, Algorithm A):
+ *   KAP  Kernel-Aware Proxy (Sec. 4.2, Eqs. 8-14; Algorithm A steps 2-5): scores every
+ *        (query block, key block) pair from stride-sampled Q and K, flags the blocks that
+ *        hold a sampled row's maximum ("HRM"), orders the candidates HRM-first by descending
+ *        score and keeps a budgeted prefix: the ordered visit list M_KAP.
+ *   OSK  Ordered-Skipping Kernel (Sec. 4.3, Eq. 5; Algorithm A steps 7-21): block-sparse
+ *        online-softmax attention that visits exactly the listed key/value blocks in the
+ *        listed order and drops the value-side work of a block when every query row's block
+ *        maximum lies more than ln(N/Delta) below the running row maximum.
+ *
+ * Conventions
+ *   - All tensors are dense, row-major, innermost dimension contiguous, base pointers
+ *     16-byte aligned.  Layouts:
+ *         q, out              [B, Hq,  N, d]   bf16
+ *         k, v                [B, Hkv, N, d]   bf16      (query head h reads KV head h / (Hq/Hkv))
+ *         order               [B, Hq, nQB, order_stride] int32   0-based key-block ids, then -1
+ *         count, visited,
+ *         scored              [B, Hq, nQB]     int32
+ *         lse                 [B, Hq, N]       float32   natural log, scaled logits
+ *     with nQB = N / 128.  Supported: d = 128, block_q = block_k = 128, N % 128 == 0.
+ *   - Unless a function says "host", every data pointer is a DEVICE pointer owned by the
+ *     caller.  The library never frees or keeps them.
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream).  They do not synchronise; outputs are valid once the stream reaches
+ *     that point.
+ *   - Return value: 0 on success, a negative cosa_status otherwise.  Nothing is enqueued
+ *     when an argument check fails.  No call throws or exits.
+ *   - Block ids, list positions and rows are 0-based (the paper counts from 1).
+ */
+#ifndef COSA_H_
+#define COSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COSA_OK = 0,
+  COSA_ERR_INVALID_ARG = -1,   /* null pointer, bad shape, budget outside (0,1], Delta >= N ...  */
+  COSA_ERR_UNSUPPORTED = -2,   /* d != 128, block != 128, N % 128 != 0, stride not a power of 2  */
+  COSA_ERR_WORKSPACE = -3,     /* workspace missing or too small                                 */
+  COSA_ERR_CUDA = -4,          /* a CUDA runtime call failed (see cosa_last_cuda_error)          */
+  COSA_ERR_DEVICE_TIMEOUT = -5,/* a bounded device-side wait ran out (from cosa_device_status)   */
+  COSA_ERR_BAD_ORDER = -6      /* an order list holds an id outside its legal range              */
+} cosa_status;
+
+/* Problem shape shared by both stages. */
+typedef struct {
+  int32_t batch;      /* B   */
+  int32_t hq;         /* Hq  */
+  int32_t hkv;        /* Hkv, divides Hq */
+  int32_t n;          /* N, sequence length, multiple of 128 */
+  int32_t d;          /* head dimension, must be 128 */
+  int32_t block_q;    /* must be 128 */
+  int32_t block_k;    /* must be 128 */
+  int32_t causal;     /* 1: candidates of query block i are key blocks j <= i (Algorithm A step 5)
+                         and the diagonal block is masked per token; 0: all key blocks */
+} cosa_shape;
+
+/* Parameters the paper names (Algorithm A "Parameter") plus optional outputs.
+ * Zero-initialise, then set what you need; cosa_default_options() fills the defaults. */
+typedef struct {
+  int32_t stride;          /* KAP sampling stride s: sampled row r is token r*s; power of two,
+                              1 <= s <= 128; default 8                                           */
+  float   skip_scale;      /* Delta of Eq. (5); <= 0 disables the threshold test (the paper's
+                              Delta = -1); must be < N otherwise; default 2000                   */
+  float   softmax_scale;   /* 0 -> 1/sqrt(d)                                                     */
+  int32_t order_stride;    /* row pitch of the order tensor in elements; 0 -> nQB                */
+  int32_t* out_scored;     /* optional [B,Hq,nQB]: blocks whose logits OSK formed                */
+  uint32_t* out_decisions; /* optional [B,Hq,nQB,ceil(order_stride/32)]: bit kk set = the block
+                              at list position kk was computed                                   */
+  float*  kap_scores;      /* optional [B,Hq,nQB,nQB]: KAP block scores s_ij (Eq. 11), j <= i    */
+  uint8_t* kap_flags;      /* optional [B,Hq,nQB,nQB]: HRM flags h_ij (Eq. 12)                   */
+  void*   workspace;       /* device scratch; NULL -> the library's own per-device scratch,
+                              which is allocated (cudaMalloc) on first use or growth             */
+  size_t  workspace_bytes;
+  int32_t impl;            /* 0 = fastest available; 1 = plain CUDA-core check kernels           */
+} cosa_options;
+
+void cosa_default_options(cosa_options* opt);
+
+/* Scratch bytes a call with explicit workspace needs.  op: 0 = KAP, 1 = OSK, 2 = both. */
+size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt);
+
+/* Number of blocks kept out of `candidates` under a budget fraction: ceil(budget*candidates)
+ * evaluated as (floor(budget_f32 * 2^20) * candidates + 2^20 - 1) >> 20, clamped to
+ * [1, candidates].  This is how K_i = B_stage1 x J (Eq. 14) and the Stage-2 cap are rounded. */
+int32_t cosa_budget_count(float budget, int32_t candidates);
+
+/*
+ * Stage 1 -- cosa_kap_select (Sec. 4.2; Algorithm A steps 2-5; Eqs. 8-14).
+ *
+ * For every query head h and query block i: sample every s-th row of Q_i and of the
+ * candidate keys, form the scaled logits (causally masked at sampled-token level), take per
+ * sampled row the maximum inside each key block (MaxPool) and divide by the row's overall
+ * maximum after the softmax (MaxNorm) -- i.e. Pbar[r,j] = exp(M[r,j] - max_j' M[r,j']) --,
+ * sum over the block's sampled rows (score s_ij), flag blocks holding some row's maximum
+ * (h_ij), sort by (h_ij descending, s_ij descending, j ascending) and keep the first
+ * K_i = cosa_budget_count(budget, candidates) ids.
+ *
+ *   q, k        in   device bf16, layouts above
+ *   budget      in   Stage-1 fraction in (0, 1]
+ *   out_order   out  device int32 [B,Hq,nQB,order_stride]; positions >= count are set to -1;
+ *                    order_stride must be >= the largest K_i
+ *   out_count   out  device int32 [B,Hq,nQB]
+ * Scores are evaluated so that the list equals the one exact arithmetic would give whenever
+ * neighbouring scores differ by more than ~1e-9 relative.
+ */
+int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape,
+                    float budget, int32_t* out_order, int32_t* out_count, void* stream);
+int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape,
+                       float budget, int32_t* out_order, int32_t* out_count, void* stream,
+                       const cosa_options* opt);
+
+/*
+ * Stage 2 -- cosa_osk_attention (Sec. 4.3; Algorithm A steps 7-21; skip rule Eq. 5).
+ *
+ * For every (h, i): m = -inf, l = 0, O = 0; for kk = 0 .. count-1: j = order[kk];
+ * S = Q_i K_j^T * scale (token-level causal mask when j == i); m_loc = rowmax S;
+ * m' = m; m = max(m, m_loc); the block is skipped iff Stage 2 is on, Delta > 0 and
+ * max_r (m_loc[r] - m[r]) < ln(Delta / N); otherwise P = exp(S - m),
+ * l = exp(m'-m) l + rowsum P, O = diag(exp(m'-m)) O + P V_j.  At the end O /= l and
+ * lse = m + ln l.
+ *
+ *   tightened_budget  >= 1: Stage 2 off (no threshold test, no cap): the call is exactly
+ *                     attention restricted to the listed blocks; with full lists, dense
+ *                     attention.  < 1: the threshold test runs with Delta = opt->skip_scale
+ *                     and the walk also ends once cosa_budget_count(tightened_budget,
+ *                     candidates) blocks (at most count) have been computed.
+ *   order, count      in   as produced by cosa_kap_select (or any caller-built lists whose
+ *                          ids are legal: 0 <= j < nQB, and j <= i when causal)
+ *   out               out  device bf16 [B,Hq,N,d]
+ *   out_lse           out  device float32 [B,Hq,N], may be NULL
+ *   out_visited       out  device int32 [B,Hq,nQB] number of computed blocks, may be NULL
+ * P is rounded to bf16 before the PV product, accumulation is float32.
+ */
+int cosa_osk_attention(const void* q, const void* k, const void* v, const cosa_shape* shape,
+                       const int32_t* order, const int32_t* count, float tightened_budget,
+                       void* out, float* out_lse, int32_t* out_visited, void* stream);
+int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cosa_shape* shape,
+                          const int32_t* order, const int32_t* count, float tightened_budget,
+                          void* out, float* out_lse, int32_t* out_visited, void* stream,
+                          const cosa_options* opt);
+
+/*
+ * Read-only check of caller-built lists (Eq. 14 encoding): every id at a position < count is
+ * in [0, nQB) and, when causal, <= its query block; count is in [1, order_stride].
+ * Writes 0 or COSA_ERR_BAD_ORDER to the device word *out_status_dev (asynchronously).
+ */
+int cosa_validate_order(const int32_t* order, const int32_t* count, const cosa_shape* shape,
+                        int32_t order_stride, int32_t* out_status_dev, void* stream);
+
+/*
+ * Whole path on HOST buffers (Algorithm A end to end): copies q, k, v to the device
+ * workspace, runs KAP then OSK, copies out / lse / visited back.  All data pointers are HOST
+ * pointers (pinned memory gives asynchronous copies); `device_workspace` is a DEVICE buffer of
+ * at least cosa_host_call_workspace_bytes() bytes.  Outputs are valid after the stream is
+ * synchronised.  out_lse_host and out_visited_host may be NULL.
+ */
+size_t cosa_host_call_workspace_bytes(const cosa_shape* shape, const cosa_options* opt);
+int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host,
+                      const cosa_shape* shape, float budget, float tightened_budget,
+                      void* out_host, float* out_lse_host, int32_t* out_visited_host,
+                      void* device_workspace, size_t device_workspace_bytes, void* stream,
+                      const cosa_options* opt);
+
+/* Synchronises `stream` and returns the device status word of the current device: 0, or
+ * COSA_ERR_DEVICE_TIMEOUT if a bounded wait inside a kernel gave up (the kernel then wrote
+ * no further results), then clears it. */
+int cosa_device_status(void* stream);
+
+/* Text of the last failing CUDA runtime call on this thread ("" if none). */
+const char* cosa_last_cuda_error(void);
+const char* cosa_status_string(int status);
+int cosa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COSA_H_ */

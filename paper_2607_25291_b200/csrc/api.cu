@@ -1,0 +1,300 @@
+// The C ABI declared in include/cosa.h: argument checks, option resolution, kernel dispatch.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace cosa {
+
+__device__ int32_t g_status_word = 0;
+
+static thread_local char tl_cuda_error[256] = "";
+
+static int cuda_fail(cudaError_t e, const char* what) {
+  snprintf(tl_cuda_error, sizeof(tl_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+  return COSA_ERR_CUDA;
+}
+
+int32_t* device_status_word() {
+  void* ptr = nullptr;
+  if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess) return nullptr;
+  return static_cast<int32_t*>(ptr);
+}
+
+// ---- the library's own per-device scratch (used when options.workspace is NULL) ----
+namespace {
+constexpr int kMaxDevices = 64;
+struct OwnScratch { void* ptr = nullptr; size_t bytes = 0; };
+OwnScratch g_scratch[kMaxDevices];
+std::mutex g_scratch_mu;
+
+int own_scratch(size_t need, void** out) {
+  *out = nullptr;
+  if (need == 0) return COSA_OK;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+  if (dev < 0 || dev >= kMaxDevices) return COSA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mu);
+  OwnScratch& s = g_scratch[dev];
+  if (s.bytes < need) {
+    if (s.ptr) {
+      e = cudaFree(s.ptr);  // synchronises: earlier users of the old scratch have finished
+      s.ptr = nullptr; s.bytes = 0;
+      if (e != cudaSuccess) return cuda_fail(e, "cudaFree(scratch)");
+    }
+    e = cudaMalloc(&s.ptr, need);
+    if (e != cudaSuccess) { s.ptr = nullptr; return cuda_fail(e, "cudaMalloc(scratch)"); }
+    s.bytes = need;
+  }
+  *out = s.ptr;
+  return COSA_OK;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_shape(const cosa_shape* s) {
+  if (!s) return COSA_ERR_INVALID_ARG;
+  if (s->batch < 1 || s->hq < 1 || s->hkv < 1 || s->n < 1) return COSA_ERR_INVALID_ARG;
+  if (s->hq % s->hkv != 0) return COSA_ERR_INVALID_ARG;
+  if (s->d != kHeadDim || s->block_q != kBlock || s->block_k != kBlock) return COSA_ERR_UNSUPPORTED;
+  if (s->n % kBlock != 0) return COSA_ERR_UNSUPPORTED;
+  return COSA_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+cosa_options resolve_options(const cosa_options* opt) {
+  cosa_options o;
+  cosa_default_options(&o);
+  if (opt) {
+    o = *opt;
+    if (o.stride == 0) o.stride = 8;
+    if (o.skip_scale == 0.f) o.skip_scale = 2000.f;
+  }
+  return o;
+}
+}  // namespace
+
+// scratch the kernels of one call need (beyond inputs and outputs)
+static size_t kap_scratch_bytes(const cosa_shape*, const cosa_options&) { return 0; }
+static size_t osk_scratch_bytes(const cosa_shape*, const cosa_options&) { return 0; }
+
+}  // namespace cosa
+
+using namespace cosa;
+
+extern "C" {
+
+void cosa_default_options(cosa_options* opt) {
+  if (!opt) return;
+  memset(opt, 0, sizeof(*opt));
+  opt->stride = 8;
+  opt->skip_scale = 2000.f;
+}
+
+int32_t cosa_budget_count(float budget, int32_t candidates) {
+  return budget_count_fx(budget_to_fx(budget), candidates);
+}
+
+size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt) {
+  if (check_shape(shape) != COSA_OK) return 0;
+  cosa_options o = resolve_options(opt);
+  size_t a = align_up(kap_scratch_bytes(shape, o), 256), b = align_up(osk_scratch_bytes(shape, o), 256);
+  if (op == 0) return a;
+  if (op == 1) return b;
+  return a > b ? a : b;
+}
+
+int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, float budget, int32_t* out_order,
+                       int32_t* out_count, void* stream, const cosa_options* opt) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!q || !k || !out_order || !out_count) return COSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return COSA_ERR_INVALID_ARG;
+  if (!(budget > 0.f) || budget > 1.f) return COSA_ERR_INVALID_ARG;
+  cosa_options o = resolve_options(opt);
+  const int s = o.stride;
+  if (s < 1 || s > kBlock || (s & (s - 1)) != 0) return COSA_ERR_UNSUPPORTED;
+  const int nqb = shape->n / kBlock;
+  const int order_stride = o.order_stride > 0 ? o.order_stride : nqb;
+  KapParams p{};
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k = static_cast<const __nv_bfloat16*>(k);
+  p.order = out_order;
+  p.count = out_count;
+  p.dbg_scores = o.kap_scores;
+  p.dbg_flags = o.kap_flags;
+  p.batch = shape->batch; p.hq = shape->hq; p.hkv = shape->hkv; p.n = shape->n; p.nqb = nqb;
+  p.causal = shape->causal ? 1 : 0;
+  p.stride = s;
+  p.rows = kBlock / s;
+  p.order_stride = order_stride;
+  p.budget_fx = budget_to_fx(budget);
+  p.scale = o.softmax_scale > 0.f ? (double)o.softmax_scale : 1.0 / sqrt((double)shape->d);
+  // the list of the longest row must fit the pitch
+  if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
+  if (kap_exact_smem_bytes(p.rows, nqb) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
+  cudaError_t e = launch_kap_exact(p, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "kap launch");
+  return COSA_OK;
+}
+
+int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape, float budget, int32_t* out_order,
+                    int32_t* out_count, void* stream) {
+  return cosa_kap_select_ex(q, k, shape, budget, out_order, out_count, stream, nullptr);
+}
+
+int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cosa_shape* shape, const int32_t* order,
+                          const int32_t* count, float tightened_budget, void* out, float* out_lse,
+                          int32_t* out_visited, void* stream, const cosa_options* opt) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!q || !k || !v || !order || !count || !out) return COSA_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return COSA_ERR_INVALID_ARG;
+  if (!(tightened_budget > 0.f)) return COSA_ERR_INVALID_ARG;
+  cosa_options o = resolve_options(opt);
+  const int nqb = shape->n / kBlock;
+  OskParams p{};
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.k = static_cast<const __nv_bfloat16*>(k);
+  p.v = static_cast<const __nv_bfloat16*>(v);
+  p.order = order; p.count = count;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = out_lse; p.visited = out_visited;
+  p.scored = o.out_scored; p.decisions = o.out_decisions;
+  p.batch = shape->batch; p.hq = shape->hq; p.hkv = shape->hkv; p.n = shape->n; p.nqb = nqb;
+  p.causal = shape->causal ? 1 : 0;
+  p.order_stride = o.order_stride > 0 ? o.order_stride : nqb;
+  p.stage2 = tightened_budget < 1.f ? 1 : 0;
+  p.use_threshold = (p.stage2 && o.skip_scale > 0.f) ? 1 : 0;
+  if (p.use_threshold && !(o.skip_scale < (float)shape->n)) return COSA_ERR_INVALID_ARG;
+  p.cap_fx = budget_to_fx(tightened_budget);
+  p.theta = p.use_threshold ? (float)log((double)o.skip_scale / (double)shape->n) : 0.f;
+  p.scale = o.softmax_scale > 0.f ? o.softmax_scale : (float)(1.0 / sqrt((double)shape->d));
+  cudaError_t e = launch_osk_check(p, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "osk launch");
+  return COSA_OK;
+}
+
+int cosa_osk_attention(const void* q, const void* k, const void* v, const cosa_shape* shape, const int32_t* order,
+                       const int32_t* count, float tightened_budget, void* out, float* out_lse, int32_t* out_visited,
+                       void* stream) {
+  return cosa_osk_attention_ex(q, k, v, shape, order, count, tightened_budget, out, out_lse, out_visited, stream,
+                               nullptr);
+}
+
+int cosa_validate_order(const int32_t* order, const int32_t* count, const cosa_shape* shape, int32_t order_stride,
+                        int32_t* out_status_dev, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!order || !count || !out_status_dev || order_stride < 1) return COSA_ERR_INVALID_ARG;
+  const int nqb = shape->n / kBlock;
+  cudaError_t e = launch_validate_order(order, count, shape->batch * shape->hq * nqb, nqb, shape->causal ? 1 : 0,
+                                        order_stride, out_status_dev, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "validate launch");
+  return COSA_OK;
+}
+
+// ---- whole path on host buffers ----
+namespace {
+struct HostCallLayout {
+  size_t q, k, v, out, lse, order, count, visited, scratch, total;
+  size_t q_bytes, kv_bytes, lse_bytes, order_bytes, cnt_bytes;
+  int order_stride;
+};
+HostCallLayout host_layout(const cosa_shape* s, const cosa_options& o) {
+  HostCallLayout L{};
+  const size_t nqb = s->n / kBlock;
+  L.order_stride = o.order_stride > 0 ? o.order_stride : (int)nqb;
+  L.q_bytes = (size_t)s->batch * s->hq * s->n * s->d * 2;
+  L.kv_bytes = (size_t)s->batch * s->hkv * s->n * s->d * 2;
+  L.lse_bytes = (size_t)s->batch * s->hq * s->n * 4;
+  L.order_bytes = (size_t)s->batch * s->hq * nqb * L.order_stride * 4;
+  L.cnt_bytes = (size_t)s->batch * s->hq * nqb * 4;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t at = off; off += align_up(bytes, 256); return at; };
+  L.q = take(L.q_bytes); L.k = take(L.kv_bytes); L.v = take(L.kv_bytes); L.out = take(L.q_bytes);
+  L.lse = take(L.lse_bytes); L.order = take(L.order_bytes); L.count = take(L.cnt_bytes);
+  L.visited = take(L.cnt_bytes);
+  L.scratch = off;
+  size_t a = kap_scratch_bytes(s, o), b = osk_scratch_bytes(s, o);
+  off += align_up(a > b ? a : b, 256);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t cosa_host_call_workspace_bytes(const cosa_shape* shape, const cosa_options* opt) {
+  if (check_shape(shape) != COSA_OK) return 0;
+  return host_layout(shape, resolve_options(opt)).total;
+}
+
+int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host, const cosa_shape* shape,
+                      float budget, float tightened_budget, void* out_host, float* out_lse_host,
+                      int32_t* out_visited_host, void* device_workspace, size_t device_workspace_bytes, void* stream,
+                      const cosa_options* opt) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!q_host || !k_host || !v_host || !out_host || !device_workspace) return COSA_ERR_INVALID_ARG;
+  cosa_options o = resolve_options(opt);
+  HostCallLayout L = host_layout(shape, o);
+  if (device_workspace_bytes < L.total || !aligned16(device_workspace)) return COSA_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(device_workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(ws + L.q, q_host, L.q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D q");
+  if ((e = cudaMemcpyAsync(ws + L.k, k_host, L.kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D k");
+  if ((e = cudaMemcpyAsync(ws + L.v, v_host, L.kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D v");
+  o.order_stride = L.order_stride;
+  o.workspace = ws + L.scratch;
+  o.workspace_bytes = L.total - L.scratch;
+  o.kap_scores = nullptr; o.kap_flags = nullptr; o.out_scored = nullptr; o.out_decisions = nullptr;
+  rc = cosa_kap_select_ex(ws + L.q, ws + L.k, shape, budget, reinterpret_cast<int32_t*>(ws + L.order),
+                          reinterpret_cast<int32_t*>(ws + L.count), stream, &o);
+  if (rc != COSA_OK) return rc;
+  rc = cosa_osk_attention_ex(ws + L.q, ws + L.k, ws + L.v, shape, reinterpret_cast<int32_t*>(ws + L.order),
+                             reinterpret_cast<int32_t*>(ws + L.count), tightened_budget, ws + L.out,
+                             reinterpret_cast<float*>(ws + L.lse), reinterpret_cast<int32_t*>(ws + L.visited), stream, &o);
+  if (rc != COSA_OK) return rc;
+  if ((e = cudaMemcpyAsync(out_host, ws + L.out, L.q_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H out");
+  if (out_lse_host && (e = cudaMemcpyAsync(out_lse_host, ws + L.lse, L.lse_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H lse");
+  if (out_visited_host && (e = cudaMemcpyAsync(out_visited_host, ws + L.visited, L.cnt_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H visited");
+  return COSA_OK;
+}
+
+int cosa_device_status(void* stream) {
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+  int32_t word = 0;
+  e = cudaMemcpyFromSymbol(&word, g_status_word, sizeof(word));
+  if (e != cudaSuccess) return cuda_fail(e, "read status");
+  if (word != 0) {
+    int32_t zero = 0;
+    e = cudaMemcpyToSymbol(g_status_word, &zero, sizeof(zero));
+    if (e != cudaSuccess) return cuda_fail(e, "clear status");
+  }
+  return word;
+}
+
+const char* cosa_last_cuda_error(void) { return tl_cuda_error; }
+
+const char* cosa_status_string(int status) {
+  switch (status) {
+    case COSA_OK: return "ok";
+    case COSA_ERR_INVALID_ARG: return "invalid argument";
+    case COSA_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case COSA_ERR_WORKSPACE: return "workspace missing or too small";
+    case COSA_ERR_CUDA: return "CUDA runtime error";
+    case COSA_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+    case COSA_ERR_BAD_ORDER: return "order list holds an illegal block id";
+    default: return "unknown status";
+  }
+}
+
+int cosa_version(void) { return 100; }
+
+}  // extern "C"

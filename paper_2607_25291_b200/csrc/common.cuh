@@ -1,0 +1,75 @@
+// Shared declarations of the CoSA CUDA library (host launchers + small device helpers).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cosa.h"
+
+namespace cosa {
+
+constexpr int kBlock = 128;  // logical query/key block b (Sec. C.1: b = 128)
+constexpr int kHeadDim = 128;
+
+// Resolved call parameters handed to the kernels.
+struct KapParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  int32_t* order;
+  int32_t* count;
+  float* dbg_scores;     // optional
+  uint8_t* dbg_flags;    // optional
+  int batch, hq, hkv, n, nqb;
+  int causal;
+  int stride;            // s
+  int rows;              // R = 128 / s
+  int order_stride;
+  long long budget_fx;   // floor(budget_f32 * 2^20)
+  double scale;          // softmax scale applied to the sampled logits
+};
+
+struct OskParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  const __nv_bfloat16* v;
+  const int32_t* order;
+  const int32_t* count;
+  __nv_bfloat16* out;
+  float* lse;            // optional
+  int32_t* visited;      // optional
+  int32_t* scored;       // optional
+  uint32_t* decisions;   // optional
+  int batch, hq, hkv, n, nqb;
+  int causal;
+  int order_stride;
+  int stage2;            // 0: no threshold, no cap
+  int use_threshold;     // stage2 && Delta > 0
+  long long cap_fx;      // floor(tightened_budget_f32 * 2^20)
+  float theta;           // ln(Delta / N)
+  float scale;           // softmax scale
+};
+
+// ceil(fx * candidates / 2^20) clamped to [1, candidates]  (rounding of Eq. 14's K_i = B x J)
+__host__ __device__ inline int budget_count_fx(long long fx, int candidates) {
+  long long kept = (fx * (long long)candidates + ((1LL << 20) - 1)) >> 20;
+  if (kept < 1) kept = 1;
+  if (kept > candidates) kept = candidates;
+  return (int)kept;
+}
+
+inline long long budget_to_fx(float budget) {
+  double b = (double)budget * 1048576.0;
+  return (long long)b;  // floor for positive values
+}
+
+// device status word (one per device), set by kernels whose bounded waits give up
+int32_t* device_status_word();
+
+cudaError_t launch_kap_exact(const KapParams& p, cudaStream_t st);
+size_t kap_exact_smem_bytes(int rows, int nqb);
+cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
+cudaError_t launch_validate_order(const int32_t* order, const int32_t* count, int total_qb, int nqb,
+                                  int causal, int order_stride, int32_t* status, cudaStream_t st);
+
+}  // namespace cosa

@@ -1,0 +1,166 @@
+// KAP in double precision on CUDA cores: the exact (and slow) evaluation of the proxy
+// (Sec. 4.2, Eqs. 8-14; Algorithm A steps 2-5).  One CTA per (query head, query block):
+//   sampled logits z[r,c] -> M[r,j] = max_{c in block j} z[r,c] -> M*[r] = max_j M[r,j]
+//   s_j = sum_r exp(M[r,j] - M*[r]),  h_j = any_r [M[r,j] == M*[r]]
+//   order = sort by (h desc, s desc, j asc);  keep K_i = budget_count(candidates).
+// Products of two bf16 values are exact in double, so scores carry ~1e-16 relative error.
+#include "common.cuh"
+
+namespace cosa {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPad = kHeadDim + 1;  // row pitch in doubles: conflict-free column access
+
+__device__ __forceinline__ bool sorts_before(unsigned long long ka, unsigned ia, unsigned long long kb,
+                                             unsigned ib) {
+  return ka > kb || (ka == kb && ia < ib);
+}
+
+// smem: Qs[R][kPad] | Ks[KB*R][kPad] | Z[KB*R*R] | M[R][Jpad] | Mstar[R] | sort keys | sort ids
+__global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb_per_iter, int sort_cap) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int R = p.rows;
+  const int i = p.nqb - 1 - (int)blockIdx.x;  // longest lists first
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.hq / p.hkv);
+  const int J = p.causal ? i + 1 : p.nqb;
+  const int Jpad = p.nqb | 1;
+  const int tid = threadIdx.x;
+
+  double* Qs = reinterpret_cast<double*>(smem_raw);
+  double* Ks = Qs + (size_t)R * kPad;
+  double* Z = Ks + (size_t)kb_per_iter * R * kPad;
+  double* M = Z + (size_t)kb_per_iter * R * R;
+  double* Mstar = M + (size_t)R * Jpad;
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(Mstar + R);
+  unsigned* ids = reinterpret_cast<unsigned*>(keys + sort_cap);
+
+  const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+  const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
+
+  // sampled query rows of block i: tokens (i*R + r) * s
+  for (int e = tid; e < R * kHeadDim; e += kThreads) {
+    int r = e / kHeadDim, d = e % kHeadDim;
+    size_t tok = (size_t)(i * R + r) * p.stride;
+    Qs[r * kPad + d] = (double)__bfloat162float(qh[tok * kHeadDim + d]);
+  }
+
+  for (int j0 = 0; j0 < J; j0 += kb_per_iter) {
+    const int nb = min(kb_per_iter, J - j0);
+    __syncthreads();
+    for (int e = tid; e < nb * R * kHeadDim; e += kThreads) {
+      int c = e / kHeadDim, d = e % kHeadDim;  // c: sampled key within this group of blocks
+      size_t tok = (size_t)(j0 * R + c) * p.stride;
+      Ks[c * kPad + d] = (double)__bfloat162float(kh[tok * kHeadDim + d]);
+    }
+    __syncthreads();
+    for (int e = tid; e < nb * R * R; e += kThreads) {
+      int c = e % (nb * R), r = e / (nb * R);
+      const double* qr = Qs + r * kPad;
+      const double* kc = Ks + c * kPad;
+      double acc = 0.0;
+#pragma unroll 8
+      for (int d = 0; d < kHeadDim; ++d) acc = fma(qr[d], kc[d], acc);
+      Z[(size_t)r * (kb_per_iter * R) + c] = acc * p.scale;
+    }
+    __syncthreads();
+    for (int e = tid; e < nb * R; e += kThreads) {
+      int jj = e % nb, r = e / nb;
+      int j = j0 + jj;
+      const double* zr = Z + (size_t)r * (kb_per_iter * R) + jj * R;
+      int cmax = R;  // valid sampled keys of this block for this row
+      if (p.causal && j == i) cmax = r + 1;
+      double m = zr[0];
+      for (int c = 1; c < cmax; ++c) m = fmax(m, zr[c]);
+      M[(size_t)r * Jpad + j] = m;
+    }
+  }
+  __syncthreads();
+  // M*[r]: the row's maximum over all candidate blocks
+  for (int r = tid / 32; r < R; r += kThreads / 32) {
+    double m = -INFINITY;
+    for (int j = tid % 32; j < J; j += 32) m = fmax(m, M[(size_t)r * Jpad + j]);
+    for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (tid % 32 == 0) Mstar[r] = m;
+  }
+  __syncthreads();
+  const size_t dbg_row = ((size_t)(b * p.hq + h) * p.nqb + i) * p.nqb;
+  int P2 = 2;  // sort size: next power of two >= J (<= sort_cap)
+  while (P2 < J) P2 <<= 1;
+  for (int j = tid; j < P2; j += kThreads) {
+    if (j < J) {
+      double s = 0.0;
+      bool flag = false;
+      for (int r = 0; r < R; ++r) {
+        double mv = M[(size_t)r * Jpad + j], ms = Mstar[r];
+        s += exp(mv - ms);
+        flag |= (mv == ms);
+      }
+      keys[j] = (unsigned long long)__double_as_longlong(s) | (flag ? (1ULL << 63) : 0ULL);
+      ids[j] = (unsigned)j;
+      if (p.dbg_scores) p.dbg_scores[dbg_row + j] = (float)s;
+      if (p.dbg_flags) p.dbg_flags[dbg_row + j] = flag ? 1 : 0;
+    } else {
+      keys[j] = 0ULL;
+      ids[j] = 0xffffffffu;
+    }
+  }
+  __syncthreads();
+  // bitonic sort into "sorts_before" order
+  for (int k = 2; k <= P2; k <<= 1) {
+    for (int jstep = k >> 1; jstep > 0; jstep >>= 1) {
+      for (int t = tid; t < P2; t += kThreads) {
+        int u = t ^ jstep;
+        if (u > t) {
+          unsigned long long ka = keys[t], kb = keys[u];
+          unsigned ia = ids[t], ib = ids[u];
+          bool up = (t & k) == 0;
+          bool swap = up ? sorts_before(kb, ib, ka, ia) : sorts_before(ka, ia, kb, ib);
+          if (swap) {
+            keys[t] = kb; keys[u] = ka;
+            ids[t] = ib; ids[u] = ia;
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  const int K = budget_count_fx(p.budget_fx, J);
+  const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
+  int32_t* dst = p.order + row * p.order_stride;
+  for (int t = tid; t < p.order_stride; t += kThreads) dst[t] = (t < K) ? (int32_t)ids[t] : -1;
+  if (tid == 0) p.count[row] = K;
+}
+
+int next_pow2(int x) {
+  int p = 2;
+  while (p < x) p <<= 1;
+  return p;
+}
+
+int kb_per_iter_for(int rows) {
+  int kb = 256 / (rows * rows);  // enough key blocks per pass to give every thread a logit
+  return kb < 1 ? 1 : (kb > 16 ? 16 : kb);
+}
+
+}  // namespace
+
+size_t kap_exact_smem_bytes(int rows, int nqb) {
+  int kb = kb_per_iter_for(rows);
+  int sort_cap = next_pow2(nqb);
+  size_t doubles = (size_t)rows * kPad + (size_t)kb * rows * kPad + (size_t)kb * rows * rows +
+                   (size_t)rows * (nqb | 1) + rows;
+  return doubles * 8 + (size_t)sort_cap * 12;
+}
+
+cudaError_t launch_kap_exact(const KapParams& p, cudaStream_t st) {
+  size_t smem = kap_exact_smem_bytes(p.rows, p.nqb);
+  cudaError_t e = cudaFuncSetAttribute(kap_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(p.nqb, p.hq, p.batch);
+  kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, kb_per_iter_for(p.rows), next_pow2(p.nqb));
+  return cudaGetLastError();
+}
+
+}  // namespace cosa

@@ -1,0 +1,276 @@
+"""CUDA path vs the fp64 oracle, element by element, through the C ABI (via the thin binding).
+
+Bars: KAP order/count lists bit-exact; OSK visited/scored counts and decisions exact except at
+list positions whose oracle skip margin |gap - theta| / |theta| is below 1e-4 (either decision
+is then accepted and the comparison follows the GPU's choice there); OSK outputs (bf16 inputs,
+fp32 accumulation) within max-abs 2e-2 and mean-abs 2e-3 of the oracle, LSE within 1e-3.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_25291_b200 as cosa
+from oracle import cosa_oracle as O
+from synth.configs import WORKLOADS, tiny
+from tests.helpers import alloc_lists, alloc_outputs, to_dev, widen
+
+pytestmark = pytest.mark.gpu
+
+OUT_MAX, OUT_MEAN, LSE_TOL, MARGIN = 2e-2, 2e-3, 1e-3, 1e-4
+IMPLS = (0, 1)
+
+
+def _np(t):
+    return t[0].cpu().numpy()
+
+
+def run_kap(q, k, budget, stride=8, causal=True, order_stride=None, scores=False):
+    _, hq, n, _ = q.shape
+    nqb = n // 128
+    order, count = alloc_lists(hq, nqb, order_stride)
+    kw = {}
+    if scores:
+        kw["kap_scores"] = torch.zeros(1, hq, nqb, nqb, dtype=torch.float32, device="cuda")
+        kw["kap_flags"] = torch.zeros(1, hq, nqb, nqb, dtype=torch.uint8, device="cuda")
+    opt = cosa.default_options(stride=stride, **kw)
+    cosa.cosa_kap_select(q, k, budget, order, count, causal=causal, opt=opt)
+    assert cosa.cosa_device_status() == 0
+    return (order, count, kw) if scores else (order, count)
+
+
+def run_osk(q, k, v, order, count, tb, skip_scale, impl=0, causal=True):
+    bufs = alloc_outputs(q, order.shape[-1])
+    opt = cosa.default_options(skip_scale=skip_scale, impl=impl, out_scored=bufs["scored"],
+                               out_decisions=bufs["decisions"])
+    cosa.cosa_osk_attention(q, k, v, order, count, tb, bufs["out"], bufs["lse"], bufs["visited"], causal=causal,
+                            opt=opt)
+    assert cosa.cosa_device_status() == 0
+    return bufs
+
+
+def check_osk_against_oracle(qf, kf, vf, order_np, count_np, bufs, tb, skip_scale, heads, query_blocks, causal=True):
+    """Decisions, counters and outputs of the listed (head, query block) pairs."""
+    n = qf.shape[1]
+    nkb = n // 128
+    out = _np(bufs["out"].float()).astype(np.float64)
+    lse = _np(bufs["lse"]).astype(np.float64)
+    visited, scored = _np(bufs["visited"]), _np(bufs["scored"])
+    dec_words = _np(bufs["decisions"]).view(np.uint32)
+    stage2 = tb < 1.0
+    use_rule = stage2 and skip_scale > 0
+    theta = math.log(skip_scale / n) if use_rule else None
+    worst_max, sum_abs, n_el, worst_lse, free = 0.0, 0.0, 0, 0.0, 0
+    for h in heads:
+        for i in query_blocks:
+            cnt = int(count_np[h, i])
+            J = i + 1 if causal else nkb
+            cap = min(cnt, O.budget_count(tb, J)) if stage2 else cnt
+            gaps = O.osk_gaps_offline(qf, kf, order_np, count_np, h, i, causal=causal)
+            gpu_dec = [(int(dec_words[h, i, kk >> 5]) >> (kk & 31)) & 1 == 1 for kk in range(cnt)]
+            want, computed = [], 0
+            for kk in range(cnt):
+                if computed == cap:
+                    break
+                if use_rule and abs(gaps[kk] - theta) < MARGIN * abs(theta):
+                    d = gpu_dec[kk]                       # near the margin: either decision is accepted
+                    free += 1
+                else:
+                    d = not (use_rule and gaps[kk] < theta)
+                want.append(d)
+                computed += d
+            assert gpu_dec[:len(want)] == want and not any(gpu_dec[len(want):]), (h, i)
+            assert scored[h, i] == len(want) and visited[h, i] == sum(want), (h, i)
+            ids = [int(order_np[h, i, kk]) for kk, d in enumerate(want) if d]
+            ref_o, ref_l = _masked_one(qf, kf, vf, h, i, ids, causal)
+            rows = slice(i * 128, (i + 1) * 128)
+            err = np.abs(out[h, rows] - ref_o)
+            worst_max = max(worst_max, err.max())
+            sum_abs += err.sum()
+            n_el += err.size
+            worst_lse = max(worst_lse, np.abs(lse[h, rows] - ref_l).max())
+    assert worst_max < OUT_MAX, worst_max
+    assert sum_abs / n_el < OUT_MEAN, sum_abs / n_el
+    assert worst_lse < LSE_TOL, worst_lse
+    return dict(max_abs=worst_max, mean_abs=sum_abs / n_el, lse=worst_lse, near_margin=free)
+
+
+def _masked_one(qf, kf, vf, h, i, ids, causal):
+    """Oracle masked attention of one (head, query block) over key blocks `ids`."""
+    G = qf.shape[0] // kf.shape[0]
+    o, l = O.masked_attention(qf[h:h + 1], kf[h // G:h // G + 1], vf[h // G:h // G + 1], [[ids]], causal=causal,
+                              query_blocks=[i])
+    return o[0], l[0]
+
+
+# ---------------------------------------------------------------------------------- fixtures
+@pytest.fixture(scope="module")
+def small():
+    w = tiny(seed=21, hq=4, hkv=2, n=1024, needles=2)
+    qb, kb, vb, _ = w.make()
+    return dict(w=w, dev=tuple(to_dev(x) for x in (qb, kb, vb)), f64=widen(qb, kb, vb))
+
+
+@pytest.fixture(scope="module")
+def cfg1():
+    w = WORKLOADS["gqa4_4k"]
+    qb, kb, vb, _ = w.make()
+    return dict(w=w, dev=tuple(to_dev(x) for x in (qb, kb, vb)), f64=widen(qb, kb, vb))
+
+
+# ---------------------------------------------------------------------------------- KAP
+@pytest.mark.parametrize("stride", [8, 16, 32, 128])
+@pytest.mark.parametrize("budget", [0.1, 0.5, 1.0])
+def test_kap_lists_bit_exact_small(small, stride, budget):
+    q, k, _ = small["dev"]
+    qf, kf, _ = small["f64"]
+    order, count = run_kap(q, k, budget, stride)
+    ref_order, ref_count = O.kap_select(qf, kf, s=stride, budget=budget, order_stride=order.shape[-1])
+    assert np.array_equal(_np(count), ref_count)
+    assert np.array_equal(_np(order), ref_order)
+
+
+def test_kap_noncausal_and_narrow_pitch(small):
+    q, k, _ = small["dev"]
+    qf, kf, _ = small["f64"]
+    order, count = run_kap(q, k, 0.4, 8, causal=False, order_stride=5)
+    ref_order, ref_count = O.kap_select(qf, kf, s=8, budget=0.4, causal=False, order_stride=5)
+    assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    # a pitch that cannot hold the longest list is refused before anything is launched
+    order, count = alloc_lists(4, 8, 3)
+    with pytest.raises(cosa.CosaError) as e:
+        cosa.cosa_kap_select(q, k, 0.5, order, count, opt=cosa.default_options())
+    assert e.value.status == -1
+
+
+def test_kap_exported_scores_and_flags(small):
+    q, k, _ = small["dev"]
+    qf, kf, _ = small["f64"]
+    order, count, ex = run_kap(q, k, 0.5, 8, scores=True)
+    sc, fl = _np(ex["kap_scores"]), _np(ex["kap_flags"])
+    for h in range(4):
+        for i in range(8):
+            s_ref, f_ref, _ = O.kap_scores(qf, kf, h, i, 8)
+            assert np.allclose(sc[h, i, :i + 1], s_ref, rtol=1e-6, atol=0)
+            assert np.array_equal(fl[h, i, :i + 1].astype(bool), f_ref)
+
+
+def test_kap_lists_bit_exact_4k(cfg1):
+    w = cfg1["w"]
+    q, k, _ = cfg1["dev"]
+    qf, kf, _ = cfg1["f64"]
+    order, count = run_kap(q, k, w.kap_budget, w.stride)
+    ref_order, ref_count, audit = O.kap_select(qf, kf, s=w.stride, budget=w.kap_budget, order_stride=w.n_blocks,
+                                               audit=True)
+    assert audit["min_rel_score_gap"] > 1e-9 and audit["min_row_top2_gap"] > 1e-9   # inputs are well conditioned
+    assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+
+
+# ---------------------------------------------------------------------------------- OSK
+@pytest.mark.parametrize("impl", IMPLS)
+def test_osk_dense_path_matches_dense_attention(small, impl):
+    """Full lists, Stage 2 off: the library's dense path (Property 2, Eq. 4)."""
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    rng = np.random.default_rng(0)
+    ref_o, ref_l = O.dense_attention(qf, kf, vf)
+    for permute in (False, True):
+        order_np = np.full((4, 8, 8), -1, np.int32)
+        count_np = np.zeros((4, 8), np.int32)
+        for h in range(4):
+            for i in range(8):
+                ids = rng.permutation(i + 1) if permute else np.arange(i + 1)
+                order_np[h, i, :i + 1], count_np[h, i] = ids, i + 1
+        order = torch.from_numpy(order_np).cuda()[None].contiguous()
+        count = torch.from_numpy(count_np).cuda()[None].contiguous()
+        bufs = run_osk(q, k, v, order, count, 1.0, 2000.0, impl)
+        err = np.abs(_np(bufs["out"].float()) - ref_o)
+        assert err.max() < OUT_MAX and err.mean() < OUT_MEAN
+        assert np.abs(_np(bufs["lse"]) - ref_l).max() < LSE_TOL
+        assert np.array_equal(_np(bufs["visited"]), count_np) and np.array_equal(_np(bufs["scored"]), count_np)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("tb,skip_scale", [(0.3, 200.0), (0.999, 100.0), (0.2, -1.0), (1.0, 200.0), (0.05, 500.0)])
+def test_osk_skip_rule_and_cap_small(small, impl, tb, skip_scale):
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    order_np, count_np = O.kap_select(qf, kf, s=8, budget=0.75)
+    order = torch.from_numpy(order_np).cuda()[None].contiguous()
+    count = torch.from_numpy(count_np).cuda()[None].contiguous()
+    bufs = run_osk(q, k, v, order, count, tb, skip_scale, impl)
+    check_osk_against_oracle(qf, kf, vf, order_np, count_np, bufs, tb, skip_scale, range(4), range(8))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_osk_4k_workload(cfg1, impl):
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    qf, kf, vf = cfg1["f64"]
+    order, count = run_kap(q, k, w.kap_budget, w.stride)
+    bufs = run_osk(q, k, v, order, count, w.osk_budget, w.skip_scale, impl)
+    stats = check_osk_against_oracle(qf, kf, vf, _np(order), _np(count), bufs, w.osk_budget, w.skip_scale,
+                                     range(w.hq), range(w.n_blocks))
+    assert int(_np(bufs["visited"]).sum()) < int(_np(count).sum())        # Stage 2 removed something
+    print("4k", stats)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_osk_noncausal(small, impl):
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    order_np, count_np = O.kap_select(qf, kf, s=8, budget=0.6, causal=False)
+    order = torch.from_numpy(order_np).cuda()[None].contiguous()
+    count = torch.from_numpy(count_np).cuda()[None].contiguous()
+    bufs = run_osk(q, k, v, order, count, 0.5, 300.0, impl, causal=False)
+    check_osk_against_oracle(qf, kf, vf, order_np, count_np, bufs, 0.5, 300.0, range(4), range(8), causal=False)
+
+
+def test_osk_is_deterministic(cfg1):
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    order, count = run_kap(q, k, w.kap_budget, w.stride)
+    a = run_osk(q, k, v, order, count, w.osk_budget, w.skip_scale)
+    b = run_osk(q, k, v, order, count, w.osk_budget, w.skip_scale)
+    assert torch.equal(a["out"], b["out"]) and torch.equal(a["lse"], b["lse"]) and torch.equal(a["visited"], b["visited"])
+
+
+# ---------------------------------------------------------------------------------- boundary
+def test_validator_flags_bad_lists(small):
+    q, k, _ = small["dev"]
+    shape = cosa.make_shape(q, k, True)
+    order, count = run_kap(q, k, 0.5, 8)
+    status = torch.full((1,), 5, dtype=torch.int32, device="cuda")
+    cosa.cosa_validate_order(order, count, shape, status)
+    assert int(status.item()) == 0
+    bad = order.clone()
+    bad[0, 1, 3, 0] = 4                               # key block 4 > query block 3 under a causal mask
+    cosa.cosa_validate_order(bad, count, shape, status)
+    assert int(status.item()) == -6
+    badc = count.clone()
+    badc[0, 0, 0] = 0
+    cosa.cosa_validate_order(order, badc, shape, status)
+    assert int(status.item()) == -6
+
+
+def test_host_call_equals_device_calls(small):
+    w = small["w"]
+    q, k, v = small["dev"]
+    order, count = run_kap(q, k, 0.5, 8)
+    ref = run_osk(q, k, v, order, count, 0.3, 200.0)
+    shape = cosa.make_shape(q, k, True)
+    opt = cosa.default_options(skip_scale=200.0)
+    ws = torch.empty(cosa.cosa_host_call_workspace_bytes(shape, opt), dtype=torch.uint8, device="cuda")
+    qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
+    out_h = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty(ref["lse"].shape, dtype=torch.float32).pin_memory()
+    vis_h = torch.empty(ref["visited"].shape, dtype=torch.int32).pin_memory()
+    cosa.cosa_prefill_host(qh, kh, vh, shape, 0.5, 0.3, out_h, lse_h, vis_h, ws, opt=opt)
+    assert cosa.cosa_device_status() == 0
+    assert torch.equal(out_h, ref["out"].cpu()) and torch.equal(lse_h, ref["lse"].cpu())
+    assert torch.equal(vis_h, ref["visited"].cpu())
+    small_ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(cosa.CosaError) as e:
+        cosa.cosa_prefill_host(qh, kh, vh, shape, 0.5, 0.3, out_h, lse_h, vis_h, small_ws, opt=opt)
+    assert e.value.status == -3
