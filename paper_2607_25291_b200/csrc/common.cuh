@@ -69,6 +69,7 @@ int32_t* device_status_word();
 cudaError_t launch_kap_exact(const KapParams& p, cudaStream_t st);
 size_t kap_exact_smem_bytes(int rows, int nqb);
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
+cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
 cudaError_t launch_validate_order(const int32_t* order, const int32_t* count, int total_qb, int nqb,
                                   int causal, int order_stride, int32_t* status, cudaStream_t st);
 
