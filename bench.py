@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the CoSA prefill hot path (KAP + OSK) on B200.
+
+One "step" = one pass of the whole hot path (cosa_kap_select then cosa_osk_attention)
+over one synthetic attention layer.  The headline workload is the Qwen3-8B-shaped layer
+at 128K tokens (32 query / 8 KV heads, d = 128, causal, block 128, KAP budget 10 %,
+OSK budget 4 %).  `value` is the visited-block TFLOP/s of the whole job: 2*128*128*128
+FLOPs per block whose logits OSK formed plus the same per block it computed, summed over
+all ranks, divided by the (max over ranks) time of KAP + OSK.  With N > 1 every rank
+processes its own layer (independent seeds): weak scaling, no data-path collective.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+BLOCK_FLOPS = 2.0 * 128 * 128 * 128          # one 128x128x128 tile contraction
+METRIC = "osk_kap_prefill_visited_block_tflops"
+UNIT = "TFLOP/s"
+FP64_ALU_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 148 SMs x 64 FP64 FMA/clk x max SM clock
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_128k")
+    ap.add_argument("--no-comparators", action="store_true", help="skip the dense-path and SDPA timings")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        self.lines = []
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def order_pitch(cosa, budget, nqb):
+    return (cosa.cosa_budget_count(budget, nqb) + 7) // 8 * 8
+
+
+def cpu_oracle_sample(w, qb, kb, vb, seconds_hint=20.0):
+    """Times the fp64 oracle (as it stands) on a bounded sample of the workload: KAP lists and the
+    OSK walk of a few (head, query block) pairs.  Returns visited-block TFLOP/s of the sample."""
+    from oracle import cosa_oracle as O
+    from synth.generator import bf16_bits_to_f64
+    nqb = w.n_blocks
+    heads = sorted(set([0, w.hq // 2, w.hq - 1]))
+    blocks = sorted(set([nqb - 1, (3 * nqb) // 4, nqb // 2, nqb // 4]))
+    hkv_used = sorted(set(h // (w.hq // w.hkv) for h in heads))
+    # widen only the heads the sample touches (the full tensors would need tens of GB in fp64)
+    qf = {h: bf16_bits_to_f64(qb[h]) for h in heads}
+    kf = {g: bf16_bits_to_f64(kb[g]) for g in hkv_used}
+    vf = {g: bf16_bits_to_f64(vb[g]) for g in hkv_used}
+    t0 = time.perf_counter()
+    flops = 0.0
+    n_pairs = 0
+    for h in heads:
+        g = h // (w.hq // w.hkv)
+        q1, k1, v1 = qf[h][None], kf[g][None], vf[g][None]
+        order, count = O.kap_select(q1, k1, s=w.stride, budget=w.kap_budget, query_blocks=blocks,
+                                    order_stride=O.budget_count(w.kap_budget, nqb))
+        r = O.osk_attention(q1, k1, v1, order, count, skip_scale=w.skip_scale, tightened_budget=w.osk_budget,
+                            query_blocks=blocks)
+        flops += BLOCK_FLOPS * float(r["scored"].sum() + r["visited"].sum())
+        n_pairs += len(blocks)
+        if time.perf_counter() - t0 > seconds_hint:
+            break
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    return {"value": flops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"KAP lists + OSK walk of {n_pairs} (head, query block) pairs of {w.name} "
+                      f"(heads {heads[:len(heads)]}, query blocks {blocks}) in {dt:.1f} s",
+            "seconds": dt, "flops": flops}
+
+
+def run_reference(args, rank, world):
+    """The base contract's reference arm: here the fp64 oracle on the host cores."""
+    if rank != 0:
+        return
+    from synth.configs import WORKLOADS
+    w = WORKLOADS[args.workload]
+    qb, kb, vb, _ = w.make()
+    for _ in range(max(0, min(args.warmup, 1))):
+        cpu_oracle_sample(w, qb, kb, vb, seconds_hint=5.0)
+    tot_flops, tot_s, last = 0.0, 0.0, None
+    for _ in range(args.steps):
+        last = cpu_oracle_sample(w, qb, kb, vb, seconds_hint=max(5.0, 120.0 / max(args.steps, 1)))
+        tot_flops += last["flops"]; tot_s += last["seconds"]
+    value = tot_flops / tot_s / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_s / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "kap_budget": w.kap_budget,
+                       "osk_budget": w.osk_budget, "stride": w.stride, "skip_scale": w.skip_scale,
+                       "note": "each step is a bounded sample of the workload run by the fp64 oracle on host cores"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle",
+                             "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2607_25291_b200 import build as _build
+    if rank == 0 or world == 1:
+        _build.build()
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    else:
+        torch.cuda.set_device(0)
+    import paper_2607_25291_b200 as cosa
+    from synth.configs import WORKLOADS
+    dev = torch.device("cuda", local_rank if world > 1 else 0)
+    w = WORKLOADS[args.workload]
+    nqb = w.n_blocks
+
+    # ---- synthetic inputs (rank r = its own layer of the same shape: independent problems)
+    t_gen = time.perf_counter()
+    import dataclasses
+    qb, kb, vb, _ = w.make(layer=rank) if w.layers > 1 else dataclasses.replace(w, seed=w.seed + rank).make()
+    t_gen = time.perf_counter() - t_gen
+    pin = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)[None].contiguous().pin_memory()
+    qh, kh, vh = pin(qb), pin(kb), pin(vb)
+    q, k, v = (t.to(dev, non_blocking=True) for t in (qh, kh, vh))
+    pitch = order_pitch(cosa, w.kap_budget, nqb)
+    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device=dev)
+    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
+    out = torch.empty_like(q)
+    lse = torch.empty(1, w.hq, w.n, dtype=torch.float32, device=dev)
+    visited = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
+    scored = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
+    opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=scored)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if cosa.cosa_device_status() != 0:
+        raise RuntimeError("device status reports a timed-out wait")
+    n_scored, n_computed = int(scored.sum().item()), int(visited.sum().item())
+    n_listed = int(count.sum().item())
+    flops_step = BLOCK_FLOPS * (n_scored + n_computed)
+
+    # ---- timed region: K steps, CUDA events on the launching stream, max over ranks
+    sampler = ClockSampler(local_rank if world > 1 else 0)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sync_all()
+    sampler.start()
+    t_wall = time.perf_counter()
+    for s in range(args.steps):
+        ev[s][0].record(stream)
+        cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=opt, stream=stream)
+        ev[s][1].record(stream)
+        cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
+        ev[s][2].record(stream)
+    sync_all()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    kap_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    osk_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    if cosa.cosa_device_status() != 0:
+        raise RuntimeError("device status reports a timed-out wait")
+    tot = torch.tensor([total_ms, flops_step, kap_ms, osk_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        mx = tot.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = tot.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        total_ms, job_flops_step = float(mx[0]), float(sm[1])
+    else:
+        job_flops_step = flops_step
+    ms_per_step = total_ms / args.steps
+    value = job_flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end through the host-buffer entry point (H2D of q,k,v and D2H of the results in the timed region)
+    e2e = None
+    if not args.no_e2e:
+        shape = cosa.make_shape(q, k, True)
+        ws = torch.empty(cosa.cosa_host_call_workspace_bytes(shape, opt), dtype=torch.uint8, device=dev)
+        out_h = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
+        lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+        vis_h = torch.empty(visited.shape, dtype=torch.int32).pin_memory()
+        ke = max(1, min(args.steps, 3))
+        cosa.cosa_prefill_host(qh, kh, vh, shape, w.kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(ke):
+            cosa.cosa_prefill_host(qh, kh, vh, shape, w.kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
+        e1.record(stream)
+        sync_all()
+        e2e_ms = e0.elapsed_time(e1) / ke
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        h2d = (qh.numel() + kh.numel() + vh.numel()) * 2
+        d2h = out_h.numel() * 2 + lse_h.numel() * 4 + vis_h.numel() * 4
+        e2e = {"value": job_flops_step / (float(t[0]) * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": float(t[0]),
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": ke}
+        del ws
+
+    # ---- rooflines (fractions "of measured" unless the peaks file is absent)
+    peaks = measured_peaks()
+    tensor_peak = peaks["bf16_tflops_sustained"]       # kernels are timed inside a back-to-back step loop
+    osk_tflops = flops_step / (osk_ms * 1e-3) / 1e12
+    pairs = w.hq * (nqb * (nqb + 1) // 2)
+    R = 128 // w.stride
+    kap_flops = 2.0 * R * R * 128 * pairs
+    kap_tflops = kap_flops / (kap_ms * 1e-3) / 1e12
+    kap_bytes = (w.hq + w.hkv) * (w.n // w.stride) * 128 * 2 + order.numel() * 4 + count.numel() * 4
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f)
+    roof_osk = {"kernel": "osk_tc_kernel", "bound": "tensor", "achieved": osk_tflops, "peak": tensor_peak,
+                "unit": "TFLOP/s", "frac": osk_tflops / tensor_peak, "peak_source": peaks["source"] + " (sustained bf16)",
+                "frac_of_burst": osk_tflops / peaks["bf16_tflops"], "frac_of_nominal_2250": osk_tflops / 2250.0,
+                "traffic": (traffic or {}).get("osk_tc_kernel")}
+    roof_kap = {"kernel": "kap_exact_kernel", "bound": "alu", "achieved": kap_tflops, "peak": FP64_ALU_PEAK_TFLOPS,
+                "unit": "TFLOP/s", "frac": kap_tflops / FP64_ALU_PEAK_TFLOPS,
+                "peak_source": "derived: 148 SMs x 64 FP64 FMA/clk x 1965 MHz",
+                "hbm_gbs_on_algorithmic_bytes": kap_bytes / (kap_ms * 1e-3) / 1e9,
+                "hbm_frac_of_measured": kap_bytes / (kap_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                "traffic": (traffic or {}).get("kap_exact_kernel")}
+    roofline = roof_osk if osk_ms >= kap_ms else roof_kap
+
+    extras = {}
+    if rank == 0 and world == 1 and not args.no_comparators:
+        # the library's own dense path: full causal lists, Stage 2 off, same kernel
+        full = torch.full((1, w.hq, nqb, nqb), -1, dtype=torch.int32, device=dev)
+        tri = torch.arange(nqb, device=dev, dtype=torch.int32)
+        full[:] = torch.where(tri[None, :] <= tri[:, None], tri[None, :].expand(nqb, nqb), torch.full((), -1, dtype=torch.int32, device=dev))
+        fcount = (tri + 1).expand(1, w.hq, nqb).contiguous()
+        dopt = cosa.default_options(order_stride=nqb)
+        dense_out = torch.empty_like(q)
+        def dense():
+            cosa.cosa_osk_attention(q, k, v, full, fcount, 1.0, dense_out, None, None, opt=dopt, stream=stream)
+        def sdpa():
+            return torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True)
+        for name, fn in (("dense_path", dense), ("sdpa", sdpa)):
+            try:
+                fn(); torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); fn(); fn(); b.record(stream); torch.cuda.synchronize()
+                ms = a.elapsed_time(b) / 2
+                dense_flops = 2 * BLOCK_FLOPS * pairs
+                extras[name] = {"ms": ms, "tflops": dense_flops / (ms * 1e-3) / 1e12, "speedup_of_cosa_path": ms / ms_per_step}
+            except Exception as exc:  # a comparator must not take the benchmark down
+                extras[name] = {"error": str(exc)[:200]}
+        del full, dense_out
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_oracle_sample(w, qb, kb, vb)
+        cpu = {k_: cpu[k_] for k_ in ("value", "unit", "cores", "kind", "sample")}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
+                           "kap_budget": w.kap_budget, "osk_budget": w.osk_budget, "stride": w.stride,
+                           "skip_scale": w.skip_scale, "parallelism": f"layer-per-rank x{world}",
+                           "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
+                           "blocks_scored": n_scored, "blocks_computed": n_computed,
+                           "causal_block_pairs": pairs, "input_generation_s": round(t_gen, 1)},
+                "latency_ms": {"kap": kap_ms, "osk": osk_ms, "kap_plus_osk": ms_per_step},
+                "e2e": e2e, "gpu_launches": 2 * args.steps, "clocks": clocks, "roofline": roofline,
+                "roofline_osk": roof_osk, "roofline_kap": roof_kap, "cpu_baseline": cpu, "comparators": extras,
+                "wall_s_timed_region": t_wall}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
