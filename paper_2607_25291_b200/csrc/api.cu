@@ -80,7 +80,20 @@ cosa_options resolve_options(const cosa_options* opt) {
 }  // namespace
 
 // scratch the kernels of one call need (beyond inputs and outputs)
-static size_t kap_scratch_bytes(const cosa_shape*, const cosa_options&) { return 0; }
+struct KapScratch { size_t scores, jstar, redo, total; };
+static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
+  KapScratch L{};
+  const int stride = o.stride > 0 ? o.stride : 8;
+  const size_t nqb = s->n / kBlock, heads = (size_t)s->batch * s->hq;
+  if (o.impl == 1 || stride < 1 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv)) return L;  // exact kernel: none
+  size_t off = 0;
+  L.scores = off; off += align_up(heads * nqb * nqb * 4, 256);
+  L.jstar = off; off += align_up(heads * (s->n / stride) * 4, 256);
+  L.redo = off; off += align_up(heads * nqb, 256);
+  L.total = off;
+  return L;
+}
+static size_t kap_scratch_bytes(const cosa_shape* s, const cosa_options& o) { return kap_scratch_layout(s, o).total; }
 static size_t osk_scratch_bytes(const cosa_shape*, const cosa_options&) { return 0; }
 
 }  // namespace cosa
@@ -138,8 +151,39 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   // the list of the longest row must fit the pitch
   if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
   if (kap_exact_smem_bytes(p.rows, nqb) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
-  cudaError_t e = launch_kap_exact(p, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return cuda_fail(e, "kap launch");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const KapScratch L = kap_scratch_layout(shape, o);
+  if (L.total == 0) {   // double precision throughout
+    cudaError_t e = launch_kap_exact(p, nullptr, st);
+    if (e != cudaSuccess) return cuda_fail(e, "kap launch");
+    return COSA_OK;
+  }
+  // float32 screen on the tensor cores, then sort + double-precision recount of near ties, then
+  // the double-precision kernel for the few query blocks the screen could not settle
+  char* ws = static_cast<char*>(o.workspace);
+  if (ws) {
+    if (o.workspace_bytes < L.total || !aligned16(ws)) return COSA_ERR_WORKSPACE;
+  } else {
+    void* own = nullptr;
+    rc = own_scratch(L.total, &own);
+    if (rc != COSA_OK) return rc;
+    ws = static_cast<char*>(own);
+  }
+  KapScreenParams sp{};
+  sp.q = p.q; sp.k = p.k;
+  sp.scores = reinterpret_cast<float*>(ws + L.scores);
+  sp.jstar = reinterpret_cast<int32_t*>(ws + L.jstar);
+  sp.redo = reinterpret_cast<uint8_t*>(ws + L.redo);
+  sp.batch = p.batch; sp.hq = p.hq; sp.hkv = p.hkv; sp.n = p.n; sp.nqb = nqb;
+  sp.causal = p.causal; sp.stride = s;
+  sp.scale = (float)p.scale;
+  sp.tau_row = 1e-4f;
+  cudaError_t e = launch_kap_screen(sp, st);
+  if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");
+  e = launch_kap_sort(p, sp, 1.220703125e-4f, st);
+  if (e != cudaSuccess) return cuda_fail(e, "kap sort launch");
+  e = launch_kap_exact(p, sp.redo, st);
+  if (e != cudaSuccess) return cuda_fail(e, "kap recount launch");
   return COSA_OK;
 }
 

@@ -29,6 +29,20 @@ struct KapParams {
   double scale;          // softmax scale applied to the sampled logits
 };
 
+// The float32 screen of the KAP fast path (tensor cores) and what it leaves for the sort stage.
+struct KapScreenParams {
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* k;
+  float* scores;         // [B,Hq,nQB,nQB]  +-s_ij in float32, negative sign = HRM flag
+  int32_t* jstar;        // [B,Hq,N/s]      block holding each sampled row's maximum
+  uint8_t* redo;         // [B,Hq,nQB]      1 = hand this query block to the double-precision kernel
+  int batch, hq, hkv, n, nqb;
+  int causal;
+  int stride;
+  float scale;
+  float tau_row;         // two block maxima of a row closer than this (scaled logits) are "too close to call"
+};
+
 struct OskParams {
   const __nv_bfloat16* q;
   const __nv_bfloat16* k;
@@ -66,7 +80,12 @@ inline long long budget_to_fx(float budget) {
 // device status word (one per device), set by kernels whose bounded waits give up
 int32_t* device_status_word();
 
-cudaError_t launch_kap_exact(const KapParams& p, cudaStream_t st);
+// redo == nullptr: every (head, query block); else only those with redo[...] != 0
+cudaError_t launch_kap_exact(const KapParams& p, const uint8_t* redo, cudaStream_t st);
+bool kap_screen_supported(int rows, int group);
+cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
+// sorts the screened scores, recomputes near-ties in double precision, writes the lists
+cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st);
 size_t kap_exact_smem_bytes(int rows, int nqb);
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);

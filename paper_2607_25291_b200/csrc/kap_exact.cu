@@ -18,7 +18,7 @@ __device__ __forceinline__ bool sorts_before(unsigned long long ka, unsigned ia,
 }
 
 // smem: Qs[R][kPad] | Ks[KB*R][kPad] | Z[KB*R*R] | M[R][Jpad] | Mstar[R] | sort keys | sort ids
-__global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb_per_iter, int sort_cap) {
+__global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, const uint8_t* redo, int kb_per_iter, int sort_cap) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.rows;
   const int i = p.nqb - 1 - (int)blockIdx.x;  // longest lists first
@@ -27,6 +27,7 @@ __global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb
   const int J = p.causal ? i + 1 : p.nqb;
   const int Jpad = p.nqb | 1;
   const int tid = threadIdx.x;
+  if (redo && !redo[(size_t)(b * p.hq + h) * p.nqb + i]) return;  // uniform over the CTA
 
   double* Qs = reinterpret_cast<double*>(smem_raw);
   double* Ks = Qs + (size_t)R * kPad;
@@ -154,12 +155,12 @@ size_t kap_exact_smem_bytes(int rows, int nqb) {
   return doubles * 8 + (size_t)sort_cap * 12;
 }
 
-cudaError_t launch_kap_exact(const KapParams& p, cudaStream_t st) {
+cudaError_t launch_kap_exact(const KapParams& p, const uint8_t* redo, cudaStream_t st) {
   size_t smem = kap_exact_smem_bytes(p.rows, p.nqb);
   cudaError_t e = cudaFuncSetAttribute(kap_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.nqb, p.hq, p.batch);
-  kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, kb_per_iter_for(p.rows), next_pow2(p.nqb));
+  kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, redo, kb_per_iter_for(p.rows), next_pow2(p.nqb));
   return cudaGetLastError();
 }
 

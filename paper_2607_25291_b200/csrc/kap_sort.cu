@@ -1,0 +1,212 @@
+// KAP fast path, stage B: flag-grouped sort and budget prefix (Eqs. 13-14; Algorithm A step 5)
+// on the float32 screen, with a double-precision recount of every decision a rounding error
+// could change.
+//
+// One CTA per (query head, query block).  The candidates are sorted by (HRM flag descending,
+// float32 score descending, block id ascending).  Two neighbours of the sorted order that carry
+// the same flag and whose scores differ by less than tau_score (relative) are a "near tie"; a
+// maximal chain of near ties that starts inside the kept prefix (or straddles its end) is
+// recounted: for each of its blocks M[r,j] is recomputed with double-precision FMAs on the exact
+// bf16 inputs (in the same order as the double-precision kernel), M*[r] is recomputed from the
+// block the screen found to hold the row's maximum, and the chain is re-sorted by the
+// double-precision score.  Everything outside such chains is ordered as exact arithmetic would
+// order it, provided the screen's error stays below tau_score / 2 -- which the tests check.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace cosa {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxTied = 96;
+constexpr int kPad = kHeadDim + 1;
+
+struct Tied { int pos; unsigned id; double s; };
+
+__global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap, int tie_bytes) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);      // [sort_cap]
+  unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);            // [sort_cap]
+  double* Qs = reinterpret_cast<double*>(tie + tie_bytes);                            // [R][kPad]
+  double* Z = Qs + (size_t)p.rows * kPad;                                            // [R][R]
+  double* Mrow = Z + (size_t)p.rows * p.rows;                                        // [R]
+  double* Mstar = Mrow + p.rows;                                                     // [R]
+  __shared__ Tied tied[kMaxTied];
+  __shared__ int n_tied, tail_end;
+
+  const int R = p.rows;
+  const int i = p.nqb - 1 - (int)blockIdx.x;
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int g = h / (p.hq / p.hkv);
+  const int J = p.causal ? i + 1 : p.nqb;
+  const int tid = threadIdx.x;
+  const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
+  if (sp.redo[row]) return;  // a sampled row's two best blocks were too close: left to the double-precision kernel
+
+  const float* srow = sp.scores + row * p.nqb;
+  int P2 = 2;
+  while (P2 < J) P2 <<= 1;
+  for (int j = tid; j < P2; j += kThreads) {
+    unsigned long long key = 0ULL;
+    if (j < J) {
+      const float v = srow[j];
+      const unsigned hi = (__float_as_uint(fabsf(v))) | (v < 0.f ? 0x80000000u : 0u);
+      key = ((unsigned long long)hi << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
+      if (p.dbg_scores) p.dbg_scores[row * p.nqb + j] = fabsf(v);
+      if (p.dbg_flags) p.dbg_flags[row * p.nqb + j] = v < 0.f ? 1 : 0;
+    }
+    keys[j] = key;
+  }
+  if (tid == 0) { n_tied = 0; tail_end = 0; }
+  __syncthreads();
+  for (int k = 2; k <= P2; k <<= 1) {
+    for (int js = k >> 1; js > 0; js >>= 1) {
+      for (int t = tid; t < P2; t += kThreads) {
+        const int u = t ^ js;
+        if (u > t) {
+          const unsigned long long a = keys[t], c = keys[u];
+          const bool up = (t & k) == 0;               // descending order inside "up" segments
+          if (up ? (c > a) : (a > c)) { keys[t] = c; keys[u] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  const int K = budget_count_fx(p.budget_fx, J);
+  // near ties between sorted neighbours
+  for (int t = tid; t < P2; t += kThreads) {
+    unsigned char nt = 0;
+    if (t + 1 < J) {
+      const unsigned ha = (unsigned)(keys[t] >> 32), hb = (unsigned)(keys[t + 1] >> 32);
+      if ((ha >> 31) == (hb >> 31)) {
+        const float sa = __uint_as_float(ha & 0x7fffffffu), sb = __uint_as_float(hb & 0x7fffffffu);
+        nt = (sa - sb <= tau_score * sa) ? 1 : 0;
+      }
+    }
+    tie[t] = nt;
+  }
+  __syncthreads();
+  if (tid == 0) {   // a chain that straddles the end of the kept prefix reaches past it
+    int e = K;
+    while (e < J && tie[e - 1]) ++e;
+    tail_end = e;
+  }
+  __syncthreads();
+  for (int t = tid; t < tail_end; t += kThreads) {
+    const bool in_chain = (t > 0 && tie[t - 1]) || tie[t];
+    if (in_chain && (t < K || t < tail_end)) {
+      const int slot = atomicAdd(&n_tied, 1);
+      if (slot < kMaxTied) { tied[slot].pos = t; tied[slot].id = 0xffffffffu - (unsigned)(keys[t] & 0xffffffffu); }
+    }
+  }
+  __syncthreads();
+  const int nt = n_tied;
+  if (nt > kMaxTied) {          // pathological: too many near ties, let the double-precision kernel do it all
+    if (tid == 0) sp.redo[row] = 1;
+    return;
+  }
+  int32_t* dst = p.order + row * p.order_stride;
+  if (nt > 0) {
+    const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+    const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
+    const int32_t* jst = sp.jstar + (size_t)(b * p.hq + h) * (p.n / p.stride) + (size_t)i * R;
+    for (int e = tid; e < R * kHeadDim; e += kThreads) {
+      const int r = e / kHeadDim, d = e % kHeadDim;
+      Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i * R + r) * p.stride) * kHeadDim + d]);
+    }
+    __syncthreads();
+    // round -1: M*[r] from the block holding row r's maximum; rounds 0..nt-1: the chained blocks
+    for (int round = -1; round < nt; ++round) {
+      for (int e = tid; e < R * R; e += kThreads) {
+        const int r = e / R, c = e % R;
+        const int jb = round < 0 ? jst[r] : (int)tied[round].id;
+        const int kc = jb * R + c;                                    // sampled key index
+        double z = -INFINITY;
+        if (!p.causal || kc <= i * R + r) {
+          const uint4* src = reinterpret_cast<const uint4*>(kh + ((size_t)kc * p.stride) * kHeadDim);
+          const double* qr = Qs + r * kPad;
+          double acc = 0.0;
+#pragma unroll 4
+          for (int c8 = 0; c8 < kHeadDim / 8; ++c8) {
+            const uint4 wv = src[c8];
+            const unsigned ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              acc = fma(qr[c8 * 8 + 2 * u], (double)__uint_as_float(ww[u] << 16), acc);
+              acc = fma(qr[c8 * 8 + 2 * u + 1], (double)__uint_as_float(ww[u] & 0xffff0000u), acc);
+            }
+          }
+          z = acc * p.scale;
+        }
+        Z[r * R + c] = z;
+      }
+      __syncthreads();
+      if (tid < R) {
+        double m = Z[tid * R];
+        for (int c = 1; c < R; ++c) m = fmax(m, Z[tid * R + c]);
+        if (round < 0) Mstar[tid] = m; else Mrow[tid] = m;
+      }
+      __syncthreads();
+      if (round >= 0 && tid == 0) {
+        double s = 0.0;
+        for (int r = 0; r < R; ++r) s += exp(Mrow[r] - Mstar[r]);
+        tied[round].s = s;
+      }
+      __syncthreads();
+    }
+    if (tid == 0) {
+      // order the chained entries by position, then re-sort every chain by (score desc, id asc)
+      for (int a = 1; a < nt; ++a) {
+        Tied x = tied[a];
+        int c = a - 1;
+        while (c >= 0 && tied[c].pos > x.pos) { tied[c + 1] = tied[c]; --c; }
+        tied[c + 1] = x;
+      }
+      int a = 0;
+      while (a < nt) {
+        int e = a;
+        while (e + 1 < nt && tied[e + 1].pos == tied[e].pos + 1 && tie[tied[e].pos]) ++e;
+        const int first_pos = tied[a].pos;
+        for (int x = a + 1; x <= e; ++x) {          // insertion sort of one chain, positions stay
+          const unsigned idx = tied[x].id; const double sx = tied[x].s;
+          int c = x - 1;
+          while (c >= a && (tied[c].s < sx || (tied[c].s == sx && tied[c].id > idx))) {
+            tied[c + 1].id = tied[c].id; tied[c + 1].s = tied[c].s; --c;
+          }
+          tied[c + 1].id = idx; tied[c + 1].s = sx;
+        }
+        for (int x = a; x <= e; ++x) {
+          const int pos = first_pos + (x - a);
+          keys[pos] = (keys[pos] & 0xffffffff00000000ULL) | (unsigned long long)(0xffffffffu - tied[x].id);
+        }
+        a = e + 1;
+      }
+    }
+    __syncthreads();
+  }
+  for (int t = tid; t < p.order_stride; t += kThreads)
+    dst[t] = (t < K) ? (int32_t)(0xffffffffu - (unsigned)(keys[t] & 0xffffffffu)) : -1;
+  if (tid == 0) p.count[row] = K;
+}
+
+int next_pow2(int x) {
+  int v = 2;
+  while (v < x) v <<= 1;
+  return v;
+}
+
+}  // namespace
+
+cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st) {
+  const int cap = next_pow2(p.nqb);
+  const int tie_bytes = (cap + 15) / 16 * 16;
+  size_t smem = (size_t)cap * 8 + tie_bytes + ((size_t)p.rows * kPad + (size_t)p.rows * p.rows + 2 * p.rows) * 8;
+  cudaError_t e = cudaFuncSetAttribute(kap_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(p.nqb, p.hq, p.batch);
+  kap_sort_kernel<<<grid, kThreads, smem, st>>>(p, sp, tau_score, cap, tie_bytes);
+  return cudaGetLastError();
+}
+
+}  // namespace cosa
