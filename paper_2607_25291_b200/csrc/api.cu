@@ -80,7 +80,7 @@ cosa_options resolve_options(const cosa_options* opt) {
 }  // namespace
 
 // scratch the kernels of one call need (beyond inputs and outputs)
-struct KapScratch { size_t scores, jstar, redo, total; };
+struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, total; };
 static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
   KapScratch L{};
   const int stride = o.stride > 0 ? o.stride : 8;
@@ -88,8 +88,10 @@ static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o)
   if (o.impl == 1 || stride < 1 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv)) return L;  // exact kernel: none
   size_t off = 0;
   L.scores = off; off += align_up(heads * nqb * nqb * 4, 256);
-  L.jstar = off; off += align_up(heads * (s->n / stride) * 4, 256);
-  L.redo = off; off += align_up(heads * nqb, 256);
+  L.jstar = off; off += align_up(heads * (s->n / stride) * 8, 256);
+  L.ambmask = off; off += align_up(heads * nqb * 4, 256);
+  L.hard = off; off += align_up(heads * nqb, 256);
+  L.redo_list = off; off += align_up((1 + heads * nqb) * 4, 256);
   L.total = off;
   return L;
 }
@@ -173,7 +175,9 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.q = p.q; sp.k = p.k;
   sp.scores = reinterpret_cast<float*>(ws + L.scores);
   sp.jstar = reinterpret_cast<int32_t*>(ws + L.jstar);
-  sp.redo = reinterpret_cast<uint8_t*>(ws + L.redo);
+  sp.ambmask = reinterpret_cast<uint32_t*>(ws + L.ambmask);
+  sp.hard = reinterpret_cast<uint8_t*>(ws + L.hard);
+  sp.redo_list = reinterpret_cast<int32_t*>(ws + L.redo_list);
   sp.batch = p.batch; sp.hq = p.hq; sp.hkv = p.hkv; sp.n = p.n; sp.nqb = nqb;
   sp.causal = p.causal; sp.stride = s;
   sp.scale = (float)p.scale;
@@ -182,7 +186,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");
   e = launch_kap_sort(p, sp, 1.220703125e-4f, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap sort launch");
-  e = launch_kap_exact(p, sp.redo, st);
+  e = launch_kap_exact(p, sp.redo_list, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap recount launch");
   return COSA_OK;
 }

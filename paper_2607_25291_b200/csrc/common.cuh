@@ -34,8 +34,10 @@ struct KapScreenParams {
   const __nv_bfloat16* q;
   const __nv_bfloat16* k;
   float* scores;         // [B,Hq,nQB,nQB]  +-s_ij in float32, negative sign = HRM flag
-  int32_t* jstar;        // [B,Hq,N/s]      block holding each sampled row's maximum
-  uint8_t* redo;         // [B,Hq,nQB]      1 = hand this query block to the double-precision kernel
+  int32_t* jstar;        // [B,Hq,N/s,2]    blocks holding each sampled row's largest / second largest block maximum
+  uint32_t* ambmask;     // [B,Hq,nQB]      bit r: sampled row r's two best blocks are too close to call in float32
+  uint8_t* hard;         // [B,Hq,nQB]      1 = three blocks too close on some row: whole query block goes to double precision
+  int32_t* redo_list;    // [1 + B*Hq*nQB]  [0] = number of entries, then flat (b*Hq+h)*nQB+i of query blocks to redo
   int batch, hq, hkv, n, nqb;
   int causal;
   int stride;
@@ -80,8 +82,8 @@ inline long long budget_to_fx(float budget) {
 // device status word (one per device), set by kernels whose bounded waits give up
 int32_t* device_status_word();
 
-// redo == nullptr: every (head, query block); else only those with redo[...] != 0
-cudaError_t launch_kap_exact(const KapParams& p, const uint8_t* redo, cudaStream_t st);
+// redo_list == nullptr: every (head, query block); else only the listed ones (count in [0])
+cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st);
 bool kap_screen_supported(int rows, int group);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
 // sorts the screened scores, recomputes near-ties in double precision, writes the lists

@@ -18,16 +18,32 @@ __device__ __forceinline__ bool sorts_before(unsigned long long ka, unsigned ia,
 }
 
 // smem: Qs[R][kPad] | Ks[KB*R][kPad] | Z[KB*R*R] | M[R][Jpad] | Mstar[R] | sort keys | sort ids
-__global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, const uint8_t* redo, int kb_per_iter, int sort_cap) {
+__device__ void kap_exact_item(const KapParams& p, int b, int h, int i, int kb_per_iter, int sort_cap);
+
+// grid (nQB, Hq, B): one CTA per (head, query block)
+__global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb_per_iter, int sort_cap) {
+  kap_exact_item(p, blockIdx.z, blockIdx.y, p.nqb - 1 - (int)blockIdx.x, kb_per_iter, sort_cap);
+}
+
+// 1-d grid: the CTAs share out the entries of a redo list (usually empty)
+__global__ void __launch_bounds__(kThreads) kap_exact_list_kernel(KapParams p, const int32_t* redo_list, int kb_per_iter,
+                                                                 int sort_cap) {
+  const int n = redo_list[0];
+  for (int e = blockIdx.x; e < n; e += gridDim.x) {
+    const int flat = redo_list[1 + e];
+    const int i = flat % p.nqb, bh = flat / p.nqb;
+    kap_exact_item(p, bh / p.hq, bh % p.hq, i, kb_per_iter, sort_cap);
+    __syncthreads();
+  }
+}
+
+__device__ void kap_exact_item(const KapParams& p, const int b, const int h, const int i, int kb_per_iter, int sort_cap) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int R = p.rows;
-  const int i = p.nqb - 1 - (int)blockIdx.x;  // longest lists first
-  const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.hq / p.hkv);
   const int J = p.causal ? i + 1 : p.nqb;
   const int Jpad = p.nqb | 1;
   const int tid = threadIdx.x;
-  if (redo && !redo[(size_t)(b * p.hq + h) * p.nqb + i]) return;  // uniform over the CTA
 
   double* Qs = reinterpret_cast<double*>(smem_raw);
   double* Ks = Qs + (size_t)R * kPad;
@@ -155,12 +171,18 @@ size_t kap_exact_smem_bytes(int rows, int nqb) {
   return doubles * 8 + (size_t)sort_cap * 12;
 }
 
-cudaError_t launch_kap_exact(const KapParams& p, const uint8_t* redo, cudaStream_t st) {
+cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st) {
   size_t smem = kap_exact_smem_bytes(p.rows, p.nqb);
+  if (redo_list) {
+    cudaError_t e = cudaFuncSetAttribute(kap_exact_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kap_exact_list_kernel<<<148, kThreads, smem, st>>>(p, redo_list, kb_per_iter_for(p.rows), next_pow2(p.nqb));
+    return cudaGetLastError();
+  }
   cudaError_t e = cudaFuncSetAttribute(kap_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.nqb, p.hq, p.batch);
-  kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, redo, kb_per_iter_for(p.rows), next_pow2(p.nqb));
+  kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, kb_per_iter_for(p.rows), next_pow2(p.nqb));
   return cudaGetLastError();
 }
 

@@ -12,8 +12,10 @@
 // the key tiles twice: pass 1 finds, per sampled row, the largest and second largest block
 // maximum and the block holding the largest; pass 2 forms the block scores and HRM flags.
 // Float32 results are a SCREEN: the sort stage recomputes in double precision whatever a
-// rounding error could reorder, and a query block with a sampled row whose two best blocks are
-// closer than kTauRow is handed to the double-precision kernel as a whole.
+// rounding error could reorder.  For that it is told, per sampled row, the two blocks with the
+// largest block maxima and whether they are closer than tau_row (the row's HRM flag and M* are
+// then settled in double precision); three such blocks on one row send the whole query block to
+// the double-precision kernel.
 #include <math.h>
 
 #include "common.cuh"
@@ -74,6 +76,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   if (s_poisoned != 0) return;
 
   if (threadIdx.x == 0) {
+    if (blockIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
     mbar_init(smem_u32(&ctl->a_full), 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), 128); }
@@ -145,8 +148,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const int c_limit = p.causal ? r_glob : ns - 1;      // last sampled key this row may see
     const int J = p.causal ? i + 1 : p.nqb;
     constexpr int BPC = 32 / R;                          // key blocks per 32-column chunk
-    float top1 = -INFINITY, top2 = -INFINITY;
-    int jstar = 0;
+    float top1 = -INFINITY, top2 = -INFINITY, top3 = -INFINITY;
+    int jstar = 0, jstar2 = 0;
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = p.scale * kLog2e;
     float* srow = p.scores + ((size_t)(b * p.hq + h) * p.nqb + (row_ok ? i : 0)) * p.nqb;
@@ -157,11 +160,17 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       if (t == n_tiles) {
         // end of pass 1: the row's best block, and whether the runner-up is too close to call
         const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
-        unsigned any_amb = __ballot_sync(0xffffffffu, amb);
-        const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << ((lane / R) * R));
+        const bool amb3 = row_ok && (top1 - top3) * p.scale <= p.tau_row;
+        const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);
+        const int shift = (lane / R) * R;
+        const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << shift);
         if (row_ok) {
-          p.jstar[(size_t)(b * p.hq + h) * ns + r_glob] = jstar;
-          if (r == 0) p.redo[(size_t)(b * p.hq + h) * p.nqb + i] = (any_amb & grp_mask) ? 1 : 0;
+          int2 js = make_int2(jstar, jstar2);
+          reinterpret_cast<int2*>(p.jstar)[(size_t)(b * p.hq + h) * ns + r_glob] = js;
+          if (r == 0) {
+            p.ambmask[(size_t)(b * p.hq + h) * p.nqb + i] = (any_amb & grp_mask) >> shift;
+            p.hard[(size_t)(b * p.hq + h) * p.nqb + i] = (any_amb3 & grp_mask) ? 1 : 0;
+          }
         }
       }
       alive = mbar_wait(smem_u32(&ctl->s_full[sb]), (t >> 1) & 1, abort_flag);
@@ -193,8 +202,10 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
 #pragma unroll
           for (int bb = 0; bb < BPC; ++bb) {
             const float m = mb[bb];
-            if (m > top1) { top2 = top1; top1 = m; jstar = cbase / R + bb; }
-            else if (m > top2) top2 = m;
+            const int jb = cbase / R + bb;
+            if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
+            else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
+            else if (m > top3) top3 = m;
           }
         } else {
 #pragma unroll

@@ -2,15 +2,20 @@
 // on the float32 screen, with a double-precision recount of every decision a rounding error
 // could change.
 //
-// One CTA per (query head, query block).  The candidates are sorted by (HRM flag descending,
-// float32 score descending, block id ascending).  Two neighbours of the sorted order that carry
-// the same flag and whose scores differ by less than tau_score (relative) are a "near tie"; a
-// maximal chain of near ties that starts inside the kept prefix (or straddles its end) is
-// recounted: for each of its blocks M[r,j] is recomputed with double-precision FMAs on the exact
-// bf16 inputs (in the same order as the double-precision kernel), M*[r] is recomputed from the
-// block the screen found to hold the row's maximum, and the chain is re-sorted by the
-// double-precision score.  Everything outside such chains is ordered as exact arithmetic would
-// order it, provided the screen's error stays below tau_score / 2 -- which the tests check.
+// One CTA per (query head, query block).
+//  1. Rows whose two largest block maxima the screen could not tell apart (ambmask) are settled
+//     first: both blocks are re-evaluated with double-precision FMAs on the exact bf16 inputs,
+//     which fixes the row's M* and which block(s) earn the HRM flag from that row (Eq. 12).
+//  2. The candidates are sorted by (HRM flag descending, float32 score descending, block id
+//     ascending).
+//  3. Two sorted neighbours with the same flag whose scores differ by less than tau_score
+//     (relative) are a "near tie"; a maximal chain of near ties that starts inside the kept
+//     prefix (or straddles its end) is recounted: M[r,j] of each of its blocks and M*[r] are
+//     recomputed in double precision (same operation order as the double-precision kernel) and
+//     the chain is re-sorted by the double-precision score, ties by ascending block id.
+// Everything outside such chains is ordered as exact arithmetic would order it provided the
+// screen's error stays below tau_score / 2, which the tests check.  Query blocks the screen
+// marked "hard", or with more chained entries than fit, go to the double-precision kernel.
 #include <math.h>
 
 #include "common.cuh"
@@ -20,19 +25,56 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kMaxTied = 96;
+constexpr int kMaxRows = 32;
 constexpr int kPad = kHeadDim + 1;
 
 struct Tied { int pos; unsigned id; double s; };
 
-__global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap, int tie_bytes) {
+// dest[r] = max over the visible sampled keys c of block jb[r] of (Q~[r] . K~[jb[r]*R + c]) * scale, in double
+// precision; rows with jb[r] < 0 are left alone.  All threads of the CTA call it.
+__device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, const __nv_bfloat16* kh, int i, int R,
+                              const int* jb, double* dest, int tid) {
+  for (int e = tid; e < R * R; e += kThreads) {
+    const int r = e / R, c = e % R;
+    double z = -INFINITY;
+    const int kc = jb[r] * R + c;  // sampled key index
+    if (jb[r] >= 0 && (!p.causal || kc <= i * R + r)) {
+      const uint4* src = reinterpret_cast<const uint4*>(kh + ((size_t)kc * p.stride) * kHeadDim);
+      const double* qr = Qs + r * kPad;
+      double acc = 0.0;
+#pragma unroll 4
+      for (int c8 = 0; c8 < kHeadDim / 8; ++c8) {
+        const uint4 wv = src[c8];
+        const unsigned ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          acc = fma(qr[c8 * 8 + 2 * u], (double)__uint_as_float(ww[u] << 16), acc);
+          acc = fma(qr[c8 * 8 + 2 * u + 1], (double)__uint_as_float(ww[u] & 0xffff0000u), acc);
+        }
+      }
+      z = acc * p.scale;
+    }
+    Z[r * R + c] = z;
+  }
+  __syncthreads();
+  if (tid < R && jb[tid] >= 0) {
+    double m = Z[tid * R];
+    for (int c = 1; c < R; ++c) m = fmax(m, Z[tid * R + c]);
+    dest[tid] = m;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap,
+                                                            int tie_bytes) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);      // [sort_cap]
-  unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);            // [sort_cap]
-  double* Qs = reinterpret_cast<double*>(tie + tie_bytes);                            // [R][kPad]
-  double* Z = Qs + (size_t)p.rows * kPad;                                            // [R][R]
-  double* Mrow = Z + (size_t)p.rows * p.rows;                                        // [R]
-  double* Mstar = Mrow + p.rows;                                                     // [R]
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
+  unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);        // [tie_bytes]
+  double* Qs = reinterpret_cast<double*>(tie + tie_bytes);                       // [R][kPad]
+  double* Z = Qs + (size_t)p.rows * kPad;                                        // [R][R]
   __shared__ Tied tied[kMaxTied];
+  __shared__ double Mrow[kMaxRows], Mstar[kMaxRows], Msecond[kMaxRows];
+  __shared__ int jb[kMaxRows], j1[kMaxRows], j2[kMaxRows];
   __shared__ int n_tied, tail_end;
 
   const int R = p.rows;
@@ -42,7 +84,13 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   const int J = p.causal ? i + 1 : p.nqb;
   const int tid = threadIdx.x;
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  if (sp.redo[row]) return;  // a sampled row's two best blocks were too close: left to the double-precision kernel
+  if (sp.hard[row]) {  // left to the double-precision kernel
+    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row;
+    return;
+  }
+  const unsigned amb = sp.ambmask[row];
+  const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+  const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
 
   const float* srow = sp.scores + row * p.nqb;
   int P2 = 2;
@@ -53,20 +101,72 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
       const float v = srow[j];
       const unsigned hi = (__float_as_uint(fabsf(v))) | (v < 0.f ? 0x80000000u : 0u);
       key = ((unsigned long long)hi << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
-      if (p.dbg_scores) p.dbg_scores[row * p.nqb + j] = fabsf(v);
-      if (p.dbg_flags) p.dbg_flags[row * p.nqb + j] = v < 0.f ? 1 : 0;
     }
     keys[j] = key;
   }
   if (tid == 0) { n_tied = 0; tail_end = 0; }
+  if (tid < R) {
+    const int2 js = reinterpret_cast<const int2*>(sp.jstar)[(size_t)(b * p.hq + h) * (p.n / p.stride) + (size_t)i * R + tid];
+    j1[tid] = js.x; j2[tid] = js.y;
+  }
+  bool have_mstar = false;
+  auto load_q_and_mstar = [&]() {
+    for (int e = tid; e < R * kHeadDim; e += kThreads) {
+      const int r = e / kHeadDim, d = e % kHeadDim;
+      Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i * R + r) * p.stride) * kHeadDim + d]);
+    }
+    if (tid < R) jb[tid] = j1[tid];
+    __syncthreads();
+    f64_block_max(p, Qs, Z, kh, i, R, jb, Mstar, tid);
+    have_mstar = true;
+  };
   __syncthreads();
+
+  if (amb) {
+    // ---- 1. settle the rows the screen could not call
+    load_q_and_mstar();
+    if (tid < R) { jb[tid] = ((amb >> tid) & 1u) ? j2[tid] : -1; Msecond[tid] = -INFINITY; }
+    __syncthreads();
+    f64_block_max(p, Qs, Z, kh, i, R, jb, Msecond, tid);
+    if (tid == 0) {
+      for (int r = 0; r < R; ++r) {
+        if (!((amb >> r) & 1u)) continue;
+        for (int which = 0; which < 2; ++which) {       // the HRM flag of both of the row's contenders
+          const int j = which ? j2[r] : j1[r];
+          bool flag = false;
+          for (int q = 0; q < R && !flag; ++q) {
+            if ((amb >> q) & 1u) {
+              const double best = fmax(Mstar[q], Msecond[q]);
+              flag = (j == j1[q] && Mstar[q] == best) || (j == j2[q] && Msecond[q] == best);
+            } else {
+              flag = (j == j1[q]);
+            }
+          }
+          keys[j] = (keys[j] & 0x7fffffffffffffffULL) | (flag ? 0x8000000000000000ULL : 0ULL);
+        }
+      }
+      for (int r = 0; r < R; ++r)
+        if ((amb >> r) & 1u) Mstar[r] = fmax(Mstar[r], Msecond[r]);
+    }
+    __syncthreads();
+  }
+  if (p.dbg_scores || p.dbg_flags) {
+    for (int j = tid; j < J; j += kThreads) {
+      const unsigned hi = (unsigned)(keys[j] >> 32);
+      if (p.dbg_scores) p.dbg_scores[row * p.nqb + j] = __uint_as_float(hi & 0x7fffffffu);
+      if (p.dbg_flags) p.dbg_flags[row * p.nqb + j] = (unsigned char)(hi >> 31);
+    }
+    __syncthreads();
+  }
+
+  // ---- 2. bitonic sort, descending in (flag, float32 score, -id)
   for (int k = 2; k <= P2; k <<= 1) {
     for (int js = k >> 1; js > 0; js >>= 1) {
       for (int t = tid; t < P2; t += kThreads) {
         const int u = t ^ js;
         if (u > t) {
           const unsigned long long a = keys[t], c = keys[u];
-          const bool up = (t & k) == 0;               // descending order inside "up" segments
+          const bool up = (t & k) == 0;
           if (up ? (c > a) : (a > c)) { keys[t] = c; keys[u] = a; }
         }
       }
@@ -74,7 +174,8 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     }
   }
   const int K = budget_count_fx(p.budget_fx, J);
-  // near ties between sorted neighbours
+
+  // ---- 3. near ties between sorted neighbours
   for (int t = tid; t < P2; t += kThreads) {
     unsigned char nt = 0;
     if (t + 1 < J) {
@@ -87,68 +188,31 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     tie[t] = nt;
   }
   __syncthreads();
-  if (tid == 0) {   // a chain that straddles the end of the kept prefix reaches past it
+  if (tid == 0) {  // a chain that straddles the end of the kept prefix reaches past it
     int e = K;
     while (e < J && tie[e - 1]) ++e;
     tail_end = e;
   }
   __syncthreads();
   for (int t = tid; t < tail_end; t += kThreads) {
-    const bool in_chain = (t > 0 && tie[t - 1]) || tie[t];
-    if (in_chain && (t < K || t < tail_end)) {
+    if ((t > 0 && tie[t - 1]) || tie[t]) {
       const int slot = atomicAdd(&n_tied, 1);
       if (slot < kMaxTied) { tied[slot].pos = t; tied[slot].id = 0xffffffffu - (unsigned)(keys[t] & 0xffffffffu); }
     }
   }
   __syncthreads();
   const int nt = n_tied;
-  if (nt > kMaxTied) {          // pathological: too many near ties, let the double-precision kernel do it all
-    if (tid == 0) sp.redo[row] = 1;
+  if (nt > kMaxTied) {  // pathological: too many near ties
+    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row;
     return;
   }
-  int32_t* dst = p.order + row * p.order_stride;
   if (nt > 0) {
-    const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
-    const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
-    const int32_t* jst = sp.jstar + (size_t)(b * p.hq + h) * (p.n / p.stride) + (size_t)i * R;
-    for (int e = tid; e < R * kHeadDim; e += kThreads) {
-      const int r = e / kHeadDim, d = e % kHeadDim;
-      Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i * R + r) * p.stride) * kHeadDim + d]);
-    }
-    __syncthreads();
-    // round -1: M*[r] from the block holding row r's maximum; rounds 0..nt-1: the chained blocks
-    for (int round = -1; round < nt; ++round) {
-      for (int e = tid; e < R * R; e += kThreads) {
-        const int r = e / R, c = e % R;
-        const int jb = round < 0 ? jst[r] : (int)tied[round].id;
-        const int kc = jb * R + c;                                    // sampled key index
-        double z = -INFINITY;
-        if (!p.causal || kc <= i * R + r) {
-          const uint4* src = reinterpret_cast<const uint4*>(kh + ((size_t)kc * p.stride) * kHeadDim);
-          const double* qr = Qs + r * kPad;
-          double acc = 0.0;
-#pragma unroll 4
-          for (int c8 = 0; c8 < kHeadDim / 8; ++c8) {
-            const uint4 wv = src[c8];
-            const unsigned ww[4] = {wv.x, wv.y, wv.z, wv.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              acc = fma(qr[c8 * 8 + 2 * u], (double)__uint_as_float(ww[u] << 16), acc);
-              acc = fma(qr[c8 * 8 + 2 * u + 1], (double)__uint_as_float(ww[u] & 0xffff0000u), acc);
-            }
-          }
-          z = acc * p.scale;
-        }
-        Z[r * R + c] = z;
-      }
+    if (!have_mstar) load_q_and_mstar();
+    for (int round = 0; round < nt; ++round) {
+      if (tid < R) jb[tid] = (int)tied[round].id;
       __syncthreads();
-      if (tid < R) {
-        double m = Z[tid * R];
-        for (int c = 1; c < R; ++c) m = fmax(m, Z[tid * R + c]);
-        if (round < 0) Mstar[tid] = m; else Mrow[tid] = m;
-      }
-      __syncthreads();
-      if (round >= 0 && tid == 0) {
+      f64_block_max(p, Qs, Z, kh, i, R, jb, Mrow, tid);
+      if (tid == 0) {
         double s = 0.0;
         for (int r = 0; r < R; ++r) s += exp(Mrow[r] - Mstar[r]);
         tied[round].s = s;
@@ -168,8 +232,9 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
         int e = a;
         while (e + 1 < nt && tied[e + 1].pos == tied[e].pos + 1 && tie[tied[e].pos]) ++e;
         const int first_pos = tied[a].pos;
-        for (int x = a + 1; x <= e; ++x) {          // insertion sort of one chain, positions stay
-          const unsigned idx = tied[x].id; const double sx = tied[x].s;
+        for (int x = a + 1; x <= e; ++x) {  // insertion sort of one chain; the positions stay
+          const unsigned idx = tied[x].id;
+          const double sx = tied[x].s;
           int c = x - 1;
           while (c >= a && (tied[c].s < sx || (tied[c].s == sx && tied[c].id > idx))) {
             tied[c + 1].id = tied[c].id; tied[c + 1].s = tied[c].s; --c;
@@ -185,6 +250,7 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     }
     __syncthreads();
   }
+  int32_t* dst = p.order + row * p.order_stride;
   for (int t = tid; t < p.order_stride; t += kThreads)
     dst[t] = (t < K) ? (int32_t)(0xffffffffu - (unsigned)(keys[t] & 0xffffffffu)) : -1;
   if (tid == 0) p.count[row] = K;
@@ -199,9 +265,10 @@ int next_pow2(int x) {
 }  // namespace
 
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st) {
+  if (p.rows > kMaxRows) return cudaErrorInvalidValue;
   const int cap = next_pow2(p.nqb);
   const int tie_bytes = (cap + 15) / 16 * 16;
-  size_t smem = (size_t)cap * 8 + tie_bytes + ((size_t)p.rows * kPad + (size_t)p.rows * p.rows + 2 * p.rows) * 8;
+  size_t smem = (size_t)cap * 8 + tie_bytes + ((size_t)p.rows * kPad + (size_t)p.rows * p.rows) * 8;
   cudaError_t e = cudaFuncSetAttribute(kap_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.nqb, p.hq, p.batch);
