@@ -36,7 +36,7 @@ FP64_ALU_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12   # 148 SMs x 64 FP64 FMA/c
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_128k")
@@ -70,7 +70,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
@@ -116,19 +116,18 @@ def cpu_oracle_sample(w, qb, kb, vb, seconds_hint=20.0):
     from oracle import cosa_oracle as O
     from synth.generator import bf16_bits_to_f64
     nqb = w.n_blocks
-    heads = sorted(set([0, w.hq // 2, w.hq - 1]))
-    blocks = sorted(set([nqb - 1, (3 * nqb) // 4, nqb // 2, nqb // 4]))
-    hkv_used = sorted(set(h // (w.hq // w.hkv) for h in heads))
-    # widen only the heads the sample touches (the full tensors would need tens of GB in fp64)
-    qf = {h: bf16_bits_to_f64(qb[h]) for h in heads}
-    kf = {g: bf16_bits_to_f64(kb[g]) for g in hkv_used}
-    vf = {g: bf16_bits_to_f64(vb[g]) for g in hkv_used}
+    G = w.hq // w.hkv
+    heads = [g * G + (g % G) for g in range(w.hkv)] + [h for h in range(w.hq) if h % G != (h // G) % G]
+    blocks = sorted(set(int(x) for x in np.linspace(nqb // 48, nqb - 1, 48)))
     t0 = time.perf_counter()
     flops = 0.0
     n_pairs = 0
+    used = []
     for h in heads:
-        g = h // (w.hq // w.hkv)
-        q1, k1, v1 = qf[h][None], kf[g][None], vf[g][None]
+        g = h // G
+        # widen one head at a time (the full tensors would need tens of GB in fp64); widening is timed too
+        q1, k1, v1 = bf16_bits_to_f64(qb[h])[None], bf16_bits_to_f64(kb[g])[None], bf16_bits_to_f64(vb[g])[None]
+        used.append(h)
         order, count = O.kap_select(q1, k1, s=w.stride, budget=w.kap_budget, query_blocks=blocks,
                                     order_stride=O.budget_count(w.kap_budget, nqb))
         r = O.osk_attention(q1, k1, v1, order, count, skip_scale=w.skip_scale, tightened_budget=w.osk_budget,
@@ -144,8 +143,8 @@ def cpu_oracle_sample(w, qb, kb, vb, seconds_hint=20.0):
     except Exception:
         cores = os.cpu_count()
     return {"value": flops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"KAP lists + OSK walk of {n_pairs} (head, query block) pairs of {w.name} "
-                      f"(heads {heads[:len(heads)]}, query blocks {blocks}) in {dt:.1f} s",
+            "sample": f"KAP lists + OSK walk of {n_pairs} (head, query block) pairs of {w.name}: heads {used} x "
+                      f"{len(blocks)} query blocks evenly spaced in [{blocks[0]}, {blocks[-1]}], {dt:.1f} s of numpy fp64",
             "seconds": dt, "flops": flops}
 
 

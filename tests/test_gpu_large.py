@@ -1,0 +1,127 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times: the CUDA path runs the
+whole workload, the fp64 oracle re-derives a sample of (head, query block) pairs one by one -- all heads x
+query blocks {0, 1, 2, every 37th, last 3} -- plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_25291_b200 as cosa
+from oracle import cosa_oracle as O
+from synth.configs import SWEEP_STAGE1, SWEEP_STAGE2_MULT, WORKLOADS
+from synth.generator import bf16_bits_to_f64
+from tests.helpers import to_dev
+from tests.test_gpu_parity import _np, check_osk_against_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_blocks(nqb):
+    return sorted(set([0, 1, 2] + list(range(37, nqb, 37)) + [nqb - 3, nqb - 2, nqb - 1]))
+
+
+class HeadView:
+    """Presents one query head (and its KV head) of the bf16 bit tensors as the fp64 arrays the oracle takes."""
+    def __init__(self, qb, kb, vb):
+        self.qb, self.kb, self.vb = qb, kb, vb
+        self.G = qb.shape[0] // kb.shape[0]
+        self.cache = {}
+
+    def get(self, h):
+        g = h // self.G
+        if ("q", h) not in self.cache:
+            self.cache = {k: v for k, v in self.cache.items() if k[0] != "q"}
+            self.cache[("q", h)] = bf16_bits_to_f64(self.qb[h])[None]
+        if ("kv", g) not in self.cache:
+            self.cache = {k: v for k, v in self.cache.items() if k[0] != "kv"}
+            self.cache[("kv", g)] = (bf16_bits_to_f64(self.kb[g])[None], bf16_bits_to_f64(self.vb[g])[None])
+        return (self.cache[("q", h)],) + self.cache[("kv", g)]
+
+
+def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, blocks, check_all_kap=False):
+    q, k, v = (to_dev(x) for x in (qb, kb, vb))
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(kap_budget, nqb) + 7) // 8 * 8
+    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+    bufs = dict(out=torch.empty_like(q), lse=torch.empty(1, w.hq, w.n, dtype=torch.float32, device="cuda"),
+                visited=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                scored=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                decisions=torch.zeros(1, w.hq, nqb, (pitch + 31) // 32, dtype=torch.int32, device="cuda"))
+    opt = cosa.default_options(stride=w.stride, skip_scale=skip_scale, order_stride=pitch,
+                               out_scored=bufs["scored"], out_decisions=bufs["decisions"])
+    cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt)
+    cosa.cosa_osk_attention(q, k, v, order, count, osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+    assert cosa.cosa_device_status() == 0
+    # properties at full size
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cosa.cosa_validate_order(order, count, cosa.make_shape(q, k, True), status)
+    assert int(status.item()) == 0
+    order_np, count_np = _np(order), _np(count)
+    J = np.arange(1, nqb + 1)
+    want_count = np.array([O.budget_count(kap_budget, int(j)) for j in J])
+    assert (count_np == want_count[None, :]).all()
+    vis, sco = _np(bufs["visited"]), _np(bufs["scored"])
+    if osk_budget < 1.0:
+        cap = np.minimum(want_count, np.array([O.budget_count(osk_budget, int(j)) for j in J]))
+        assert (vis <= cap[None, :]).all()
+    else:
+        assert (vis == count_np).all()
+    assert (sco <= count_np).all() and (vis >= 1).all() and (vis <= sco).all()
+    assert torch.isfinite(bufs["out"].float()).all() and torch.isfinite(bufs["lse"]).all()
+    for h in range(w.hq):                                   # every list holds distinct ids
+        rows = np.sort(np.where(order_np[h] < 0, np.arange(order_np.shape[-1])[None, :] + 10 ** 6, order_np[h]), axis=1)
+        assert (np.diff(rows, axis=1) != 0).all()
+    # sampled parity against the oracle
+    hv = HeadView(qb, kb, vb)
+    stats = []
+    for h in kap_heads:
+        qf, kf, vf = hv.get(h)
+        ref_order, ref_count = O.kap_select(qf, kf, s=w.stride, budget=kap_budget, order_stride=pitch,
+                                            query_blocks=(None if check_all_kap else blocks))
+        sel = range(nqb) if check_all_kap else blocks
+        for i in sel:
+            assert ref_count[0, i] == count_np[h, i], (h, i)
+            assert np.array_equal(ref_order[0, i], order_np[h, i]), (h, i)
+        one = {k_: t[:, h:h + 1] for k_, t in bufs.items()}
+        stats.append(check_osk_against_oracle(qf, kf, vf, order_np[h:h + 1], count_np[h:h + 1], one, osk_budget,
+                                              skip_scale, [0], blocks))
+    return dict(max_abs=max(s["max_abs"] for s in stats), mean_abs=float(np.mean([s["mean_abs"] for s in stats])),
+                lse=max(s["lse"] for s in stats), near_margin=sum(s["near_margin"] for s in stats),
+                scored=int(sco.sum()), computed=int(vis.sum()), listed=int(count_np.sum()))
+
+
+def test_qwen3_32k_full_kap_and_sampled_osk():
+    w = WORKLOADS["qwen3_32k"]
+    qb, kb, vb, _ = w.make()
+    stats = run_and_check(w, qb, kb, vb, w.kap_budget, w.osk_budget, w.skip_scale, range(w.hq),
+                          sample_blocks(w.n_blocks), check_all_kap=True)
+    assert stats["computed"] < stats["scored"] < stats["listed"]        # both Stage-2 mechanisms are at work
+    print("32k", stats)
+
+
+def test_qwen3_128k_sampled():
+    w = WORKLOADS["qwen3_128k"]
+    qb, kb, vb, _ = w.make()
+    stats = run_and_check(w, qb, kb, vb, w.kap_budget, w.osk_budget, w.skip_scale, range(w.hq),
+                          sample_blocks(w.n_blocks))
+    assert stats["computed"] < stats["scored"]
+    print("128k", stats)
+
+
+def test_llama31_64k_budget_sweep_sampled():
+    w = WORKLOADS["llama31_64k_sweep"]
+    qb, kb, vb, _ = w.make()
+    blocks = sample_blocks(w.n_blocks)[::2]
+    for b1 in SWEEP_STAGE1:
+        for mult in SWEEP_STAGE2_MULT:
+            tb = 1.0 if mult == 1.0 else b1 * mult            # the 1.0x column runs with Stage 2 off
+            stats = run_and_check(w, qb, kb, vb, b1, tb, w.skip_scale, [0, 13, 31], blocks)
+            print("64k sweep", b1, mult, stats)
+
+
+def test_qwen3_128k_stack_layers_sampled():
+    w = WORKLOADS["qwen3_128k_x36"]
+    for layer in (0, 4):                                       # 8 and 128 needle blocks per head
+        qb, kb, vb, _ = w.make(layer=layer)
+        stats = run_and_check(w, qb, kb, vb, w.kap_budget, w.osk_budget, w.skip_scale, [1, 18], sample_blocks(w.n_blocks)[::3])
+        print("128k stack layer", layer, stats)
