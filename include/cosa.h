@@ -119,6 +119,33 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape,
                        const cosa_options* opt);
 
 /*
+ * cosa_kap_select_static -- cosa_kap_select_ex without any device allocation.  (The paper has no
+ * counterpart: this entry point exists for the way the library is hosted, not for the method.)
+ *
+ * For callers that cannot obtain device memory at call time: servers whose own pool took the whole
+ * GPU at start-up, and request loops that must not trigger the device-wide synchronisation of
+ * cudaMalloc/cudaFree.  The scratch the fast KAP path needs between its kernels lives in a fixed
+ * array of cosa_kap_select_static_max_bytes() (4 MiB) inside the library's device image; every GPU
+ * that loads the library holds that array until the process exits.
+ *
+ *   - Arguments and results are those of cosa_kap_select_ex; opt->workspace is ignored.  Inputs and
+ *     outputs are still the caller's buffers.
+ *   - Returns COSA_ERR_WORKSPACE, and enqueues nothing, when cosa_workspace_bytes(0, shape, opt)
+ *     exceeds the array: roughly B*Hq*(N/128)^2*4 bytes, e.g. 8 heads at N = 16384 fit, 32 heads at
+ *     N = 32768 do not.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call before starting any stream capture.
+ *   - All calls on one device share the array, which keeps whatever the last call left in it; the
+ *     kernels overwrite or reset everything they read, so back-to-back calls on one stream are fine,
+ *     but two calls that can overlap on the GPU (different streams, no ordering) race on it.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine.
+ */
+size_t cosa_kap_select_static_max_bytes(void);
+int cosa_kap_select_static(const void* q, const void* k, const cosa_shape* shape, float budget,
+                           int32_t* out_order, int32_t* out_count, void* stream,
+                           const cosa_options* opt);
+
+/*
  * Stage 2 -- cosa_osk_attention (Sec. 4.3; Algorithm A steps 7-21; skip rule Eq. 5).
  *
  * For every (h, i): m = -inf, l = 0, O = 0; for kk = 0 .. count-1: j = order[kk];

@@ -28,7 +28,7 @@ COSA_ERR_BAD_ORDER = -6
 
 EXPORTS = (
     "cosa_default_options", "cosa_workspace_bytes", "cosa_budget_count", "cosa_kap_select",
-    "cosa_kap_select_ex", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_validate_order",
+    "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_validate_order",
     "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status",
     "cosa_last_cuda_error", "cosa_status_string", "cosa_version",
 )
@@ -74,6 +74,10 @@ def _load():
     lib.cosa_budget_count.restype = c_int32
     lib.cosa_kap_select.argtypes = [c_void_p, c_void_p, POINTER(CosaShape), c_float, c_void_p, c_void_p, c_void_p]
     lib.cosa_kap_select_ex.argtypes = lib.cosa_kap_select.argtypes + [POINTER(CosaOptions)]
+    lib.cosa_kap_select_static.argtypes = lib.cosa_kap_select_ex.argtypes
+    lib.cosa_kap_select_static.restype = c_int
+    lib.cosa_kap_select_static_max_bytes.argtypes = []
+    lib.cosa_kap_select_static_max_bytes.restype = c_size_t
     lib.cosa_osk_attention.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(CosaShape), c_void_p, c_void_p, c_float,
                                        c_void_p, c_void_p, c_void_p, c_void_p]
     lib.cosa_osk_attention_ex.argtypes = lib.cosa_osk_attention.argtypes + [POINTER(CosaOptions)]
@@ -157,6 +161,25 @@ def cosa_kap_select(q, k, budget: float, out_order, out_count, causal=True, stre
         if opt.order_stride == 0:
             opt.order_stride = out_order.shape[-1]
         _check(lib.cosa_kap_select_ex(*args, byref(opt)), "cosa_kap_select_ex")
+
+
+def cosa_kap_select_static_max_bytes() -> int:
+    return int(_load().cosa_kap_select_static_max_bytes())
+
+
+def cosa_kap_select_static(q, k, budget: float, out_order, out_count, causal=True, stream=None,
+                           opt: CosaOptions | None = None):
+    """Stage 1 with the library's built-in scratch array: no device allocation (see cosa.h for the size limit)."""
+    lib = _load()
+    shape = make_shape(q, k, causal)
+    if opt is None:
+        opt = default_options()
+    if opt.order_stride == 0:
+        opt.order_stride = out_order.shape[-1]
+    _check(lib.cosa_kap_select_static(_dev_ptr(q, torch.bfloat16, "q"), _dev_ptr(k, torch.bfloat16, "k"), byref(shape),
+                                      c_float(budget), _dev_ptr(out_order, torch.int32, "out_order"),
+                                      _dev_ptr(out_count, torch.int32, "out_count"), _stream_ptr(stream), byref(opt)),
+           "cosa_kap_select_static")
 
 
 def cosa_osk_attention(q, k, v, order, count, tightened_budget: float, out, out_lse=None, out_visited=None,
