@@ -258,13 +258,8 @@ def main():
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     if cosa.cosa_device_status() != 0:
         raise RuntimeError("device status reports a timed-out wait")
-    tot = torch.tensor([total_ms, flops_step, kap_ms, osk_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        mx = tot.clone(); dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = tot.clone(); dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        total_ms, job_flops_step = float(mx[0]), float(sm[1])
-    else:
-        job_flops_step = flops_step
+    from paper_2607_25291_b200.shard import reduce_job
+    total_ms, job_flops_step = reduce_job(total_ms, flops_step, dev)      # max time, summed work over ranks
     ms_per_step = total_ms / args.steps
     value = job_flops_step / (ms_per_step * 1e-3) / 1e12
 
