@@ -4,13 +4,17 @@
 //   warp 0       K loader: one TMA tile load per listed key block ("physical jumping": only the
 //                listed pages are ever touched), running ahead by the number of blocks that are
 //                already certain to be scored
-//   warp 1       MMA issuer: S = Q K_j^T into one of two TMEM buffers, O += P V_j into a third
+//   warp 1       MMA issuer: S = Q K_j^T into one of two TMEM buffers and O += P V_j, issued in
+//                whatever order their operands become ready (a PV product never blocks the next
+//                QK^T while its V tile is still in flight)
 //   warps 2..5   one thread per query row: read S from TMEM, running row maxima, the tile-wide
-//                vote of Eq. (5), and -- only if the block is computed -- exp, row sums, the
-//                rescale of O, P as bf16 back to shared memory, and the V tile load
+//                vote of Eq. (5), and -- only if the block is computed -- the V tile load, exp,
+//                row sums, the rescale of O, and P as bf16 into one of two TMEM buffers, from
+//                where the PV product reads it as its A operand
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
-// expect.  Every wait is bounded; a wait that runs out sets the device status word and the CTA
-// winds down without writing results.
+// expect.  TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
+// Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
+// down without writing results.
 #include <math.h>
 
 #include "common.cuh"
@@ -21,18 +25,19 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kKStages = 2;
-constexpr int kVStages = 2;
+constexpr int kKStages = 3;
+constexpr int kVStages = 3;
 constexpr int kTileBytes = kBlock * kHeadDim * 2;  // 32 KiB: one 128 x 128 bf16 tile
 constexpr int kHalfBytes = kTileBytes / 2;         // one TMA box: 128 rows x 64 columns
 constexpr int kThreads = 192;
 constexpr int kTmemCols = 512;
 constexpr int kDecRing = 64;
 constexpr uint32_t kDecComputed = 1, kDecEnd = 2;
+constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
 struct __align__(8) Control {
   unsigned long long q_full, k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
-  unsigned long long s_full[2], s_empty[2], p_full, p_empty;
+  unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2];
   uint32_t tmem_base;
   volatile int n_needed;  // list positions [0, n_needed) are certain to be scored
   volatile int n_dec;     // decisions published so far
@@ -41,11 +46,16 @@ struct __align__(8) Control {
   float red[2][4];
 };
 
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (1 + kKStages + kVStages + 1) + sizeof(Control);
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (1 + kKStages + kVStages) + sizeof(Control);
 
 __device__ __forceinline__ void report_timeout(Control* c, int32_t* status) {
   c->abort_flag = 1;
   atomicMin(status, (int32_t)COSA_ERR_DEVICE_TIMEOUT);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&t);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -58,9 +68,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t q_sm = base;
   const uint32_t k_sm = q_sm + kTileBytes;
   const uint32_t v_sm = k_sm + kKStages * kTileBytes;
-  const uint32_t p_sm = v_sm + kVStages * kTileBytes;
-  unsigned char* p_ptr = smem + (size_t)kTileBytes * (1 + kKStages + kVStages);
-  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (1 + kKStages + kVStages + 1));
+  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (1 + kKStages + kVStages));
 
   // work item: KV head major, then query blocks from the longest list down, the group's query
   // heads innermost, so that CTAs resident together read the same K/V pages
@@ -92,9 +100,10 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     mbar_init(smem_u32(&ctl->q_full), 1);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&ctl->v_full[s]), 1); mbar_init(smem_u32(&ctl->v_empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kBlock); }
-    mbar_init(smem_u32(&ctl->p_full), kBlock);
-    mbar_init(smem_u32(&ctl->p_empty), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
+      mbar_init(smem_u32(&ctl->p_full[s]), kBlock); mbar_init(smem_u32(&ctl->p_empty[s]), 1);
+    }
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
     ctl->abort_flag = 0;
@@ -112,6 +121,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
+  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 448u};
   volatile int* abort_flag = &ctl->abort_flag;
 
   if (cnt == 0) {
@@ -139,8 +149,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         while (kk >= ctl->n_needed) {          // not yet certain that this block will be scored
           const int nd = ctl->n_dec;
           if (nd > 0 && (ctl->dec[(nd - 1) % kDecRing] & kDecEnd)) { ok = false; break; }
-          if (*abort_flag || clock64() - t0 > (1LL << 31)) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
-          __nanosleep(64);
+          if (*abort_flag || clock64() - t0 > kWaitBudget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+          __nanosleep(32);
         }
         if (!ok && kk >= ctl->n_needed) break;
         const int st = kk % kKStages;
@@ -156,58 +166,69 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer (dataflow order)
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] and K_j [N x K], both K-major
-      const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] K-major, V_j [K x N] N-major
+      const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
       bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
-      int kk_qk = 0, kk_pv = 0, n_pv = 0;
+      int kk_qk = 0;       // next QK^T to issue
+      int kk_seen = 0;     // decisions read so far
+      int n_known = 0;     // computed blocks among them
+      int n_pv = 0;        // PV products issued
+      int n_total = -1;    // number of scored blocks, once the end of the walk is known
+      long long t_last = clock64();
       while (alive) {
-        while (alive && kk_qk < ctl->n_needed && kk_qk - kk_pv < 2) {
+        bool progress = false;
+        const int nd = ctl->n_dec;
+        while (kk_seen < nd) {
+          const uint32_t d = ctl->dec[kk_seen % kDecRing];
+          if (d & kDecComputed) ++n_known;
+          if (d & kDecEnd) n_total = kk_seen + 1;
+          ++kk_seen;
+          progress = true;
+        }
+        if (n_pv < n_known) {
+          const int pb = n_pv & 1, vs = n_pv % kVStages;
+          if (mbar_try_wait(smem_u32(&ctl->p_full[pb]), (n_pv >> 1) & 1) &&
+              mbar_try_wait(smem_u32(&ctl->v_full[vs]), (n_pv / kVStages) & 1)) {
+            tc_fence_after();
+            const uint32_t vt = v_sm + vs * kTileBytes;
+#pragma unroll
+            for (int ks = 0; ks < kBlock / 16; ++ks)  // 16 keys per MMA: 8 TMEM columns of P, 2 KiB of V
+              mma_ts(tmem_o, tmem_p[pb] + ks * 8, smem_desc_sw128(vt + ks * 2048, kHalfBytes, 1024), idesc_pv,
+                     (n_pv > 0) || (ks > 0));
+            mma_commit(smem_u32(&ctl->p_empty[pb]));
+            mma_commit(smem_u32(&ctl->v_empty[vs]));
+            ++n_pv;
+            progress = true;
+          }
+        }
+        if (kk_qk < ctl->n_needed) {
           const int st = kk_qk % kKStages, sb = kk_qk & 1;
-          alive = mbar_wait(smem_u32(&ctl->k_full[st]), (kk_qk / kKStages) & 1, abort_flag) &&
-                  mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk_qk >> 1) & 1) ^ 1, abort_flag);
-          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-          tc_fence_after();
-          const uint32_t kt = k_sm + st * kTileBytes;
+          if (mbar_try_wait(smem_u32(&ctl->k_full[st]), (kk_qk / kKStages) & 1) &&
+              mbar_try_wait(smem_u32(&ctl->s_empty[sb]), ((kk_qk >> 1) & 1) ^ 1)) {
+            tc_fence_after();
+            const uint32_t kt = k_sm + st * kTileBytes;
 #pragma unroll
-          for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-            const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;  // 16 elements of d per MMA
-            mma_ss(tmem_s[sb], smem_desc_sw128(q_sm + off, 16, 1024), smem_desc_sw128(kt + off, 16, 1024), idesc_qk,
-                   ks > 0);
+            for (int ks = 0; ks < kHeadDim / 16; ++ks) {
+              const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;  // 16 elements of d per MMA
+              mma_ss(tmem_s[sb], smem_desc_sw128(q_sm + off, 16, 1024), smem_desc_sw128(kt + off, 16, 1024), idesc_qk,
+                     ks > 0);
+            }
+            mma_commit(smem_u32(&ctl->s_full[sb]));
+            mma_commit(smem_u32(&ctl->k_empty[st]));
+            ++kk_qk;
+            progress = true;
           }
-          mma_commit(smem_u32(&ctl->s_full[sb]));
-          mma_commit(smem_u32(&ctl->k_empty[st]));
-          ++kk_qk;
         }
-        if (!alive) break;
-        // decision of list position kk_pv
-        const long long t0 = clock64();
-        while (ctl->n_dec <= kk_pv) {
-          if (*abort_flag || clock64() - t0 > (1LL << 31)) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+        if (n_total >= 0 && n_pv == n_known && kk_qk >= n_total) break;
+        if (progress) {
+          t_last = clock64();
+        } else if (*abort_flag || clock64() - t_last > kWaitBudget) {
+          if (!*abort_flag) report_timeout(ctl, status);
+          alive = false;
         }
-        if (!alive) break;
-        const uint32_t d = ctl->dec[kk_pv % kDecRing];
-        if (d & kDecComputed) {
-          const int vs = n_pv % kVStages;
-          alive = mbar_wait(smem_u32(&ctl->p_full), n_pv & 1, abort_flag) &&
-                  mbar_wait(smem_u32(&ctl->v_full[vs]), (n_pv / kVStages) & 1, abort_flag);
-          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-          tc_fence_after();
-          const uint32_t vt = v_sm + vs * kTileBytes;
-#pragma unroll
-          for (int ks = 0; ks < kBlock / 16; ++ks) {  // 16 keys per MMA
-            const uint64_t adesc = smem_desc_sw128(p_sm + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024);
-            const uint64_t bdesc = smem_desc_sw128(vt + ks * 2048, kHalfBytes, 1024);
-            mma_ss(tmem_o, adesc, bdesc, idesc_pv, (n_pv > 0) || (ks > 0));
-          }
-          mma_commit(smem_u32(&ctl->p_empty));
-          mma_commit(smem_u32(&ctl->v_empty[vs]));
-          ++n_pv;
-        }
-        ++kk_pv;
-        if (d & kDecEnd) break;
       }
     }
   } else {
@@ -219,12 +240,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
     const float theta2 = p.theta * kLog2e;
-    float m = -INFINITY, l = 0.f;
+    float m = -INFINITY, l = 0.f;             // m in scaled base-2 units
     int computed = 0, n_needed = min(cnt, cap), scored = 0;
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
-    uint32_t s[kBlock];
+    uint32_t s[kBlock];                       // raw logits of this row, then probabilities
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int sb = kk & 1;
       const int j = min(max(list[kk], 0), p.nqb - 1);
@@ -236,15 +257,17 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->s_empty[sb]));   // the buffer may take the logits of block kk+2
-      const bool diag = p.causal && j == i;
-      float m_loc = -INFINITY;
+      if (p.causal && j == i) {                   // token-level causal mask on the diagonal block
 #pragma unroll
-      for (int c = 0; c < kBlock; ++c) {
-        float x = __uint_as_float(s[c]) * scale2;
-        if (diag && c > r) x = -INFINITY;         // token-level causal mask on the diagonal block
-        s[c] = __float_as_uint(x);
-        m_loc = fmaxf(m_loc, x);
+        for (int c = 0; c < kBlock; ++c) if (c > r) s[c] = 0xff800000u;  // -inf
       }
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < kBlock; c += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
+      }
+      const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
       const float m_prev = m;
       m = fmaxf(m, m_loc);
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N)
@@ -279,56 +302,58 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         if (p.decisions && ((kk & 31) == 31 || last)) { p.decisions[row * dec_words + (kk >> 5)] = dec_word; dec_word = 0; }
       }
       if (compute) {
-        const float alpha = exp2f(m_prev - m);    // 0 for the first block, 1 when no row maximum moved
-        float rowsum = 0.f;
+        const float alpha = ex2_approx(m_prev - m);   // 0 for the first block, 1 when no row maximum moved
+        const float neg_m = -m;
+        float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < kBlock; ++c) {
-          float e = exp2f(__uint_as_float(s[c]) - m);
-          rowsum += e;
-          s[c] = __float_as_uint(e);
-        }
-        l = alpha * l + rowsum;
-        if (n_before > 0) {
-          // P buffer free and O up to date once the previous PV product has finished
-          alive = mbar_wait(smem_u32(&ctl->p_empty), (n_before - 1) & 1, abort_flag);
-          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-          tc_fence_after();
-          if (__any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O, only if a row maximum moved
-            uint32_t o[32];
+        for (int c = 0; c < kBlock; c += 4) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              tmem_ld32(tmem_o + lane_addr + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-              tmem_st32(tmem_o + lane_addr + c * 32, o);
-            }
-            tmem_wait_st();
+          for (int u = 0; u < 4; ++u) {
+            const float e = ex2_approx(fmaf(__uint_as_float(s[c + u]), scale2, neg_m));   // exp(S - m)
+            rs[u] += e;
+            s[c + u] = __float_as_uint(e);
           }
         }
-        // P as bf16, row r, in the K-major 128-byte-swizzled layout of an MMA A operand
+        l = alpha * l + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
+        const int pb = n_before & 1;
+        if (n_before > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+          // O = diag(alpha) O: only if a row maximum moved, and only after the previous PV product
+          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag);
+          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+          tc_fence_after();
+          uint32_t o[32];
 #pragma unroll
-        for (int ch = 0; ch < 16; ++ch) {
-          uint4 pk;
-          pk.x = __float_as_uint(0.f);
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(s[ch * 8 + 0]), __uint_as_float(s[ch * 8 + 1]));
-          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(s[ch * 8 + 2]), __uint_as_float(s[ch * 8 + 3]));
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(s[ch * 8 + 4]), __uint_as_float(s[ch * 8 + 5]));
-          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(s[ch * 8 + 6]), __uint_as_float(s[ch * 8 + 7]));
-          pk.x = *reinterpret_cast<uint32_t*>(&t0); pk.y = *reinterpret_cast<uint32_t*>(&t1);
-          pk.z = *reinterpret_cast<uint32_t*>(&t2); pk.w = *reinterpret_cast<uint32_t*>(&t3);
-          const int half = ch >> 3, chunk = ch & 7;
-          *reinterpret_cast<uint4*>(p_ptr + half * kHalfBytes + r * 128 + ((chunk ^ (r & 7)) << 4)) = pk;
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_o + lane_addr + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tmem_o + lane_addr + c * 32, o);
+          }
+          tmem_wait_st();
         }
-        fence_proxy_async_smem();
+        // this P buffer was last read by the PV product two computed blocks ago
+        alive = mbar_wait(smem_u32(&ctl->p_empty[pb]), ((n_before >> 1) & 1) ^ 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        tc_fence_after();
+        // P as bf16: two keys per 32-bit TMEM column, row r in lane r
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t pk[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            pk[e] = pack_bf16(__uint_as_float(s[c * 64 + 2 * e]), __uint_as_float(s[c * 64 + 2 * e + 1]));
+          tmem_st32(tmem_p[pb] + lane_addr + c * 32, pk);
+        }
+        tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(smem_u32(&ctl->p_full));
+        mbar_arrive(smem_u32(&ctl->p_full[pb]));
       }
       if (last) break;
     }
     // ---- epilogue: O / l, LSE, counters
     if (alive && computed > 0) {
-      alive = mbar_wait(smem_u32(&ctl->p_empty), (computed - 1) & 1, abort_flag);
+      alive = mbar_wait(smem_u32(&ctl->p_empty[(computed - 1) & 1]), ((computed - 1) >> 1) & 1, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
     }
     if (alive && !*abort_flag) {
@@ -343,12 +368,10 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 #pragma unroll
         for (int e = 0; e < 32; e += 8) {
           uint4 pk;
-          __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-          __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-          __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-          __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-          pk.x = *reinterpret_cast<uint32_t*>(&t0); pk.y = *reinterpret_cast<uint32_t*>(&t1);
-          pk.z = *reinterpret_cast<uint32_t*>(&t2); pk.w = *reinterpret_cast<uint32_t*>(&t3);
+          pk.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
+          pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+          pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+          pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
           *reinterpret_cast<uint4*>(dst + c * 32 + e) = pk;
         }
       }
