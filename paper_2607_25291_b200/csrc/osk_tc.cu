@@ -1,16 +1,17 @@
 // OSK on the sm_100a tensor cores (Sec. 4.3; Algorithm A steps 7-21; skip rule Eq. 5).
 //
-// One CTA per (query head, query block), six warps:
+// One CTA per (query head, query block), ten warps:
 //   warp 0       K loader: one TMA tile load per listed key block ("physical jumping": only the
 //                listed pages are ever touched), running ahead by the number of blocks that are
 //                already certain to be scored
 //   warp 1       MMA issuer: S = Q K_j^T into one of two TMEM buffers and O += P V_j, issued in
 //                whatever order their operands become ready (a PV product never blocks the next
 //                QK^T while its V tile is still in flight)
-//   warps 2..5   one thread per query row: read S from TMEM, running row maxima, the tile-wide
-//                vote of Eq. (5), and -- only if the block is computed -- the V tile load, exp,
-//                row sums, the rescale of O, and P as bf16 into one of two TMEM buffers, from
-//                where the PV product reads it as its A operand
+//   warps 2..9   two threads per query row (one per 64-column half of the tile, so that every SM
+//                sub-partition holds two such warps and their latencies overlap): read S from
+//                TMEM, running row maxima, the tile-wide vote of Eq. (5), and -- only if the block
+//                is computed -- the V tile load, exp, row sums, the rescale of O, and P as bf16
+//                into one of two TMEM buffers, from where the PV product reads it as its A operand
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
 // expect.  TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
@@ -26,10 +27,11 @@ namespace {
 using namespace ptx;
 
 constexpr int kKStages = 3;
-constexpr int kVStages = 3;
+constexpr int kVStages = 2;
 constexpr int kTileBytes = kBlock * kHeadDim * 2;  // 32 KiB: one 128 x 128 bf16 tile
 constexpr int kHalfBytes = kTileBytes / 2;         // one TMA box: 128 rows x 64 columns
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
+constexpr int kSoftmaxThreads = 256;
 constexpr int kTmemCols = 512;
 constexpr int kDecRing = 64;
 constexpr uint32_t kDecComputed = 1, kDecEnd = 2;
@@ -43,7 +45,9 @@ struct __align__(8) Control {
   volatile int n_dec;     // decisions published so far
   volatile int abort_flag;
   volatile uint32_t dec[kDecRing];
-  float red[2][4];
+  unsigned long long x_bar;  // softmax threads: partial row maxima published (one phase per block)
+  float xch[2][2][kBlock];   // [parity][column half][row]: partial row maxima (raw logits), then partial row sums
+  float mrow[2][kBlock];     // [parity][row]: running row maximum before the block under test
 };
 
 constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (1 + kKStages + kVStages) + sizeof(Control);
@@ -101,9 +105,10 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&ctl->v_full[s]), 1); mbar_init(smem_u32(&ctl->v_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
-      mbar_init(smem_u32(&ctl->p_full[s]), kBlock); mbar_init(smem_u32(&ctl->p_empty[s]), 1);
+      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kSoftmaxThreads);
+      mbar_init(smem_u32(&ctl->p_full[s]), kSoftmaxThreads); mbar_init(smem_u32(&ctl->p_empty[s]), 1);
     }
+    mbar_init(smem_u32(&ctl->x_bar), kSoftmaxThreads);
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
     ctl->abort_flag = 0;
@@ -126,7 +131,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 
   if (cnt == 0) {
     // an empty list (not produced by KAP): zero output, nothing visited
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
       const int r = (warp & 3) * 32 + lane;
       uint4 z = make_uint4(0, 0, 0, 0);
       uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)q_row0 + r) * kHeadDim);
@@ -234,18 +239,19 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else {
     // ------------------------------------------------------------------ softmax / vote rows
     const int sub = warp & 3;                 // this warp may touch TMEM lanes [32*sub, 32*sub+32)
+    const int half = (warp - 2) >> 2;         // which 64 columns of the tile this thread owns
     const int r = sub * 32 + lane;            // query row inside the tile
     const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
     const bool leader = (threadIdx.x == 64);
     const float kLog2e = 1.4426950408889634f;
     const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
     const float theta2 = p.theta * kLog2e;
-    float m = -INFINITY, l = 0.f;             // m in scaled base-2 units
+    float m = -INFINITY, l = 0.f;             // m in scaled base-2 units; l: this thread's half of the row sum
     int computed = 0, n_needed = min(cnt, cap), scored = 0;
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
-    uint32_t s[kBlock];                       // raw logits of this row, then probabilities
+    uint32_t s[64];                           // raw logits of this half row, then probabilities
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int sb = kk & 1;
       const int j = min(max(list[kk], 0), p.nqb - 1);
@@ -253,30 +259,41 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
       tc_fence_after();
 #pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s[sb] + lane_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      for (int c = 0; c < 2; ++c)
+        tmem_ld32(tmem_s[sb] + lane_addr + half * 64 + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->s_empty[sb]));   // the buffer may take the logits of block kk+2
       if (p.causal && j == i) {                   // token-level causal mask on the diagonal block
 #pragma unroll
-        for (int c = 0; c < kBlock; ++c) if (c > r) s[c] = 0xff800000u;  // -inf
+        for (int c = 0; c < 64; ++c) if (half * 64 + c > r) s[c] = 0xff800000u;  // -inf
       }
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < kBlock; c += 4) {
+      for (int c = 0; c < 64; c += 4) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
       }
-      const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
+      const float pm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      ctl->xch[kk & 1][half][r] = pm;
+      if (half == 0) ctl->mrow[kk & 1][r] = m;
+      mbar_arrive(smem_u32(&ctl->x_bar));
+      alive = mbar_wait(smem_u32(&ctl->x_bar), kk & 1, abort_flag);
+      if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+      const float m_loc = fmaxf(pm, ctl->xch[kk & 1][half ^ 1][r]) * scale2;   // scale > 0 commutes with max
       const float m_prev = m;
       m = fmaxf(m, m_loc);
-      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N)
-      float gap = m_loc - m;
+      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N).  Every warp evaluates the
+      // statistic over all 128 rows from the published values (4 rows per lane): no second barrier.
+      float gm = -INFINITY;
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) gap = fmaxf(gap, __shfl_xor_sync(0xffffffffu, gap, o));
-      if (lane == 0) ctl->red[kk & 1][sub] = gap;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      const float gm = fmaxf(fmaxf(ctl->red[kk & 1][0], ctl->red[kk & 1][1]), fmaxf(ctl->red[kk & 1][2], ctl->red[kk & 1][3]));
+      for (int q4 = 0; q4 < 4; ++q4) {
+        const int rr = lane + 32 * q4;
+        const float ml = fmaxf(ctl->xch[kk & 1][0][rr], ctl->xch[kk & 1][1][rr]) * scale2;
+        gm = fmaxf(gm, ml - fmaxf(ctl->mrow[kk & 1][rr], ml));
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
       const bool compute = !(p.use_threshold && gm < theta2);
       ++scored;
       const int n_before = computed;
@@ -306,7 +323,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const float neg_m = -m;
         float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int c = 0; c < kBlock; c += 4) {
+        for (int c = 0; c < 64; c += 4) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
             const float e = ex2_approx(fmaf(__uint_as_float(s[c + u]), scale2, neg_m));   // exp(S - m)
@@ -323,12 +340,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           tc_fence_after();
           uint32_t o[32];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_o + lane_addr + c * 32, o);
+          for (int c = 0; c < 2; ++c) {
+            tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, o);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem_o + lane_addr + c * 32, o);
+            tmem_st32(tmem_o + lane_addr + half * 64 + c * 32, o);
           }
           tmem_wait_st();
         }
@@ -336,14 +353,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         alive = mbar_wait(smem_u32(&ctl->p_empty[pb]), ((n_before >> 1) & 1) ^ 1, abort_flag);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
-        // P as bf16: two keys per 32-bit TMEM column, row r in lane r
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        // P as bf16: two keys per 32-bit TMEM column, row r in lane r; this thread's 64 keys = 32 columns
+        {
           uint32_t pk[32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e)
-            pk[e] = pack_bf16(__uint_as_float(s[c * 64 + 2 * e]), __uint_as_float(s[c * 64 + 2 * e + 1]));
-          tmem_st32(tmem_p[pb] + lane_addr + c * 32, pk);
+          for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(__uint_as_float(s[2 * e]), __uint_as_float(s[2 * e + 1]));
+          tmem_st32(tmem_p[pb] + lane_addr + half * 32, pk);
         }
         tmem_wait_st();
         tc_fence_before();
@@ -356,14 +371,18 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       alive = mbar_wait(smem_u32(&ctl->p_empty[(computed - 1) & 1]), ((computed - 1) >> 1) & 1, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
     }
+    // the two halves of a row add their row sums (every softmax thread reaches this barrier)
+    ctl->xch[0][half][r] = l;
+    asm volatile("bar.sync 2, 256;" ::: "memory");
+    l += ctl->xch[0][half ^ 1][r];
     if (alive && !*abort_flag) {
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* dst = p.out + ((size_t)q_row0 + r) * kHeadDim;
+      __nv_bfloat16* dst = p.out + ((size_t)q_row0 + r) * kHeadDim + half * 64;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t o[32];
-        tmem_ld32(tmem_o + lane_addr + c * 32, o);
+        tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, o);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 32; e += 8) {
@@ -375,7 +394,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           *reinterpret_cast<uint4*>(dst + c * 32 + e) = pk;
         }
       }
-      if (p.lse) p.lse[(size_t)q_row0 + r] = (m + log2f(l)) * 0.6931471805599453f;
+      if (p.lse && half == 0) p.lse[(size_t)q_row0 + r] = (m + log2f(l)) * 0.6931471805599453f;
       if (leader) {
         if (p.visited) p.visited[row] = computed;
         if (p.scored) p.scored[row] = scored;
