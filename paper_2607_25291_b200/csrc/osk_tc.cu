@@ -1,19 +1,29 @@
 // OSK on the sm_100a tensor cores (Sec. 4.3; Algorithm A steps 7-21; skip rule Eq. 5).
 //
-// One CTA per (query head, query block), ten warps:
+// One CTA per (query head, query block), twelve warps in three warp groups (the first gives
+// registers to the other two with setmaxnreg):
 //   warp 0       K loader: one TMA tile load per listed key block ("physical jumping": only the
 //                listed pages are ever touched), running ahead by the number of blocks that are
 //                already certain to be scored
 //   warp 1       MMA issuer: S = Q K_j^T into one of two TMEM buffers and O += P V_j, issued in
-//                whatever order their operands become ready (a PV product never blocks the next
-//                QK^T while its V tile is still in flight)
-//   warps 2..9   two threads per query row (one per 64-column half of the tile, so that every SM
-//                sub-partition holds two such warps and their latencies overlap): read S from
-//                TMEM, running row maxima, the tile-wide vote of Eq. (5), and -- only if the block
-//                is computed -- the V tile load, exp, row sums, the rescale of O, and P as bf16
-//                into one of two TMEM buffers, from where the PV product reads it as its A operand
+//                whatever order their operands become ready.  Both products take their A operand
+//                (Q, resp. P) from tensor memory, so each MMA reads only 4 KiB of shared memory
+//                and the tensor pipe is not held back by operand fetch.
+//   warp 2       controller (see below); warp 3 idle
+//   warps 4..7   softmax group A: list positions 0, 2, 4, ...   (one thread per query row)
+//   warps 8..11  softmax group B: list positions 1, 3, 5, ...
+//                A group copies its S tile from TMEM to registers (freeing the buffer at once),
+//                takes the row maxima, receives the running maxima after the previous position
+//                from the other group, publishes its own, and -- only if the block is computed --
+//                rescales O, forms P = exp(S - m) as bf16 in TMEM and adds row sums.  The two
+//                groups overlap: while one is in its exp phase the other already takes the maxima
+//                of the next block.
+//   controller: the tile-wide vote of Eq. (5) from the published row statistics,
+//                the cap on computed blocks, the V tile load of computed blocks, and the
+//                decisions the other warps follow
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
-// expect.  TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
+// expect; Q goes from global memory through registers straight into TMEM.
+// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P [384,448) Q [448,512).
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
 // down without writing results.
 #include <math.h>
@@ -26,31 +36,37 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kKStages = 3;
+constexpr int kKStages = 4;
 constexpr int kVStages = 2;
 constexpr int kTileBytes = kBlock * kHeadDim * 2;  // 32 KiB: one 128 x 128 bf16 tile
 constexpr int kHalfBytes = kTileBytes / 2;         // one TMA box: 128 rows x 64 columns
-constexpr int kThreads = 320;
-constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
-constexpr int kDecRing = 64;
-constexpr uint32_t kDecComputed = 1, kDecEnd = 2;
+constexpr int kDecRing = 16;
+constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks before this position
 constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
 struct __align__(8) Control {
   unsigned long long q_full, k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
-  unsigned long long s_full[2], s_empty[2], p_full[2], p_empty[2];
+  unsigned long long s_full[2], s_empty[2], p_full;
+  unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1]: a waiter may run two products ahead
+                                  // of the tensor pipe, which one barrier's single parity bit cannot tell apart
+  unsigned long long m_ready[2];  // a group has published the row statistics of its position
+  unsigned long long dec_bar[2];  // the controller has published the decision of that position
+  unsigned long long fin_bar;     // both groups have published their final partial sums
   uint32_t tmem_base;
-  volatile int n_needed;  // list positions [0, n_needed) are certain to be scored
-  volatile int n_dec;     // decisions published so far
+  volatile int n_needed;          // list positions [0, n_needed) are certain to be scored
+  volatile int n_dec;             // decisions published so far
+  volatile int end_kk;            // last scored position, -1 until known
+  volatile int final_computed;
   volatile int abort_flag;
   volatile uint32_t dec[kDecRing];
-  unsigned long long x_bar;  // softmax threads: partial row maxima published (one phase per block)
-  float xch[2][2][kBlock];   // [parity][column half][row]: partial row maxima (raw logits), then partial row sums
-  float mrow[2][kBlock];     // [parity][row]: running row maximum before the block under test
+  float mloc[2][kBlock];          // [position parity][row]: block row maxima (scaled, base 2)
+  float mrow[2][kBlock];          // [position parity][row]: running row maxima including that block
+  float fin_m[2][kBlock], fin_l[2][kBlock];
 };
 
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (1 + kKStages + kVStages) + sizeof(Control);
+constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (kKStages + kVStages) + sizeof(Control);
 
 __device__ __forceinline__ void report_timeout(Control* c, int32_t* status) {
   c->abort_flag = 1;
@@ -62,6 +78,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// bounded spin on a volatile counter: true once *v >= want
+__device__ __forceinline__ bool spin_until_ge(volatile int* v, int want, volatile int* abort_flag) {
+  if (*v >= want) return true;
+  const long long t0 = clock64();
+  while (*v < want) {
+    if (*abort_flag || clock64() - t0 > kWaitBudget) return false;
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, OskParams p, int32_t* status) {
@@ -69,10 +95,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
   unsigned char* smem = smem_raw + (base - raw);
-  const uint32_t q_sm = base;
-  const uint32_t k_sm = q_sm + kTileBytes;
+  const uint32_t k_sm = base;
   const uint32_t v_sm = k_sm + kKStages * kTileBytes;
-  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (1 + kKStages + kVStages));
+  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (kKStages + kVStages));
 
   // work item: KV head major, then query blocks from the longest list down, the group's query
   // heads innermost, so that CTAs resident together read the same K/V pages
@@ -101,20 +126,23 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   if (s_poisoned != 0) return;
 
   if (threadIdx.x == 0) {
-    mbar_init(smem_u32(&ctl->q_full), 1);
+    mbar_init(smem_u32(&ctl->q_full), kBlock);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&ctl->v_full[s]), 1); mbar_init(smem_u32(&ctl->v_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kSoftmaxThreads);
-      mbar_init(smem_u32(&ctl->p_full[s]), kSoftmaxThreads); mbar_init(smem_u32(&ctl->p_empty[s]), 1);
+      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
+      mbar_init(smem_u32(&ctl->m_ready[s]), kBlock); mbar_init(smem_u32(&ctl->dec_bar[s]), 1);
     }
-    mbar_init(smem_u32(&ctl->x_bar), kSoftmaxThreads);
+    mbar_init(smem_u32(&ctl->p_full), kBlock); mbar_init(smem_u32(&ctl->p_empty[0]), 1); mbar_init(smem_u32(&ctl->p_empty[1]), 1);
+    mbar_init(smem_u32(&ctl->fin_bar), 2 * kBlock);
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
+    ctl->end_kk = -1;
+    ctl->final_computed = 0;
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
-    prefetch_tensormap(&q_map); prefetch_tensormap(&k_map); prefetch_tensormap(&v_map);
+    prefetch_tensormap(&k_map); prefetch_tensormap(&v_map);
   }
   if (warp == 0) {
     tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
@@ -126,34 +154,25 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
-  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 448u};
+  const uint32_t tmem_p = tmem + 384u;
+  const uint32_t tmem_q = tmem + 448u;
   volatile int* abort_flag = &ctl->abort_flag;
+  const float kLog2e = 1.4426950408889634f;
+  const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
+  const float theta2 = p.theta * kLog2e;
 
+  // register budget: the control warps need few, the softmax threads hold a whole S row
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
   if (cnt == 0) {
-    // an empty list (not produced by KAP): zero output, nothing visited
-    if (warp >= 2 && warp < 6) {
-      const int r = (warp & 3) * 32 + lane;
-      uint4 z = make_uint4(0, 0, 0, 0);
-      uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)q_row0 + r) * kHeadDim);
-      for (int c = 0; c < kHeadDim / 8; ++c) dst[c] = z;
-      if (p.lse) p.lse[(size_t)q_row0 + r] = -INFINITY;
-      if (threadIdx.x == 64) {
-        if (p.visited) p.visited[row] = 0;
-        if (p.scored) p.scored[row] = 0;
-      }
-    }
   } else if (warp == 0) {
     // ------------------------------------------------------------------ K loader
     if (lane == 0) {
-      mbar_expect_tx(smem_u32(&ctl->q_full), kTileBytes);
-      tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_full));
-      tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, smem_u32(&ctl->q_full));
       for (int kk = 0; kk < cnt; ++kk) {
         const long long t0 = clock64();
         bool ok = true;
         while (kk >= ctl->n_needed) {          // not yet certain that this block will be scored
-          const int nd = ctl->n_dec;
-          if (nd > 0 && (ctl->dec[(nd - 1) % kDecRing] & kDecEnd)) { ok = false; break; }
+          if (ctl->end_kk >= 0) { ok = false; break; }
           if (*abort_flag || clock64() - t0 > kWaitBudget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           __nanosleep(32);
         }
@@ -175,6 +194,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] and K_j [N x K], both K-major
       const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
+      // Q sits in TMEM once the first softmax group has copied it there
       bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
       int kk_qk = 0;       // next QK^T to issue
@@ -194,16 +214,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           progress = true;
         }
         if (n_pv < n_known) {
-          const int pb = n_pv & 1, vs = n_pv % kVStages;
-          if (mbar_try_wait(smem_u32(&ctl->p_full[pb]), (n_pv >> 1) & 1) &&
-              mbar_try_wait(smem_u32(&ctl->v_full[vs]), (n_pv / kVStages) & 1)) {
+          const int vs = n_pv % kVStages;
+          if (mbar_test_wait(smem_u32(&ctl->p_full), n_pv & 1) &&
+              mbar_test_wait(smem_u32(&ctl->v_full[vs]), (n_pv / kVStages) & 1)) {
             tc_fence_after();
             const uint32_t vt = v_sm + vs * kTileBytes;
 #pragma unroll
             for (int ks = 0; ks < kBlock / 16; ++ks)  // 16 keys per MMA: 8 TMEM columns of P, 2 KiB of V
-              mma_ts(tmem_o, tmem_p[pb] + ks * 8, smem_desc_sw128(vt + ks * 2048, kHalfBytes, 1024), idesc_pv,
+              mma_ts(tmem_o, tmem_p + ks * 8, smem_desc_sw128(vt + ks * 2048, kHalfBytes, 1024), idesc_pv,
                      (n_pv > 0) || (ks > 0));
-            mma_commit(smem_u32(&ctl->p_empty[pb]));
+            mma_commit(smem_u32(&ctl->p_empty[n_pv & 1]));
             mma_commit(smem_u32(&ctl->v_empty[vs]));
             ++n_pv;
             progress = true;
@@ -211,15 +231,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         }
         if (kk_qk < ctl->n_needed) {
           const int st = kk_qk % kKStages, sb = kk_qk & 1;
-          if (mbar_try_wait(smem_u32(&ctl->k_full[st]), (kk_qk / kKStages) & 1) &&
-              mbar_try_wait(smem_u32(&ctl->s_empty[sb]), ((kk_qk >> 1) & 1) ^ 1)) {
+          if (mbar_test_wait(smem_u32(&ctl->k_full[st]), (kk_qk / kKStages) & 1) &&
+              mbar_test_wait(smem_u32(&ctl->s_empty[sb]), ((kk_qk >> 1) & 1) ^ 1)) {
             tc_fence_after();
             const uint32_t kt = k_sm + st * kTileBytes;
 #pragma unroll
             for (int ks = 0; ks < kHeadDim / 16; ++ks) {
               const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;  // 16 elements of d per MMA
-              mma_ss(tmem_s[sb], smem_desc_sw128(q_sm + off, 16, 1024), smem_desc_sw128(kt + off, 16, 1024), idesc_qk,
-                     ks > 0);
+              mma_ts(tmem_s[sb], tmem_q + ks * 8, smem_desc_sw128(kt + off, 16, 1024), idesc_qk, ks > 0);
             }
             mma_commit(smem_u32(&ctl->s_full[sb]));
             mma_commit(smem_u32(&ctl->k_empty[st]));
@@ -236,62 +255,21 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         }
       }
     }
-  } else {
-    // ------------------------------------------------------------------ softmax / vote rows
-    const int sub = warp & 3;                 // this warp may touch TMEM lanes [32*sub, 32*sub+32)
-    const int half = (warp - 2) >> 2;         // which 64 columns of the tile this thread owns
-    const int r = sub * 32 + lane;            // query row inside the tile
-    const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
-    const bool leader = (threadIdx.x == 64);
-    const float kLog2e = 1.4426950408889634f;
-    const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
-    const float theta2 = p.theta * kLog2e;
-    float m = -INFINITY, l = 0.f;             // m in scaled base-2 units; l: this thread's half of the row sum
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ controller
     int computed = 0, n_needed = min(cnt, cap), scored = 0;
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
-    uint32_t s[64];                           // raw logits of this half row, then probabilities
     for (int kk = 0; kk < cnt && alive; ++kk) {
-      const int sb = kk & 1;
-      const int j = min(max(list[kk], 0), p.nqb - 1);
-      alive = mbar_wait(smem_u32(&ctl->s_full[sb]), (kk >> 1) & 1, abort_flag);
-      if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-      tc_fence_after();
-#pragma unroll
-      for (int c = 0; c < 2; ++c)
-        tmem_ld32(tmem_s[sb] + lane_addr + half * 64 + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->s_empty[sb]));   // the buffer may take the logits of block kk+2
-      if (p.causal && j == i) {                   // token-level causal mask on the diagonal block
-#pragma unroll
-        for (int c = 0; c < 64; ++c) if (half * 64 + c > r) s[c] = 0xff800000u;  // -inf
-      }
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int c = 0; c < 64; c += 4) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
-      }
-      const float pm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-      ctl->xch[kk & 1][half][r] = pm;
-      if (half == 0) ctl->mrow[kk & 1][r] = m;
-      mbar_arrive(smem_u32(&ctl->x_bar));
-      alive = mbar_wait(smem_u32(&ctl->x_bar), kk & 1, abort_flag);
-      if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-      const float m_loc = fmaxf(pm, ctl->xch[kk & 1][half ^ 1][r]) * scale2;   // scale > 0 commutes with max
-      const float m_prev = m;
-      m = fmaxf(m, m_loc);
-      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N).  Every warp evaluates the
-      // statistic over all 128 rows from the published values (4 rows per lane): no second barrier.
+      const int par = kk & 1;
+      const int j = min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
+      alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag);
+      if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
+      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block
       float gm = -INFINITY;
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        const int rr = lane + 32 * q4;
-        const float ml = fmaxf(ctl->xch[kk & 1][0][rr], ctl->xch[kk & 1][1][rr]) * scale2;
-        gm = fmaxf(gm, ml - fmaxf(ctl->mrow[kk & 1][rr], ml));
-      }
+      for (int q4 = 0; q4 < 4; ++q4) gm = fmaxf(gm, ctl->mloc[par][lane + 32 * q4] - ctl->mrow[par][lane + 32 * q4]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
       const bool compute = !(p.use_threshold && gm < theta2);
@@ -299,7 +277,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const int n_before = computed;
       if (compute) ++computed; else n_needed = min(cnt, n_needed + 1);
       const bool last = (computed == cap) || (kk == cnt - 1);
-      if (leader) {
+      if (lane == 0) {
+        ctl->n_needed = n_needed;
+        ctl->dec[kk % kDecRing] = (compute ? kDecComputed : 0u) | (last ? kDecEnd : 0u) | ((uint32_t)n_before << 8);
+        if (last) ctl->final_computed = computed;
+        mbar_arrive(smem_u32(&ctl->dec_bar[par]));   // release: the waiting group sees the decision
+        __threadfence_block();                       // pollers of the counters below see it too
+        ctl->n_dec = kk + 1;
+        if (last) ctl->end_kk = kk;
         if (compute) {                            // fetch V_j now that the block is known to be computed
           const int vs = n_before % kVStages;
           if (!mbar_wait(smem_u32(&ctl->v_empty[vs]), ((n_before / kVStages) & 1) ^ 1, abort_flag)) {
@@ -312,94 +297,195 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           }
           dec_word |= 1u << (kk & 31);
         }
-        ctl->n_needed = n_needed;
-        ctl->dec[kk % kDecRing] = (compute ? kDecComputed : 0u) | (last ? kDecEnd : 0u);
-        __threadfence_block();
-        ctl->n_dec = kk + 1;
         if (p.decisions && ((kk & 31) == 31 || last)) { p.decisions[row * dec_words + (kk >> 5)] = dec_word; dec_word = 0; }
       }
-      if (compute) {
-        const float alpha = ex2_approx(m_prev - m);   // 0 for the first block, 1 when no row maximum moved
-        const float neg_m = -m;
-        float rs[4] = {0.f, 0.f, 0.f, 0.f};
+      __syncwarp();
+      if (last) break;
+    }
+    if (lane == 0 && alive && !*abort_flag) {
+      if (p.visited) p.visited[row] = computed;
+      if (p.scored) p.scored[row] = scored;
+    }
+  }
+  } else {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+  if (cnt == 0) {
+    // an empty list (not produced by KAP): zero output, nothing visited
+    if (warp < 8) {
+      const int r = (warp & 3) * 32 + lane;
+      uint4 z = make_uint4(0, 0, 0, 0);
+      uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)q_row0 + r) * kHeadDim);
+      for (int c = 0; c < kHeadDim / 8; ++c) dst[c] = z;
+      if (p.lse) p.lse[(size_t)q_row0 + r] = -INFINITY;
+      if (threadIdx.x == 128) {
+        if (p.visited) p.visited[row] = 0;
+        if (p.scored) p.scored[row] = 0;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax groups
+    const int grp = (warp - 4) >> 2;          // 0: even list positions, 1: odd list positions
+    const int sub = warp & 3;                 // this warp may touch TMEM lanes [32*sub, 32*sub+32)
+    const int r = sub * 32 + lane;            // query row inside the tile
+    const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
+    float m_ref = -INFINITY, l = 0.f;         // this group's partial row sum and the maximum it refers to
+    bool alive = true;
+    uint32_t s[kBlock];                       // this row's raw logits, then probabilities
+    if (grp == 0) {
+      // Q row -> TMEM as the A operand of QK^T: lane = row, two consecutive d per 32-bit column
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)q_row0 + r) * kHeadDim);
 #pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const float e = ex2_approx(fmaf(__uint_as_float(s[c + u]), scale2, neg_m));   // exp(S - m)
-            rs[u] += e;
-            s[c + u] = __float_as_uint(e);
+      for (int c = 0; c < 16; ++c) {
+        const uint4 wv = src[c];
+        s[4 * c] = wv.x; s[4 * c + 1] = wv.y; s[4 * c + 2] = wv.z; s[4 * c + 3] = wv.w;
+      }
+      tmem_st32(tmem_q + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_st32(tmem_q + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->q_full));
+    }
+    for (int kk = grp; kk < cnt && alive; kk += 2) {
+      const int j = min(max(list[kk], 0), p.nqb - 1);
+      // wait for S(kk), or learn that the walk ended before this position
+      {
+        const uint32_t bar = smem_u32(&ctl->s_full[grp]), par = (kk >> 1) & 1;
+        bool ended = false;
+        if (!mbar_try_wait(bar, par)) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, par)) {
+            const int e = ctl->end_kk;
+            if (e >= 0 && kk > e) { ended = true; break; }
+            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
-        l = alpha * l + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
-        const int pb = n_before & 1;
-        if (n_before > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-          // O = diag(alpha) O: only if a row maximum moved, and only after the previous PV product
-          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag);
-          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-          tc_fence_after();
+        if (ended || !alive) break;
+      }
+      tc_fence_after();
+      const bool diag = p.causal && j == i;
+      // ---- S row to registers; the TMEM buffer is free for position kk+2 at once
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tmem_s[grp] + lane_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->s_empty[grp]));
+      if (diag) {                                 // token-level causal mask on the diagonal block
+#pragma unroll
+        for (int c = 0; c < kBlock; ++c) if (c > r) s[c] = 0xff800000u;  // -inf
+      }
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < kBlock; c += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
+      }
+      const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
+      // ---- running maximum before this position comes from the other group
+      float m_in = -INFINITY;
+      if (kk > 0) {
+        alive = mbar_wait(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        m_in = ctl->mrow[grp ^ 1][r];
+      }
+      const float m_new = fmaxf(m_in, m_loc);
+      // the controller must have read this slot's previous contents (position kk-2)
+      if (kk >= 2 && !spin_until_ge(&ctl->n_dec, kk - 1, abort_flag)) {
+        alive = false; if (!*abort_flag) report_timeout(ctl, status); break;
+      }
+      ctl->mloc[grp][r] = m_loc;
+      ctl->mrow[grp][r] = m_new;
+      mbar_arrive(smem_u32(&ctl->m_ready[grp]));
+      // ---- the controller's decision
+      alive = mbar_wait(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag);
+      if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+      const uint32_t d = ctl->dec[kk % kDecRing];
+      const bool last = (d & kDecEnd) != 0;
+      if (!(d & kDecComputed)) {                  // skipped: nothing is added to l or O
+        if (last) break;
+        continue;
+      }
+      const int n_before = (int)(d >> 8);
+      // ---- P = exp(S - m), row sums (in registers)
+      const float alpha = ex2_approx(m_in - m_new);   // O refers to m_in: skipped blocks never move the maximum
+      const float neg_m = -m_new;
+      float rs[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < kBlock; c += 4) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float e = ex2_approx(fmaf(__uint_as_float(s[c + u]), scale2, neg_m));
+          rs[u] += e;
+          s[c + u] = __float_as_uint(e);
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < 64; ++c) s[c] = pack_bf16(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1]));
+      // ---- the previous PV product must have finished: P is free and O may be rescaled
+      if (n_before > 0) {
+        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O, only if a row maximum moved
           uint32_t o[32];
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, o);
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_o + lane_addr + c * 32, o);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem_o + lane_addr + half * 64 + c * 32, o);
+            tmem_st32(tmem_o + lane_addr + c * 32, o);
           }
-          tmem_wait_st();
         }
-        // this P buffer was last read by the PV product two computed blocks ago
-        alive = mbar_wait(smem_u32(&ctl->p_empty[pb]), ((n_before >> 1) & 1) ^ 1, abort_flag);
-        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-        tc_fence_after();
-        // P as bf16: two keys per 32-bit TMEM column, row r in lane r; this thread's 64 keys = 32 columns
-        {
-          uint32_t pk[32];
-#pragma unroll
-          for (int e = 0; e < 32; ++e) pk[e] = pack_bf16(__uint_as_float(s[2 * e]), __uint_as_float(s[2 * e + 1]));
-          tmem_st32(tmem_p[pb] + lane_addr + half * 32, pk);
-        }
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctl->p_full[pb]));
       }
+      tmem_st32(tmem_p + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_st32(tmem_p + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->p_full));
+      l = l * ex2_approx(m_ref - m_new) + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
+      m_ref = m_new;
       if (last) break;
     }
-    // ---- epilogue: O / l, LSE, counters
-    if (alive && computed > 0) {
-      alive = mbar_wait(smem_u32(&ctl->p_empty[(computed - 1) & 1]), ((computed - 1) >> 1) & 1, abort_flag);
+    // ---- the two groups combine their partial sums; every softmax thread reaches this point
+    ctl->fin_m[grp][r] = m_ref;
+    ctl->fin_l[grp][r] = l;
+    mbar_arrive(smem_u32(&ctl->fin_bar));
+    if (alive) {
+      alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
     }
-    // the two halves of a row add their row sums (every softmax thread reaches this barrier)
-    ctl->xch[0][half][r] = l;
-    asm volatile("bar.sync 2, 256;" ::: "memory");
-    l += ctl->xch[0][half ^ 1][r];
     if (alive && !*abort_flag) {
-      tc_fence_after();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* dst = p.out + ((size_t)q_row0 + r) * kHeadDim + half * 64;
-#pragma unroll
-      for (int c = 0; c < 2; ++c) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + lane_addr + half * 64 + c * 32, o);
-        tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; e += 8) {
-          uint4 pk;
-          pk.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-          pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-          pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-          pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-          *reinterpret_cast<uint4*>(dst + c * 32 + e) = pk;
-        }
+      const float ma = ctl->fin_m[0][r], mb = ctl->fin_m[1][r];
+      const float mf = fmaxf(ma, mb);            // the running maximum is monotone: this is its final value
+      const float lt = ctl->fin_l[0][r] * ex2_approx(ma - mf) + ctl->fin_l[1][r] * ex2_approx(mb - mf);
+      const int n_comp = ctl->final_computed;
+      if (n_comp > 0) {
+        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag);
+        if (!alive && !*abort_flag) report_timeout(ctl, status);
       }
-      if (p.lse && half == 0) p.lse[(size_t)q_row0 + r] = (m + log2f(l)) * 0.6931471805599453f;
-      if (leader) {
-        if (p.visited) p.visited[row] = computed;
-        if (p.scored) p.scored[row] = scored;
+      if (alive) {
+        tc_fence_after();
+        const float inv = lt > 0.f ? 1.f / lt : 0.f;
+        __nv_bfloat16* dst = p.out + ((size_t)q_row0 + r) * kHeadDim + grp * 64;   // each group writes half the row
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_addr + grp * 64 + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 pk;
+            pk.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
+            pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+            pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+            pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + c * 32 + e) = pk;
+          }
+        }
+        if (p.lse && grp == 0) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
       }
     }
+  }
   }
   tc_fence_before();
   __syncthreads();

@@ -125,3 +125,31 @@ def test_qwen3_128k_stack_layers_sampled():
         qb, kb, vb, _ = w.make(layer=layer)
         stats = run_and_check(w, qb, kb, vb, w.kap_budget, w.osk_budget, w.skip_scale, [1, 18], sample_blocks(w.n_blocks)[::3])
         print("128k stack layer", layer, stats)
+
+
+def test_dense_path_long_lists_sampled():
+    """The library's dense path (full causal lists of up to 1024 blocks, Stage 2 off) at 128K: sampled query
+    blocks against the oracle's dense attention, every block counted as visited."""
+    w = WORKLOADS["qwen3_128k"]
+    qb, kb, vb, _ = w.make()
+    q, k, v = (to_dev(x) for x in (qb, kb, vb))
+    nqb = w.n_blocks
+    tri = torch.arange(nqb, device="cuda", dtype=torch.int32)
+    full = torch.where(tri[None, :] <= tri[:, None], tri[None, :].expand(nqb, nqb),
+                       torch.full((), -1, dtype=torch.int32, device="cuda")).expand(1, w.hq, nqb, nqb).contiguous()
+    fcount = (tri + 1).expand(1, w.hq, nqb).contiguous()
+    out = torch.empty_like(q)
+    lse = torch.empty(1, w.hq, w.n, dtype=torch.float32, device="cuda")
+    vis = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+    cosa.cosa_osk_attention(q, k, v, full, fcount, 1.0, out, lse, vis, opt=cosa.default_options(order_stride=nqb))
+    assert cosa.cosa_device_status() == 0
+    assert torch.equal(vis, fcount)
+    hv = HeadView(qb, kb, vb)
+    for h, blocks in ((0, [0, 1, 300, 1023]), (17, [511, 1022]), (31, [2, 777])):
+        qf, kf, vf = hv.get(h)
+        ref_o, ref_l = O.dense_attention(qf, kf, vf, query_blocks=blocks)
+        for a, i in enumerate(blocks):
+            got = out[0, h, i * 128:(i + 1) * 128].float().cpu().numpy().astype(np.float64)
+            err = np.abs(got - ref_o[0, a * 128:(a + 1) * 128])
+            assert err.max() < 2e-2 and err.mean() < 2e-3, (h, i, err.max(), err.mean())
+            assert np.abs(lse[0, h, i * 128:(i + 1) * 128].cpu().numpy() - ref_l[0, a * 128:(a + 1) * 128]).max() < 1e-3
