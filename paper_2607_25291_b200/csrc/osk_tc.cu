@@ -5,11 +5,12 @@
 //   warp 0       K loader: one TMA tile load per listed key block ("physical jumping": only the
 //                listed pages are ever touched), running ahead by the number of blocks that are
 //                already certain to be scored
-//   warp 1       MMA issuer: S = Q K_j^T into one of two TMEM buffers and O += P V_j, issued in
-//                whatever order their operands become ready.  Both products take their A operand
-//                (Q, resp. P) from tensor memory, so each MMA reads only 4 KiB of shared memory
-//                and the tensor pipe is not held back by operand fetch.
-//   warp 2       controller (see below); warp 3 idle
+//   warp 1       QK issuer: S = Q K_j^T into one of two TMEM buffers
+//   warp 3       PV issuer: O += P V_j.  Two issuing threads, because a single thread's
+//                instruction stream (descriptors, barrier tests, commits) is what limits how fast
+//                MMAs reach the tensor pipe.  Both products take their A operand (Q, resp. P)
+//                from tensor memory.
+//   warp 2       controller (see below)
 //   warps 4..7   softmax group A: list positions 0, 2, 4, ...   (one thread per query row)
 //   warps 8..11  softmax group B: list positions 1, 3, 5, ...
 //                A group copies its S tile from TMEM to registers (freeing the buffer at once),
@@ -190,69 +191,61 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (dataflow order)
+    // ------------------------------------------------------------------ QK issuer
     if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] and K_j [N x K], both K-major
-      const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
+      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] from TMEM, K_j [N x K] K-major
       // Q sits in TMEM once the first softmax group has copied it there
       bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
-      int kk_qk = 0;       // next QK^T to issue
-      int kk_seen = 0;     // decisions read so far
-      int n_known = 0;     // computed blocks among them
-      int n_pv = 0;        // PV products issued
-      int n_total = -1;    // number of scored blocks, once the end of the walk is known
-      long long t_last = clock64();
-      while (alive) {
-        bool progress = false;
-        const int nd = ctl->n_dec;
-        while (kk_seen < nd) {
-          const uint32_t d = ctl->dec[kk_seen % kDecRing];
-          if (d & kDecComputed) ++n_known;
-          if (d & kDecEnd) n_total = kk_seen + 1;
-          ++kk_seen;
-          progress = true;
+      const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
+      for (int kk = 0; kk < cnt && alive; ++kk) {
+        if (kk >= ctl->n_needed) {               // not yet certain that this block will be scored
+          const long long t0 = clock64();
+          bool ended = false;
+          while (kk >= ctl->n_needed) {
+            if (ctl->end_kk >= 0) { ended = kk >= ctl->n_needed; break; }
+            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+          }
+          if (ended || !alive) break;
         }
-        if (n_pv < n_known) {
-          const int vs = n_pv % kVStages;
-          if (mbar_test_wait(smem_u32(&ctl->p_full), n_pv & 1) &&
-              mbar_test_wait(smem_u32(&ctl->v_full[vs]), (n_pv / kVStages) & 1)) {
-            tc_fence_after();
-            const uint32_t vt = v_sm + vs * kTileBytes;
-#pragma unroll
-            for (int ks = 0; ks < kBlock / 16; ++ks)  // 16 keys per MMA: 8 TMEM columns of P, 2 KiB of V
-              mma_ts(tmem_o, tmem_p + ks * 8, smem_desc_sw128(vt + ks * 2048, kHalfBytes, 1024), idesc_pv,
-                     (n_pv > 0) || (ks > 0));
-            mma_commit(smem_u32(&ctl->p_empty[n_pv & 1]));
-            mma_commit(smem_u32(&ctl->v_empty[vs]));
-            ++n_pv;
-            progress = true;
+        const int st = kk % kKStages, sb = kk & 1;
+        alive = mbar_wait(smem_u32(&ctl->k_full[st]), (kk / kKStages) & 1, abort_flag) &&
+                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        tc_fence_after();
+        // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
+        mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+            tmem_s[sb], tmem_q, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk, false);
+        mma_commit(smem_u32(&ctl->s_full[sb]));
+        mma_commit(smem_u32(&ctl->k_empty[st]));
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ PV issuer
+    if (lane == 0) {
+      const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
+      const uint64_t vdesc0 = smem_desc_sw128(v_sm, kHalfBytes, 1024);
+      bool alive = true;
+      for (int n = 0; alive; ++n) {
+        // the next computed block's P, or the end of the walk
+        const uint32_t bar = smem_u32(&ctl->p_full), par = n & 1;
+        bool done = false;
+        if (!mbar_try_wait(bar, par)) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(bar, par)) {
+            if (ctl->end_kk >= 0 && n >= ctl->final_computed) { done = true; break; }
+            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
-        if (kk_qk < ctl->n_needed) {
-          const int st = kk_qk % kKStages, sb = kk_qk & 1;
-          if (mbar_test_wait(smem_u32(&ctl->k_full[st]), (kk_qk / kKStages) & 1) &&
-              mbar_test_wait(smem_u32(&ctl->s_empty[sb]), ((kk_qk >> 1) & 1) ^ 1)) {
-            tc_fence_after();
-            const uint32_t kt = k_sm + st * kTileBytes;
-#pragma unroll
-            for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-              const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;  // 16 elements of d per MMA
-              mma_ts(tmem_s[sb], tmem_q + ks * 8, smem_desc_sw128(kt + off, 16, 1024), idesc_qk, ks > 0);
-            }
-            mma_commit(smem_u32(&ctl->s_full[sb]));
-            mma_commit(smem_u32(&ctl->k_empty[st]));
-            ++kk_qk;
-            progress = true;
-          }
-        }
-        if (n_total >= 0 && n_pv == n_known && kk_qk >= n_total) break;
-        if (progress) {
-          t_last = clock64();
-        } else if (*abort_flag || clock64() - t_last > kWaitBudget) {
-          if (!*abort_flag) report_timeout(ctl, status);
-          alive = false;
-        }
+        if (done || !alive) break;
+        const int vs = n % kVStages;
+        alive = mbar_wait(smem_u32(&ctl->v_full[vs]), (n / kVStages) & 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        tc_fence_after();
+        // 16 keys per MMA: 8 TMEM columns of P, 2 KiB (two 8-key groups) of the V tile
+        mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p, vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
+        mma_commit(smem_u32(&ctl->p_empty[n & 1]));
+        mma_commit(smem_u32(&ctl->v_empty[vs]));
       }
     }
   } else if (warp == 2) {

@@ -149,6 +149,29 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Eight MMAs in one go: D[tmem] (+)= A[tmem] * B[smem] over K = 128 (8 steps of 16).  The A operand
+// advances by 8 TMEM columns per step; the B descriptor's start-address field advances by the eight
+// 16-byte units given in b_step (descriptor low word += b_step[i] relative to step 0).  Built as
+// one asm block so that the issuing thread spends as few instructions as possible per MMA: a single
+// thread's instruction stream is what feeds the tensor pipe.
+template <int S1, int S2, int S3, int S4, int S5, int S6, int S7>
+__device__ __forceinline__ void mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc0, uint32_t idesc, bool accumulate_first) {
+  uint32_t acc = accumulate_first ? 1u : 0u;
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b32 a;\n\t.reg .b64 b;\n\t"
+      "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.s64 b, %2, %5;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 16;\n\tadd.s64 b, %2, %6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 24;\n\tadd.s64 b, %2, %7;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 32;\n\tadd.s64 b, %2, %8;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 40;\n\tadd.s64 b, %2, %9;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 48;\n\tadd.s64 b, %2, %10;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "add.u32 a, %1, 56;\n\tadd.s64 b, %2, %11;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p1;\n\t"
+      "}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc0), "r"(idesc), "r"(acc), "n"(S1), "n"(S2), "n"(S3), "n"(S4), "n"(S5), "n"(S6), "n"(S7)
+      : "memory");
+}
 // The mbarrier receives one arrival when every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
