@@ -48,10 +48,13 @@ constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks
 constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
 struct __align__(8) Control {
-  unsigned long long q_full, k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
-  unsigned long long s_full[2], s_empty[2], p_full;
-  unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1]: a waiter may run two products ahead
-                                  // of the tensor pipe, which one barrier's single parity bit cannot tell apart
+  unsigned long long q_full, k_full[kKStages], v_full[kVStages];
+  unsigned long long k_empty[kKStages];  // QK^T of that stage finished: the stage is free AND its S tile is ready
+  unsigned long long s_empty[2], p_full;
+  unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1] (P free, O updated, V stage n & 1 free); two
+                                  // barriers because a waiter may run two products ahead of the tensor pipe, which one
+                                  // barrier's single parity bit cannot tell apart
+  unsigned long long out_bar[2];  // a softmax group has staged its half of the output tile
   unsigned long long m_ready[2];  // a group has published the row statistics of its position
   unsigned long long dec_bar[2];  // the controller has published the decision of that position
   unsigned long long fin_bar;     // both groups have published their final partial sums
@@ -61,6 +64,7 @@ struct __align__(8) Control {
   volatile int end_kk;            // last scored position, -1 until known
   volatile int final_computed;
   volatile int abort_flag;
+  int poisoned;
   volatile uint32_t dec[kDecRing];
   float mloc[2][kBlock];          // [position parity][row]: block row maxima (scaled, base 2)
   float mrow[2][kBlock];          // [position parity][row]: running row maxima including that block
@@ -91,7 +95,8 @@ __device__ __forceinline__ bool spin_until_ge(volatile int* v, int want, volatil
 
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
-              const __grid_constant__ CUtensorMap v_map, OskParams p, int32_t* status) {
+              const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
+              int32_t* status) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -120,21 +125,19 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  // once some CTA has reported a timeout the rest of the grid returns at once
-  __shared__ int s_poisoned;
-  if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int32_t*>(status);
-  __syncthreads();
-  if (s_poisoned != 0) return;
-
+  static_assert(kVStages == 2, "PV product n frees V stage n & 1 together with p_empty[n & 1]");
   if (threadIdx.x == 0) {
+    // once some CTA has reported a timeout the rest of the grid returns at once
+    ctl->poisoned = *reinterpret_cast<volatile int32_t*>(status);
     mbar_init(smem_u32(&ctl->q_full), kBlock);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
-    for (int s = 0; s < kVStages; ++s) { mbar_init(smem_u32(&ctl->v_full[s]), 1); mbar_init(smem_u32(&ctl->v_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
+      mbar_init(smem_u32(&ctl->v_full[s]), 1);
+      mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
       mbar_init(smem_u32(&ctl->m_ready[s]), kBlock); mbar_init(smem_u32(&ctl->dec_bar[s]), 1);
+      mbar_init(smem_u32(&ctl->p_empty[s]), 1); mbar_init(smem_u32(&ctl->out_bar[s]), kBlock);
     }
-    mbar_init(smem_u32(&ctl->p_full), kBlock); mbar_init(smem_u32(&ctl->p_empty[0]), 1); mbar_init(smem_u32(&ctl->p_empty[1]), 1);
+    mbar_init(smem_u32(&ctl->p_full), kBlock);
     mbar_init(smem_u32(&ctl->fin_bar), 2 * kBlock);
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
@@ -143,15 +146,29 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
-    prefetch_tensormap(&k_map); prefetch_tensormap(&v_map);
+    if (ctl->poisoned == 0) {
+      // the first K tiles are requested before the rest of the CTA has even finished setting up
+      const int n_first = min(min(cnt, cap), kKStages);
+      for (int kk = 0; kk < n_first; ++kk) {
+        const int j = min(max(list[kk], 0), p.nqb - 1);
+        const uint32_t dst = k_sm + kk * kTileBytes, bar = smem_u32(&ctl->k_full[kk]);
+        mbar_expect_tx(bar, kTileBytes);
+        tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
+        tma_load_2d(dst + kHalfBytes, &k_map, 64, kv_row0 + j * kBlock, bar);
+      }
+    }
   }
-  if (warp == 0) {
+  if (warp == 1) {
     tmem_alloc(smem_u32(&ctl->tmem_base), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (ctl->poisoned != 0) {
+    if (warp == 1) tmem_dealloc(ctl->tmem_base, kTmemCols);
+    return;
+  }
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
@@ -169,7 +186,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else if (warp == 0) {
     // ------------------------------------------------------------------ K loader
     if (lane == 0) {
-      for (int kk = 0; kk < cnt; ++kk) {
+      for (int kk = min(min(cnt, cap), kKStages); kk < cnt; ++kk) {   // the first tiles were requested in the prologue
         const long long t0 = clock64();
         bool ok = true;
         while (kk >= ctl->n_needed) {          // not yet certain that this block will be scored
@@ -216,7 +233,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
         mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
             tmem_s[sb], tmem_q, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk, false);
-        mma_commit(smem_u32(&ctl->s_full[sb]));
         mma_commit(smem_u32(&ctl->k_empty[st]));
       }
     }
@@ -245,7 +261,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         // 16 keys per MMA: 8 TMEM columns of P, 2 KiB (two 8-key groups) of the V tile
         mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p, vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
         mma_commit(smem_u32(&ctl->p_empty[n & 1]));
-        mma_commit(smem_u32(&ctl->v_empty[vs]));
       }
     }
   } else if (warp == 2) {
@@ -280,7 +295,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         if (last) ctl->end_kk = kk;
         if (compute) {                            // fetch V_j now that the block is known to be computed
           const int vs = n_before % kVStages;
-          if (!mbar_wait(smem_u32(&ctl->v_empty[vs]), ((n_before / kVStages) & 1) ^ 1, abort_flag)) {
+          if (!mbar_wait(smem_u32(&ctl->p_empty[vs]), ((n_before >> 1) & 1) ^ 1, abort_flag)) {   // PV n-2 read this stage
             if (!*abort_flag) report_timeout(ctl, status);
           } else {
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
@@ -342,7 +357,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const int j = min(max(list[kk], 0), p.nqb - 1);
       // wait for S(kk), or learn that the walk ended before this position
       {
-        const uint32_t bar = smem_u32(&ctl->s_full[grp]), par = (kk >> 1) & 1;
+        const uint32_t bar = smem_u32(&ctl->k_empty[kk % kKStages]), par = (kk / kKStages) & 1;   // QK^T(kk) finished
         bool ended = false;
         if (!mbar_try_wait(bar, par)) {
           const long long t0 = clock64();
@@ -459,7 +474,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (alive) {
         tc_fence_after();
         const float inv = lt > 0.f ? 1.f / lt : 0.f;
-        __nv_bfloat16* dst = p.out + ((size_t)q_row0 + r) * kHeadDim + grp * 64;   // each group writes half the row
+        // stage this group's 64 columns of the tile in (now idle) K stage memory, swizzled like a TMA box,
+        // and let one thread store the whole half tile with a single bulk tensor copy
+        unsigned char* stage = smem + grp * kHalfBytes;
 #pragma unroll
         for (int c = 0; c < 2; ++c) {
           uint32_t o[32];
@@ -472,7 +489,18 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
             pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
             pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
             pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + c * 32 + e) = pk;
+            const int chunk = c * 4 + (e >> 3);
+            *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) = pk;
+          }
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(smem_u32(&ctl->out_bar[grp]));
+        if (r == 0) {
+          if (mbar_wait(smem_u32(&ctl->out_bar[grp]), 0, abort_flag)) {
+            tma_store_2d(&o_map, grp * 64, q_row0, k_sm + grp * kHalfBytes);
+            tma_store_commit_and_wait_read();
+          } else if (!*abort_flag) {
+            report_timeout(ctl, status);
           }
         }
         if (p.lse && grp == 0) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
@@ -482,7 +510,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -518,9 +546,9 @@ bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows) {
 }  // namespace
 
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
-  CUtensorMap qm, km, vm;
+  CUtensorMap qm, km, vm, om;
   if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, (uint64_t)p.batch * p.hkv * p.n) ||
-      !make_tile_map(&vm, p.v, (uint64_t)p.batch * p.hkv * p.n))
+      !make_tile_map(&vm, p.v, (uint64_t)p.batch * p.hkv * p.n) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
     return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(osk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
@@ -531,7 +559,7 @@ cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
   }
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;
-  osk_tc_kernel<<<p.batch * p.hq * p.nqb, kThreads, kSmemBytes, st>>>(qm, km, vm, p, status);
+  osk_tc_kernel<<<p.batch * p.hq * p.nqb, kThreads, kSmemBytes, st>>>(qm, km, vm, om, p, status);
   return cudaGetLastError();
 }
 
