@@ -29,13 +29,17 @@ using namespace ptx;
 constexpr int kStages = 4;
 constexpr int kTileBytes = 128 * kHeadDim * 2;
 constexpr int kHalfBytes = kTileBytes / 2;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;        // producer warp, MMA warp, 2 x 4 epilogue warps
 constexpr int kTmemCols = 256;
 
 struct __align__(8) ScreenCtl {
-  unsigned long long a_full, k_full[kStages], k_empty[kStages], s_full[2], s_empty[2];
+  unsigned long long a_full, k_full[kStages];
+  unsigned long long k_empty[kStages];  // the tile's MMAs finished: stage free and logits ready
+  unsigned long long s_empty[2], x_bar;
   uint32_t tmem_base;
   volatile int abort_flag;
+  float xt[2][3][128];                  // pass-1 exchange between the two column halves: top-3 block maxima
+  int xj[2][2][128];                    // ... and the blocks holding the two largest
 };
 constexpr size_t kScreenSmem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(ScreenCtl);
 
@@ -79,7 +83,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     if (blockIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
     mbar_init(smem_u32(&ctl->a_full), 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&ctl->s_full[s]), 1); mbar_init(smem_u32(&ctl->s_empty[s]), 128); }
+    for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), 256);
+    mbar_init(smem_u32(&ctl->x_bar), 256);
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -127,18 +132,16 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         tc_fence_after();
         const uint32_t kt = k_sm + st * kTileBytes;
-#pragma unroll
-        for (int ks = 0; ks < kHeadDim / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          mma_ss(tmem + sb * 128, smem_desc_sw128(a_sm + off, 16, 1024), smem_desc_sw128(kt + off, 16, 1024), idesc, ks > 0);
-        }
-        mma_commit(smem_u32(&ctl->s_full[sb]));
+        mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+            tmem + sb * 128, smem_desc_sw128(a_sm, 16, 1024), smem_desc_sw128(kt, 16, 1024), idesc);
         mma_commit(smem_u32(&ctl->k_empty[st]));
       }
     }
   } else {
-    // ---------------------------------------------------------------- one thread per sampled query row
+    // ---------------------------------------------------------------- two threads per sampled query row
+    // (one per 64-column half of every tile: two epilogue warps per SM sub-partition overlap their latencies)
     const int sub = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int row = sub * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
     const int grp = row / R, r = row % R;
@@ -155,16 +158,30 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     float* srow = p.scores + ((size_t)(b * p.hq + h) * p.nqb + (row_ok ? i : 0)) * p.nqb;
     bool alive = true;
     for (int t = 0; t < 2 * n_tiles && alive; ++t) {
-      const int sb = t & 1, jt = t % n_tiles;
+      const int sb = t & 1, jt = t % n_tiles, st = t % kStages;
       const bool pass2 = t >= n_tiles;
       if (t == n_tiles) {
-        // end of pass 1: the row's best block, and whether the runner-up is too close to call
+        // end of pass 1: merge the two halves' top-3 block maxima of every row
+        ctl->xt[half][0][row] = top1; ctl->xt[half][1][row] = top2; ctl->xt[half][2][row] = top3;
+        ctl->xj[half][0][row] = jstar; ctl->xj[half][1][row] = jstar2;
+        mbar_arrive(smem_u32(&ctl->x_bar));
+        alive = mbar_wait(smem_u32(&ctl->x_bar), 0, abort_flag);
+        if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+          const float m = ctl->xt[half ^ 1][q][row];
+          const int jb = q < 2 ? ctl->xj[half ^ 1][q][row] : 0;
+          if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
+          else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
+          else if (m > top3) top3 = m;
+        }
+        // the row's best block, and whether the runner-up is too close to call
         const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
         const bool amb3 = row_ok && (top1 - top3) * p.scale <= p.tau_row;
         const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);
         const int shift = (lane / R) * R;
         const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << shift);
-        if (row_ok) {
+        if (row_ok && half == 0) {
           int2 js = make_int2(jstar, jstar2);
           reinterpret_cast<int2*>(p.jstar)[(size_t)(b * p.hq + h) * ns + r_glob] = js;
           if (r == 0) {
@@ -173,30 +190,35 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           }
         }
       }
-      alive = mbar_wait(smem_u32(&ctl->s_full[sb]), (t >> 1) & 1, abort_flag);
+      alive = mbar_wait(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag);   // this tile's MMAs finished
       if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
       tc_fence_after();
-      const int col0 = jt * 128;
+      const int col0 = jt * 128 + half * 64;
+      uint32_t v[2][32];
+      tmem_ld32(tmem + sb * 128 + lane_addr + half * 64, v[0]);
+      tmem_ld32(tmem + sb * 128 + lane_addr + half * 64 + 32, v[1]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->s_empty[sb]));
 #pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        uint32_t v[32];
-        tmem_ld32(tmem + sb * 128 + lane_addr + c4 * 32, v);
-        tmem_wait_ld();
-        if (c4 == 3) { tc_fence_before(); mbar_arrive(smem_u32(&ctl->s_empty[sb])); }
-        const int cbase = col0 + c4 * 32;
+      for (int c2 = 0; c2 < 2; ++c2) {
+        const int cbase = col0 + c2 * 32;
         float mb[BPC];
 #pragma unroll
         for (int bb = 0; bb < BPC; ++bb) {
-          float m = -INFINITY;
+          float m0 = -INFINITY, m1 = -INFINITY;
           if (cbase + bb * R + R - 1 <= c_limit) {        // whole block visible: no masking
 #pragma unroll
-            for (int e = 0; e < R; ++e) m = fmaxf(m, __uint_as_float(v[bb * R + e]));
+            for (int e = 0; e < R; e += 2) {
+              m0 = fmaxf(m0, __uint_as_float(v[c2][bb * R + e]));
+              m1 = fmaxf(m1, __uint_as_float(v[c2][bb * R + e + 1]));
+            }
           } else {
 #pragma unroll
             for (int e = 0; e < R; ++e)
-              if (cbase + bb * R + e <= c_limit) m = fmaxf(m, __uint_as_float(v[bb * R + e]));
+              if (cbase + bb * R + e <= c_limit) m0 = fmaxf(m0, __uint_as_float(v[c2][bb * R + e]));
           }
-          mb[bb] = m;
+          mb[bb] = fmaxf(m0, m1);
         }
         if (!pass2) {
 #pragma unroll
@@ -210,7 +232,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         } else {
 #pragma unroll
           for (int bb = 0; bb < BPC; ++bb) {
-            float e = exp2f((mb[bb] - top1) * scale2);   // exp(M[r,j] - M*[r]); 0 for invisible blocks
+            float e = ex2_approx((mb[bb] - top1) * scale2);   // exp(M[r,j] - M*[r]); 0 for invisible blocks
             unsigned f = (mb[bb] == top1) ? 1u : 0u;
             if (!row_ok) { e = 0.f; f = 0u; }
 #pragma unroll

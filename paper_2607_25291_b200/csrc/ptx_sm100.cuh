@@ -182,6 +182,25 @@ __device__ __forceinline__ void mma_ts_x8(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "l"(bdesc0), "r"(idesc), "r"(acc), "n"(S1), "n"(S2), "n"(S3), "n"(S4), "n"(S5), "n"(S6), "n"(S7)
       : "memory");
 }
+// Eight MMAs, both operands K-major in shared memory: D[tmem] = A[smem] * B[smem] over K = 128.
+// Both descriptors advance by the same eight offsets (16-byte units).
+template <int S1, int S2, int S3, int S4, int S5, int S6, int S7>
+__device__ __forceinline__ void mma_ss_x8(uint32_t d_tmem, uint64_t adesc0, uint64_t bdesc0, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a, b;\n\t"
+      "setp.ne.b32 p0, 0, 0;\n\tsetp.eq.b32 p1, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p0;\n\t"
+      "add.s64 a, %1, %4;\n\tadd.s64 b, %2, %4;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %5;\n\tadd.s64 b, %2, %5;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %6;\n\tadd.s64 b, %2, %6;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %7;\n\tadd.s64 b, %2, %7;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %8;\n\tadd.s64 b, %2, %8;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %9;\n\tadd.s64 b, %2, %9;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "add.s64 a, %1, %10;\n\tadd.s64 b, %2, %10;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p1;\n\t"
+      "}" ::"r"(d_tmem),
+      "l"(adesc0), "l"(bdesc0), "r"(idesc), "n"(S1), "n"(S2), "n"(S3), "n"(S4), "n"(S5), "n"(S6), "n"(S7)
+      : "memory");
+}
 // The mbarrier receives one arrival when every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
