@@ -160,17 +160,69 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   }
 
   // ---- 2. bitonic sort, descending in (flag, float32 score, -id)
-  for (int k = 2; k <= P2; k <<= 1) {
-    for (int js = k >> 1; js > 0; js >>= 1) {
-      for (int t = tid; t < P2; t += kThreads) {
-        const int u = t ^ js;
-        if (u > t) {
-          const unsigned long long a = keys[t], c = keys[u];
-          const bool up = (t & k) == 0;
-          if (up ? (c > a) : (a > c)) { keys[t] = c; keys[u] = a; }
+  if (P2 <= 4 * kThreads) {
+    // four consecutive keys per thread: exchanges at distance < 4 stay in registers, distances 4..64 go
+    // through warp shuffles, and only distances >= 128 need shared memory and a CTA barrier
+    unsigned long long kr[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) kr[q] = (tid * 4 + q < P2) ? keys[tid * 4 + q] : 0ULL;
+    for (int k = 2; k <= P2; k <<= 1) {
+      for (int js = k >> 1; js > 0; js >>= 1) {
+        if (js >= 128) {
+          __syncthreads();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) if (tid * 4 + q < P2) keys[tid * 4 + q] = kr[q];
+          __syncthreads();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int e = tid * 4 + q;
+            if (e < P2) {
+              const unsigned long long other = keys[e ^ js];
+              const bool want_max = ((e & k) == 0) == ((e & js) == 0);   // the lower index of a pair keeps the larger key in "up" segments
+              kr[q] = want_max ? (other > kr[q] ? other : kr[q]) : (other < kr[q] ? other : kr[q]);
+            }
+          }
+        } else if (js >= 4) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int e = tid * 4 + q;
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, kr[q], js >> 2);
+            const bool want_max = ((e & k) == 0) == ((e & js) == 0);
+            kr[q] = want_max ? (other > kr[q] ? other : kr[q]) : (other < kr[q] ? other : kr[q]);
+          }
+        } else {
+          // both keys of a pair live in this thread; for k >= 4 all four share one direction
+          const bool up = ((tid * 4) & k) == 0;
+          auto cx = [](unsigned long long& first, unsigned long long& second, bool descending) {
+            const bool keep = descending ? (first >= second) : (first <= second);
+            const unsigned long long f = keep ? first : second, g = keep ? second : first;
+            first = f; second = g;
+          };
+          if (js == 2) {
+            cx(kr[0], kr[2], up); cx(kr[1], kr[3], up);
+          } else {
+            cx(kr[0], kr[1], k == 2 ? true : up); cx(kr[2], kr[3], k == 2 ? false : up);
+          }
         }
       }
-      __syncthreads();
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 4; ++q) if (tid * 4 + q < P2) keys[tid * 4 + q] = kr[q];
+    __syncthreads();
+  } else {
+    for (int k = 2; k <= P2; k <<= 1) {
+      for (int js = k >> 1; js > 0; js >>= 1) {
+        for (int t = tid; t < P2; t += kThreads) {
+          const int u = t ^ js;
+          if (u > t) {
+            const unsigned long long a = keys[t], c = keys[u];
+            const bool up = (t & k) == 0;
+            if (up ? (c > a) : (a > c)) { keys[t] = c; keys[u] = a; }
+          }
+        }
+        __syncthreads();
+      }
     }
   }
   const int K = budget_count_fx(p.budget_fx, J);
