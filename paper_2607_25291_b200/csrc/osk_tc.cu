@@ -8,8 +8,8 @@
 //   warp 1       QK issuer: S = Q K_j^T into one of two TMEM buffers
 //   warp 3       PV issuer: O += P V_j.  Two issuing threads, because a single thread's
 //                instruction stream (descriptors, barrier tests, commits) is what limits how fast
-//                MMAs reach the tensor pipe.  Both products take their A operand (Q, resp. P)
-//                from tensor memory.
+//                MMAs reach the tensor pipe.  Both products take their A operand (Q, resp. P) from
+//                tensor memory: with both operands in shared memory the QK^T product ran slower.
 //   warp 2       controller (see below)
 //   warps 4..7   softmax group A: list positions 0, 2, 4, ...   (one thread per query row)
 //   warps 8..11  softmax group B: list positions 1, 3, 5, ...
@@ -23,7 +23,7 @@
 //                the cap on computed blocks, the V tile load of computed blocks, and the
 //                decisions the other warps follow
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
-// expect; Q goes from global memory through registers straight into TMEM.
+// expect; the Q tile is fetched by TMA as well and copied from shared memory into TMEM by the first group.
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P [384,448) Q [448,512).
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
 // down without writing results.
@@ -48,13 +48,13 @@ constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks
 constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
 struct __align__(8) Control {
-  unsigned long long q_full, k_full[kKStages], v_full[kVStages];
+  unsigned long long q_stage, q_full, k_full[kKStages], v_full[kVStages];   // Q tile landed / Q copied into TMEM
   unsigned long long k_empty[kKStages];  // QK^T of that stage finished: the stage is free AND its S tile is ready
   unsigned long long s_empty[2], p_full;
   unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1] (P free, O updated, V stage n & 1 free); two
                                   // barriers because a waiter may run two products ahead of the tensor pipe, which one
                                   // barrier's single parity bit cannot tell apart
-  unsigned long long out_bar[2];  // a softmax group has staged its half of the output tile
+  unsigned long long out_bar;     // the output tile has been staged in shared memory
   unsigned long long m_ready[2];  // a group has published the row statistics of its position
   unsigned long long dec_bar[2];  // the controller has published the decision of that position
   unsigned long long fin_bar;     // both groups have published their final partial sums
@@ -66,12 +66,13 @@ struct __align__(8) Control {
   volatile int abort_flag;
   int poisoned;
   volatile uint32_t dec[kDecRing];
-  float mloc[2][kBlock];          // [position parity][row]: block row maxima (scaled, base 2)
+  unsigned gapw[2][4];            // [position parity][warp]: bits of max over the warp's rows of (m_loc - m), <= 0
   float mrow[2][kBlock];          // [position parity][row]: running row maxima including that block
-  float fin_m[2][kBlock], fin_l[2][kBlock];
+  float fin_m[kBlock], fin_l[kBlock];   // the second group's partial row sums and their reference maxima
 };
 
-constexpr size_t kSmemBytes = 1024 /*alignment slack*/ + (size_t)kTileBytes * (kKStages + kVStages) + sizeof(Control);
+constexpr size_t kSmemBytes = (size_t)kTileBytes * (kKStages + kVStages + 1) + sizeof(Control);
+static_assert(kSmemBytes <= 232448, "shared memory budget of one CTA");
 
 __device__ __forceinline__ void report_timeout(Control* c, int32_t* status) {
   c->abort_flag = 1;
@@ -83,27 +84,21 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
-// bounded spin on a volatile counter: true once *v >= want
-__device__ __forceinline__ bool spin_until_ge(volatile int* v, int want, volatile int* abort_flag) {
-  if (*v >= want) return true;
-  const long long t0 = clock64();
-  while (*v < want) {
-    if (*abort_flag || clock64() - t0 > kWaitBudget) return false;
-  }
-  return true;
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
               int32_t* status) {
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
-  unsigned char* smem = smem_raw + (base - raw);
+  extern __shared__ __align__(1024) unsigned char smem_raw[];   // swizzled tiles need 1024-byte alignment
+  unsigned char* smem = smem_raw;
+  const uint32_t base = smem_u32(smem_raw);
+  if (base & 1023u) {   // never expected; refuse to run rather than compute on misplaced tiles
+    if (threadIdx.x == 0) atomicMin(status, (int32_t)COSA_ERR_CUDA);
+    return;
+  }
   const uint32_t k_sm = base;
   const uint32_t v_sm = k_sm + kKStages * kTileBytes;
-  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (kKStages + kVStages));
+  const uint32_t q_sm = v_sm + kVStages * kTileBytes;
+  Control* ctl = reinterpret_cast<Control*>(smem + (size_t)kTileBytes * (kKStages + kVStages + 1));
 
   // work item: KV head major, then query blocks from the longest list down, the group's query
   // heads innermost, so that CTAs resident together read the same K/V pages
@@ -125,20 +120,30 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  static_assert(kVStages == 2, "PV product n frees V stage n & 1 together with p_empty[n & 1]");
+  // global loads whose latency should overlap the set-up: the first list entries and the status word
+  int first_ids[kKStages] = {0, 0, 0, 0};
+  int poisoned_early = 0;
+  if (threadIdx.x == 0) {
+    poisoned_early = *reinterpret_cast<volatile int32_t*>(status);
+#pragma unroll
+    for (int kk = 0; kk < kKStages; ++kk) first_ids[kk] = kk < p.order_stride ? list[kk] : 0;
+  }
+
+  static_assert(kVStages == 2 && kKStages == 4, "PV product n frees V stage n & 1 together with p_empty[n & 1]");
   if (threadIdx.x == 0) {
     // once some CTA has reported a timeout the rest of the grid returns at once
-    ctl->poisoned = *reinterpret_cast<volatile int32_t*>(status);
-    mbar_init(smem_u32(&ctl->q_full), kBlock);
+    ctl->poisoned = poisoned_early;
+    mbar_init(smem_u32(&ctl->q_stage), 1); mbar_init(smem_u32(&ctl->q_full), kBlock);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&ctl->v_full[s]), 1);
       mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
       mbar_init(smem_u32(&ctl->m_ready[s]), kBlock); mbar_init(smem_u32(&ctl->dec_bar[s]), 1);
-      mbar_init(smem_u32(&ctl->p_empty[s]), 1); mbar_init(smem_u32(&ctl->out_bar[s]), kBlock);
+      mbar_init(smem_u32(&ctl->p_empty[s]), 1);
     }
+    mbar_init(smem_u32(&ctl->out_bar), kBlock);
     mbar_init(smem_u32(&ctl->p_full), kBlock);
-    mbar_init(smem_u32(&ctl->fin_bar), 2 * kBlock);
+    mbar_init(smem_u32(&ctl->fin_bar), kBlock);
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
     ctl->end_kk = -1;
@@ -147,10 +152,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     mbar_fence_init();
     fence_proxy_async_smem();
     if (ctl->poisoned == 0) {
-      // the first K tiles are requested before the rest of the CTA has even finished setting up
+      // Q and the first K tiles are requested before the rest of the CTA has even finished setting up
+      mbar_expect_tx(smem_u32(&ctl->q_stage), kTileBytes);
+      tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_stage));
+      tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, smem_u32(&ctl->q_stage));
       const int n_first = min(min(cnt, cap), kKStages);
       for (int kk = 0; kk < n_first; ++kk) {
-        const int j = min(max(list[kk], 0), p.nqb - 1);
+        const int j = min(max(first_ids[kk], 0), p.nqb - 1);
         const uint32_t dst = k_sm + kk * kTileBytes, bar = smem_u32(&ctl->k_full[kk]);
         mbar_expect_tx(bar, kTileBytes);
         tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
@@ -211,7 +219,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     // ------------------------------------------------------------------ QK issuer
     if (lane == 0) {
       const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] from TMEM, K_j [N x K] K-major
-      // Q sits in TMEM once the first softmax group has copied it there
       bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
       const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
@@ -274,12 +281,10 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const int j = min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
       alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
-      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block
-      float gm = -INFINITY;
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) gm = fmaxf(gm, ctl->mloc[par][lane + 32 * q4] - ctl->mrow[par][lane + 32 * q4]);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, o));
+      // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
+      // The statistic is <= 0, so among bit patterns the smallest unsigned word is the largest value.
+      const volatile unsigned* gw = ctl->gapw[par];
+      const float gm = __uint_as_float(min(min(gw[0], gw[1]), min(gw[2], gw[3])));
       const bool compute = !(p.use_threshold && gm < theta2);
       ++scored;
       const int n_before = computed;
@@ -340,11 +345,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     bool alive = true;
     uint32_t s[kBlock];                       // this row's raw logits, then probabilities
     if (grp == 0) {
-      // Q row -> TMEM as the A operand of QK^T: lane = row, two consecutive d per 32-bit column
-      const uint4* src = reinterpret_cast<const uint4*>(p.q + ((size_t)q_row0 + r) * kHeadDim);
+      // Q row: shared memory (TMA box layout, 16-byte chunks swizzled by row) -> TMEM as the A operand of
+      // QK^T: lane = row, two consecutive d per 32-bit column
+      alive = mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag);
+      if (!alive && !*abort_flag) report_timeout(ctl, status);
+      const unsigned char* qs = smem + (size_t)kTileBytes * (kKStages + kVStages);
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const uint4 wv = src[c];
+        const uint4 wv = *reinterpret_cast<const uint4*>(qs + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
         s[4 * c] = wv.x; s[4 * c + 1] = wv.y; s[4 * c + 2] = wv.z; s[4 * c + 3] = wv.w;
       }
       tmem_st32(tmem_q + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
@@ -396,11 +404,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         m_in = ctl->mrow[grp ^ 1][r];
       }
       const float m_new = fmaxf(m_in, m_loc);
-      // the controller must have read this slot's previous contents (position kk-2)
-      if (kk >= 2 && !spin_until_ge(&ctl->n_dec, kk - 1, abort_flag)) {
-        alive = false; if (!*abort_flag) report_timeout(ctl, status); break;
-      }
-      ctl->mloc[grp][r] = m_loc;
+      // (the slots written here were last read for position kk-2, whose decision this group has already received)
+      const unsigned gbits = __reduce_min_sync(0xffffffffu, __float_as_uint(m_loc - m_new));
+      if (lane == 0) ctl->gapw[grp][sub] = gbits;
       ctl->mrow[grp][r] = m_new;
       mbar_arrive(smem_u32(&ctl->m_ready[grp]));
       // ---- the controller's decision
@@ -454,56 +460,60 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       m_ref = m_new;
       if (last) break;
     }
-    // ---- the two groups combine their partial sums; every softmax thread reaches this point
-    ctl->fin_m[grp][r] = m_ref;
-    ctl->fin_l[grp][r] = l;
-    mbar_arrive(smem_u32(&ctl->fin_bar));
-    if (alive) {
-      alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag);
-      if (!alive && !*abort_flag) report_timeout(ctl, status);
-    }
-    if (alive && !*abort_flag) {
-      const float ma = ctl->fin_m[0][r], mb = ctl->fin_m[1][r];
-      const float mf = fmaxf(ma, mb);            // the running maximum is monotone: this is its final value
-      const float lt = ctl->fin_l[0][r] * ex2_approx(ma - mf) + ctl->fin_l[1][r] * ex2_approx(mb - mf);
-      const int n_comp = ctl->final_computed;
-      if (n_comp > 0) {
-        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag);
+    // ---- the second group hands its partial sums to the first, which finishes the tile
+    if (grp == 1) {
+      ctl->fin_m[r] = m_ref;
+      ctl->fin_l[r] = l;
+      mbar_arrive(smem_u32(&ctl->fin_bar));
+    } else {
+      if (alive) {
+        alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag);
         if (!alive && !*abort_flag) report_timeout(ctl, status);
       }
-      if (alive) {
-        tc_fence_after();
-        const float inv = lt > 0.f ? 1.f / lt : 0.f;
-        // stage this group's 64 columns of the tile in (now idle) K stage memory, swizzled like a TMA box,
-        // and let one thread store the whole half tile with a single bulk tensor copy
-        unsigned char* stage = smem + grp * kHalfBytes;
+      if (alive && !*abort_flag) {
+        const float mb = ctl->fin_m[r];
+        const float mf = fmaxf(m_ref, mb);         // the running maximum is monotone: this is its final value
+        const float lt = l * ex2_approx(m_ref - mf) + ctl->fin_l[r] * ex2_approx(mb - mf);
+        const int n_comp = ctl->final_computed;
+        if (n_comp > 0) {
+          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag);
+          if (!alive && !*abort_flag) report_timeout(ctl, status);
+        }
+        if (alive) {
+          tc_fence_after();
+          const float inv = lt > 0.f ? 1.f / lt : 0.f;
+          // stage the tile in (now idle) K stage memory, swizzled like two TMA boxes of 64 columns, and let
+          // one thread store it with two bulk tensor copies
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_addr + grp * 64 + c * 32, o);
-          tmem_wait_ld();
+          for (int c = 0; c < 4; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + lane_addr + c * 32, o);
+            tmem_wait_ld();
+            unsigned char* stage = smem + (c >> 1) * kHalfBytes;
 #pragma unroll
-          for (int e = 0; e < 32; e += 8) {
-            uint4 pk;
-            pk.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
-            pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
-            pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
-            pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
-            const int chunk = c * 4 + (e >> 3);
-            *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) = pk;
+            for (int e = 0; e < 32; e += 8) {
+              uint4 pk;
+              pk.x = pack_bf16(__uint_as_float(o[e + 0]) * inv, __uint_as_float(o[e + 1]) * inv);
+              pk.y = pack_bf16(__uint_as_float(o[e + 2]) * inv, __uint_as_float(o[e + 3]) * inv);
+              pk.z = pack_bf16(__uint_as_float(o[e + 4]) * inv, __uint_as_float(o[e + 5]) * inv);
+              pk.w = pack_bf16(__uint_as_float(o[e + 6]) * inv, __uint_as_float(o[e + 7]) * inv);
+              const int chunk = (c & 1) * 4 + (e >> 3);
+              *reinterpret_cast<uint4*>(stage + r * 128 + ((chunk ^ (r & 7)) << 4)) = pk;
+            }
+          }
+          fence_proxy_async_smem();
+          mbar_arrive(smem_u32(&ctl->out_bar));
+          if (p.lse) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
+          if (r == 0) {
+            if (mbar_wait(smem_u32(&ctl->out_bar), 0, abort_flag)) {
+              tma_store_2d(&o_map, 0, q_row0, k_sm);
+              tma_store_2d(&o_map, 64, q_row0, k_sm + kHalfBytes);
+              tma_store_commit_and_wait_read();
+            } else if (!*abort_flag) {
+              report_timeout(ctl, status);
+            }
           }
         }
-        fence_proxy_async_smem();
-        mbar_arrive(smem_u32(&ctl->out_bar[grp]));
-        if (r == 0) {
-          if (mbar_wait(smem_u32(&ctl->out_bar[grp]), 0, abort_flag)) {
-            tma_store_2d(&o_map, grp * 64, q_row0, k_sm + grp * kHalfBytes);
-            tma_store_commit_and_wait_read();
-          } else if (!*abort_flag) {
-            report_timeout(ctl, status);
-          }
-        }
-        if (p.lse && grp == 0) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
       }
     }
   }
