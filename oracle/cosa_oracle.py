@@ -186,14 +186,41 @@ def flag_grouped_order(scores, flags):
     return ids
 
 
+def topp_count(scores_in_order, top_p: float):
+    """Top-p retention of Stage 1 (Sec. 4.2, text after Eq. 13; Sec. C.1: p = 0.95 for Qwen).
+
+    `scores_in_order` are the block scores s_ij taken along the computation order rho_i.
+    K_i is the length of the shortest prefix of rho_i whose scores sum to at least
+    top_p times the sum over all candidates (cumulated along rho_i, i.e. with the HRM
+    group first: the paper "retains the leading entries" of that order).  Returns
+    (K_i, margin): margin is the relative distance |cum - top_p*total| / total of the
+    closest of the two prefix sums that decide K_i (at K_i and at K_i - 1)."""
+    c = np.cumsum(np.asarray(scores_in_order, np.float64))
+    total = float(c[-1])
+    thr = float(top_p) * total
+    kept = len(c)
+    for t in range(len(c)):
+        if c[t] >= thr:
+            kept = t + 1
+            break
+    gaps = [abs(float(c[kept - 1]) - thr)]
+    if kept >= 2:
+        gaps.append(abs(float(c[kept - 2]) - thr))
+    return kept, min(gaps) / max(total, 1e-300)
+
+
 def kap_select(q, k, s=8, budget=0.25, causal=True, block=128, heads=None, query_blocks=None,
-               order_stride=None, audit=False):
+               order_stride=None, audit=False, top_p=None):
     """Ordered Stage-1 visit lists M_KAP (Eq. 14): order[h,i,:count] then -1 padding.
 
     Returns (order int32 [Hq,nQB,order_stride], count int32 [Hq,nQB]) and, if `audit`,
     a dict with the smallest decision margins met (relative gap between adjacent list
     entries of one group up to and including the retention boundary; absolute gap
-    between the two largest block maxima of a sampled row)."""
+    between the two largest block maxima of a sampled row).
+
+    `top_p` (None = off): K_i is the Top-p count of topp_count(), still capped by the
+    budget count (budget = 1 leaves Top-p alone); the audit then also holds the per-list
+    margins of that decision ("topp_margin" [Hq,nQB], inf where the cap decided)."""
     hq, n, _ = q.shape
     nqb = n // block
     nkb = nqb
@@ -202,11 +229,17 @@ def kap_select(q, k, s=8, budget=0.25, causal=True, block=128, heads=None, query
     order = np.full((hq, nqb, order_stride), -1, np.int32)
     count = np.zeros((hq, nqb), np.int32)
     min_rel_gap, min_top2 = np.inf, np.inf
+    topp_margin = np.full((hq, nqb), np.inf)
     for h in (range(hq) if heads is None else heads):
         for i in (range(nqb) if query_blocks is None else query_blocks):
             scores, flags, M = kap_scores(q, k, h, i, s, block, causal)
             rho = flag_grouped_order(scores, flags)
             K_i = budget_count(budget, len(rho))
+            if top_p is not None:
+                K_p, margin = topp_count(scores[rho], top_p)
+                if K_p <= K_i:
+                    K_i = K_p
+                    topp_margin[h, i] = margin
             order[h, i, :K_i] = rho[:K_i]
             count[h, i] = K_i
             if audit:
@@ -219,7 +252,8 @@ def kap_select(q, k, s=8, budget=0.25, causal=True, block=128, heads=None, query
                     top = np.sort(M, axis=1)
                     min_top2 = min(min_top2, float((top[:, -1] - top[:, -2]).min()))
     if audit:
-        return order, count, {"min_rel_score_gap": float(min_rel_gap), "min_row_top2_gap": float(min_top2)}
+        return order, count, {"min_rel_score_gap": float(min_rel_gap), "min_row_top2_gap": float(min_top2),
+                              "topp_margin": topp_margin}
     return order, count
 
 

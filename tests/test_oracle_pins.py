@@ -354,6 +354,71 @@ def test_budget_count_is_exact_ceiling():
             assert O.budget_count(b, J) == want, (b, J)
 
 
+# ---------------------------------------------------------------- Top-p retention (Sec. 4.2 / Sec. C.1)
+def test_topp_count_closed_forms():
+    # equal scores: the prefix sum is k, so K = ceil(p * J) (p * J not an integer here)
+    assert O.topp_count(np.ones(40), 0.33)[0] == 14
+    # p * J an integer: the prefix that reaches the threshold exactly is enough (>=), margin 0
+    kept, margin = O.topp_count(np.ones(40), 0.35)
+    assert kept == 14 and margin == 0.0
+    # geometric scores 2^-t (exact in binary): sum of k terms is 2 - 2^(1-k); 0.9 * total = 1.79999..:
+    # three terms give 1.75, four give 1.875
+    kept, margin = O.topp_count(0.5 ** np.arange(20), 0.9)
+    assert kept == 4
+    total = 2.0 - 2.0 ** -19
+    assert margin == pytest.approx(min(1.875 - 0.9 * total, 0.9 * total - 1.75) / total, rel=1e-12)
+    # p = 1 keeps everything, a vanishing p keeps the first entry only
+    rng = np.random.default_rng(5)
+    sc = rng.random(57) + 0.01
+    assert O.topp_count(sc, 1.0)[0] == 57 and O.topp_count(sc, 1e-12)[0] == 1
+    # monotone in p and minimal: one entry fewer does not reach the threshold
+    last = 1
+    for p_ in np.linspace(0.05, 0.99, 40):
+        kept, _ = O.topp_count(sc, p_)
+        assert kept >= last
+        assert math.fsum(sc[:kept]) >= p_ * math.fsum(sc) * (1 - 1e-14)
+        assert kept == 1 or math.fsum(sc[:kept - 1]) < p_ * math.fsum(sc) * (1 + 1e-14)
+        last = kept
+
+
+def test_topp_is_cumulated_along_the_flag_grouped_order():
+    # an HRM block with a small score comes first in rho and counts toward the prefix: scores (0.1*, 5, 4),
+    # p = 0.5 -> threshold 4.55: rho = (0, 1, 2), prefix sums 0.1, 5.1 -> two blocks; by score alone one would do
+    scores, flags = np.array([0.1, 5.0, 4.0]), np.array([True, False, False])
+    rho = O.flag_grouped_order(scores, flags)
+    assert rho == [0, 1, 2]
+    assert O.topp_count(scores[rho], 0.5)[0] == 2
+    assert O.topp_count(np.sort(scores)[::-1], 0.5)[0] == 1
+
+
+def test_kap_select_with_topp(small):
+    q, k, _, _ = small
+    nqb = q.shape[1] // 128
+    full, cfull = O.kap_select(q, k, s=8, budget=1.0)
+    # p = 1: whole candidate set; tiny p: the first entry; the list is always a prefix of the budget-1 list
+    _, c1 = O.kap_select(q, k, s=8, budget=1.0, top_p=1.0)
+    assert (c1 == cfull).all()
+    _, c0 = O.kap_select(q, k, s=8, budget=1.0, top_p=1e-9)
+    assert (c0 == 1).all()
+    order, count, audit = O.kap_select(q, k, s=8, budget=1.0, top_p=0.9, audit=True)
+    for h in range(q.shape[0]):
+        for i in range(nqb):
+            kept = count[h, i]
+            assert 1 <= kept <= i + 1
+            assert (order[h, i, :kept] == full[h, i, :kept]).all() and (order[h, i, kept:] == -1).all()
+            # the definition, summed independently (exactly rounded sums) over the scores of the kept blocks
+            scores, flags, _ = O.kap_scores(q, k, h, i, 8)
+            total = math.fsum(scores)
+            assert math.fsum(scores[order[h, i, :kept]]) >= 0.9 * total * (1 - 1e-13)
+            if kept > 1:
+                assert math.fsum(scores[order[h, i, :kept - 1]]) < 0.9 * total * (1 + 1e-13)
+    assert np.isfinite(audit["topp_margin"]).all()
+    # the budget count caps the Top-p count
+    _, ccap = O.kap_select(q, k, s=8, budget=0.25, top_p=0.9)
+    _, cb = O.kap_select(q, k, s=8, budget=0.25)
+    assert (ccap == np.minimum(count, cb)).all()
+
+
 def test_planted_structure_is_recalled():
     q, k, v, planted = _inputs(seed=11, hq=4, hkv=1, n=2048, needles=3)
     order, count = O.kap_select(q, k, s=8, budget=0.35)
