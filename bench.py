@@ -42,6 +42,8 @@ def parse():
     ap.add_argument("--no-comparators", action="store_true", help="skip the dense-path and SDPA timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--top-p", type=float, default=0.0,
+                    help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
     return ap.parse_args()
 
 
@@ -209,18 +211,20 @@ def main():
     pin = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)[None].contiguous().pin_memory()
     qh, kh, vh = pin(qb), pin(kb), pin(vb)
     q, k, v = (t.to(dev, non_blocking=True) for t in (qh, kh, vh))
-    pitch = order_pitch(cosa, w.kap_budget, nqb)
+    kap_budget = 1.0 if args.top_p > 0 else w.kap_budget
+    pitch = order_pitch(cosa, kap_budget, nqb)
     order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device=dev)
     count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
     out = torch.empty_like(q)
     lse = torch.empty(1, w.hq, w.n, dtype=torch.float32, device=dev)
     visited = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
     scored = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
-    opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=scored)
+    opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=scored,
+                               top_p=args.top_p)
     stream = torch.cuda.current_stream()
 
     def step():
-        cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt, stream=stream)
         cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
 
     def sync_all():
@@ -245,7 +249,7 @@ def main():
     t_wall = time.perf_counter()
     for s in range(args.steps):
         ev[s][0].record(stream)
-        cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt, stream=stream)
         ev[s][1].record(stream)
         cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
         ev[s][2].record(stream)
@@ -271,12 +275,12 @@ def main():
         lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
         vis_h = torch.empty(visited.shape, dtype=torch.int32).pin_memory()
         ke = max(1, min(args.steps, 3))
-        cosa.cosa_prefill_host(qh, kh, vh, shape, w.kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
+        cosa.cosa_prefill_host(qh, kh, vh, shape, kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
         sync_all()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(ke):
-            cosa.cosa_prefill_host(qh, kh, vh, shape, w.kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
+            cosa.cosa_prefill_host(qh, kh, vh, shape, kap_budget, w.osk_budget, out_h, lse_h, vis_h, ws, opt=opt, stream=stream)
         e1.record(stream)
         sync_all()
         e2e_ms = e0.elapsed_time(e1) / ke
@@ -352,7 +356,7 @@ def main():
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
-                           "kap_budget": w.kap_budget, "osk_budget": w.osk_budget, "stride": w.stride,
+                           "kap_budget": kap_budget, "top_p": args.top_p or None, "osk_budget": w.osk_budget, "stride": w.stride,
                            "skip_scale": w.skip_scale, "parallelism": f"layer-per-rank x{world}",
                            "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
                            "blocks_scored": n_scored, "blocks_computed": n_computed,

@@ -81,6 +81,11 @@ typedef struct {
                               which is allocated (cudaMalloc) on first use or growth             */
   size_t  workspace_bytes;
   int32_t impl;            /* 0 = fastest available; 1 = plain CUDA-core check kernels           */
+  float   top_p;           /* KAP only.  > 0: Top-p retention (Sec. 4.2, text after Eq. 13; p = 0.95
+                              in Sec. C.1): K_i = length of the shortest prefix of the order whose
+                              scores sum to >= top_p * (sum over all candidates), never more than
+                              the budget count (pass budget = 1 for Top-p alone); must be <= 1.
+                              0: the budget count alone (default)                                 */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);
@@ -102,7 +107,7 @@ int32_t cosa_budget_count(float budget, int32_t candidates);
  * maximum after the softmax (MaxNorm) -- i.e. Pbar[r,j] = exp(M[r,j] - max_j' M[r,j']) --,
  * sum over the block's sampled rows (score s_ij), flag blocks holding some row's maximum
  * (h_ij), sort by (h_ij descending, s_ij descending, j ascending) and keep the first
- * K_i = cosa_budget_count(budget, candidates) ids.
+ * K_i = cosa_budget_count(budget, candidates) ids (fewer with opt->top_p, see cosa_options).
  *
  *   q, k        in   device bf16, layouts above
  *   budget      in   Stage-1 fraction in (0, 1]
@@ -110,7 +115,9 @@ int32_t cosa_budget_count(float budget, int32_t candidates);
  *                    order_stride must be >= the largest K_i
  *   out_count   out  device int32 [B,Hq,nQB]
  * Scores are evaluated so that the list equals the one exact arithmetic would give whenever
- * neighbouring scores differ by more than ~1e-9 relative.
+ * neighbouring scores differ by more than ~1e-9 relative.  With top_p the prefix sums are taken over
+ * float32 scores (relative error < 2^-15): K_i equals the exact count unless a prefix sum lies
+ * within that error of the threshold, where it may differ by one.
  */
 int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape,
                     float budget, int32_t* out_order, int32_t* out_count, void* stream);

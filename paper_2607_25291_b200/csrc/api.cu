@@ -134,6 +134,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   cosa_options o = resolve_options(opt);
   const int s = o.stride;
   if (s < 1 || s > kBlock || (s & (s - 1)) != 0) return COSA_ERR_UNSUPPORTED;
+  if (!(o.top_p >= 0.f) || o.top_p > 1.f) return COSA_ERR_INVALID_ARG;
   const int nqb = shape->n / kBlock;
   const int order_stride = o.order_stride > 0 ? o.order_stride : nqb;
   KapParams p{};
@@ -150,6 +151,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   p.order_stride = order_stride;
   p.budget_fx = budget_to_fx(budget);
   p.scale = o.softmax_scale > 0.f ? (double)o.softmax_scale : 1.0 / sqrt((double)shape->d);
+  p.top_p = (double)o.top_p;
   // the list of the longest row must fit the pitch
   if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
   if (kap_exact_smem_bytes(p.rows, nqb) > 227 * 1024) return COSA_ERR_UNSUPPORTED;

@@ -27,6 +27,7 @@ struct KapParams {
   int order_stride;
   long long budget_fx;   // floor(budget_f32 * 2^20)
   double scale;          // softmax scale applied to the sampled logits
+  double top_p;          // > 0: Top-p retention, capped by the budget count; 0: budget count alone
 };
 
 // The float32 screen of the KAP fast path (tensor cores) and what it leaves for the sort stage.

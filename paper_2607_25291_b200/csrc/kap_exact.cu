@@ -2,7 +2,7 @@
 // (Sec. 4.2, Eqs. 8-14; Algorithm A steps 2-5).  One CTA per (query head, query block):
 //   sampled logits z[r,c] -> M[r,j] = max_{c in block j} z[r,c] -> M*[r] = max_j M[r,j]
 //   s_j = sum_r exp(M[r,j] - M*[r]),  h_j = any_r [M[r,j] == M*[r]]
-//   order = sort by (h desc, s desc, j asc);  keep K_i = budget_count(candidates).
+//   order = sort by (h desc, s desc, j asc);  keep K_i = budget_count(candidates), or the Top-p prefix.
 // Products of two bf16 values are exact in double, so scores carry ~1e-16 relative error.
 #include "common.cuh"
 
@@ -143,7 +143,26 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
       __syncthreads();
     }
   }
-  const int K = budget_count_fx(p.budget_fx, J);
+  int K = budget_count_fx(p.budget_fx, J);
+  if (p.top_p > 0.0) {
+    // Top-p retention (text after Eq. 13): prefix sums along the order, sequentially in double precision
+    __shared__ int k_topp;
+    if (tid == 0) {
+      double total = 0.0;
+      for (int t = 0; t < J; ++t) total += __longlong_as_double((long long)(keys[t] & ~(1ULL << 63)));
+      const double thr = p.top_p * total;
+      double run = 0.0;
+      int kept = J;
+      for (int t = 0; t < J; ++t) {
+        run += __longlong_as_double((long long)(keys[t] & ~(1ULL << 63)));
+        if (run >= thr) { kept = t + 1; break; }
+      }
+      k_topp = kept;
+    }
+    __syncthreads();
+    K = min(K, k_topp);
+    __syncthreads();   // the list kernel reuses k_topp for its next item
+  }
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
   int32_t* dst = p.order + row * p.order_stride;
   for (int t = tid; t < p.order_stride; t += kThreads) dst[t] = (t < K) ? (int32_t)ids[t] : -1;

@@ -1,4 +1,5 @@
-// KAP fast path, stage B: flag-grouped sort and budget prefix (Eqs. 13-14; Algorithm A step 5)
+// KAP fast path, stage B: flag-grouped sort and retained prefix (Eqs. 13-14; Algorithm A step 5;
+// budget count or Top-p, text after Eq. 13)
 // on the float32 screen, with a double-precision recount of every decision a rounding error
 // could change.
 //
@@ -225,7 +226,43 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
       }
     }
   }
-  const int K = budget_count_fx(p.budget_fx, J);
+  int K = budget_count_fx(p.budget_fx, J);
+  if (p.top_p > 0.0) {
+    // Top-p retention: the shortest prefix of the order whose scores reach top_p of the total.  Every thread
+    // owns a run of consecutive sorted entries; sums are double precision in a fixed order (deterministic).
+    __shared__ double warp_sum[kThreads / 32];
+    __shared__ int k_topp;
+    const int E = (P2 + kThreads - 1) / kThreads;
+    const int lane = tid & 31, wid = tid >> 5;
+    double loc = 0.0;
+    for (int q = 0; q < E; ++q) {
+      const int t = tid * E + q;
+      if (t < J) loc += (double)__uint_as_float((unsigned)(keys[t] >> 32) & 0x7fffffffu);
+    }
+    double incl = loc;
+    for (int o = 1; o < 32; o <<= 1) {
+      const double v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) warp_sum[wid] = incl;
+    if (tid == 0) k_topp = J;
+    __syncthreads();
+    double before = 0.0, total = 0.0;
+    for (int w = 0; w < kThreads / 32; ++w) {
+      if (w < wid) before += warp_sum[w];
+      total += warp_sum[w];
+    }
+    const double thr = p.top_p * total;
+    double run = before + (incl - loc);
+    for (int q = 0; q < E; ++q) {
+      const int t = tid * E + q;
+      if (t >= J) break;
+      run += (double)__uint_as_float((unsigned)(keys[t] >> 32) & 0x7fffffffu);
+      if (run >= thr) { atomicMin(&k_topp, t + 1); break; }
+    }
+    __syncthreads();
+    K = min(K, k_topp);
+  }
 
   // ---- 3. near ties between sorted neighbours
   for (int t = tid; t < P2; t += kThreads) {

@@ -10,7 +10,7 @@ from oracle import cosa_oracle as O
 from synth.configs import SWEEP_STAGE1, SWEEP_STAGE2_MULT, WORKLOADS
 from synth.generator import bf16_bits_to_f64
 from tests.helpers import to_dev
-from tests.test_gpu_parity import _np, check_osk_against_oracle
+from tests.test_gpu_parity import TOPP_MARGIN, _np, check_osk_against_oracle, check_topp_lists
 
 pytestmark = pytest.mark.gpu
 
@@ -37,7 +37,7 @@ class HeadView:
         return (self.cache[("q", h)],) + self.cache[("kv", g)]
 
 
-def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, blocks, check_all_kap=False):
+def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, blocks, check_all_kap=False, top_p=0.0):
     q, k, v = (to_dev(x) for x in (qb, kb, vb))
     nqb = w.n_blocks
     pitch = (cosa.cosa_budget_count(kap_budget, nqb) + 7) // 8 * 8
@@ -47,7 +47,7 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
                 visited=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
                 scored=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
                 decisions=torch.zeros(1, w.hq, nqb, (pitch + 31) // 32, dtype=torch.int32, device="cuda"))
-    opt = cosa.default_options(stride=w.stride, skip_scale=skip_scale, order_stride=pitch,
+    opt = cosa.default_options(stride=w.stride, skip_scale=skip_scale, order_stride=pitch, top_p=top_p,
                                out_scored=bufs["scored"], out_decisions=bufs["decisions"])
     cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt)
     cosa.cosa_osk_attention(q, k, v, order, count, osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
@@ -59,11 +59,14 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
     order_np, count_np = _np(order), _np(count)
     J = np.arange(1, nqb + 1)
     want_count = np.array([O.budget_count(kap_budget, int(j)) for j in J])
-    assert (count_np == want_count[None, :]).all()
+    if top_p > 0:
+        assert (count_np >= 1).all() and (count_np <= want_count[None, :]).all()
+    else:
+        assert (count_np == want_count[None, :]).all()
     vis, sco = _np(bufs["visited"]), _np(bufs["scored"])
     if osk_budget < 1.0:
         cap = np.minimum(want_count, np.array([O.budget_count(osk_budget, int(j)) for j in J]))
-        assert (vis <= cap[None, :]).all()
+        assert (vis <= np.minimum(cap[None, :], count_np)).all()
     else:
         assert (vis == count_np).all()
     assert (sco <= count_np).all() and (vis >= 1).all() and (vis <= sco).all()
@@ -76,12 +79,19 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
     stats = []
     for h in kap_heads:
         qf, kf, vf = hv.get(h)
-        ref_order, ref_count = O.kap_select(qf, kf, s=w.stride, budget=kap_budget, order_stride=pitch,
-                                            query_blocks=(None if check_all_kap else blocks))
         sel = range(nqb) if check_all_kap else blocks
-        for i in sel:
-            assert ref_count[0, i] == count_np[h, i], (h, i)
-            assert np.array_equal(ref_order[0, i], order_np[h, i]), (h, i)
+        if top_p > 0:
+            ref_order, ref_count, audit = O.kap_select(qf, kf, s=w.stride, budget=kap_budget, order_stride=pitch,
+                                                       query_blocks=(None if check_all_kap else blocks), top_p=top_p,
+                                                       audit=True)
+            check_topp_lists(order_np, count_np, ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[0],
+                             [(h, 0, i) for i in sel])
+        else:
+            ref_order, ref_count = O.kap_select(qf, kf, s=w.stride, budget=kap_budget, order_stride=pitch,
+                                                query_blocks=(None if check_all_kap else blocks))
+            for i in sel:
+                assert ref_count[0, i] == count_np[h, i], (h, i)
+                assert np.array_equal(ref_order[0, i], order_np[h, i]), (h, i)
         one = {k_: t[:, h:h + 1] for k_, t in bufs.items()}
         stats.append(check_osk_against_oracle(qf, kf, vf, order_np[h:h + 1], count_np[h:h + 1], one, osk_budget,
                                               skip_scale, [0], blocks))
@@ -106,6 +116,17 @@ def test_qwen3_128k_sampled():
                           sample_blocks(w.n_blocks))
     assert stats["computed"] < stats["scored"]
     print("128k", stats)
+
+
+def test_qwen3_32k_and_128k_topp_sampled():
+    """Stage 1 by Top-p (p = 0.95, no budget cap), Stage 2 as configured: lists of data-dependent length."""
+    for name, heads in (("qwen3_32k", range(0, 32, 5)), ("qwen3_128k", [3, 17, 30])):
+        w = WORKLOADS[name]
+        qb, kb, vb, _ = w.make()
+        stats = run_and_check(w, qb, kb, vb, 1.0, w.osk_budget, w.skip_scale, heads, sample_blocks(w.n_blocks), top_p=0.95)
+        pairs = w.hq * w.n_blocks * (w.n_blocks + 1) // 2
+        assert stats["listed"] < pairs
+        print(name, "top-p 0.95", stats, "listed fraction", stats["listed"] / pairs)
 
 
 def test_llama31_64k_budget_sweep_sampled():

@@ -26,7 +26,7 @@ def _np(t):
     return t[0].cpu().numpy()
 
 
-def run_kap(q, k, budget, stride=8, causal=True, order_stride=None, scores=False, impl=0):
+def run_kap(q, k, budget, stride=8, causal=True, order_stride=None, scores=False, impl=0, top_p=0.0):
     _, hq, n, _ = q.shape
     nqb = n // 128
     order, count = alloc_lists(hq, nqb, order_stride)
@@ -34,10 +34,35 @@ def run_kap(q, k, budget, stride=8, causal=True, order_stride=None, scores=False
     if scores:
         kw["kap_scores"] = torch.zeros(1, hq, nqb, nqb, dtype=torch.float32, device="cuda")
         kw["kap_flags"] = torch.zeros(1, hq, nqb, nqb, dtype=torch.uint8, device="cuda")
-    opt = cosa.default_options(stride=stride, impl=impl, **kw)
+    opt = cosa.default_options(stride=stride, impl=impl, top_p=top_p, **kw)
     cosa.cosa_kap_select(q, k, budget, order, count, causal=causal, opt=opt)
     assert cosa.cosa_device_status() == 0
     return (order, count, kw) if scores else (order, count)
+
+
+# Top-p counts come from prefix sums of float32 scores (relative error < 2^-15) on the fast path and of double
+# precision scores (a few ulp from the oracle's) in the exact kernel: the count must equal the oracle's unless the
+# oracle's own prefix sum lies within that error of the threshold, where it may differ by one.
+TOPP_MARGIN = {0: 2.0 ** -14, 1: 1e-12}
+
+
+def check_topp_lists(order_np, count_np, ref_order, ref_count, margin, tol, pairs):
+    """GPU lists against the oracle's Top-p lists for the (h_gpu, h_ref, i) triples in `pairs`."""
+    off = 0
+    for hg, hr, i in pairs:
+        kept, want = int(count_np[hg, i]), int(ref_count[hr, i])
+        if margin[hr, i] > tol:
+            assert kept == want, (hg, i, kept, want, margin[hr, i])
+        else:
+            assert abs(kept - want) <= 1, (hg, i, kept, want)
+            off += kept != want
+        both = min(kept, want)
+        assert np.array_equal(order_np[hg, i, :both], ref_order[hr, i, :both]), (hg, i)
+        assert (order_np[hg, i, kept:] == -1).all()
+        if kept > want:                                     # one more entry than the oracle: a fresh candidate id
+            extra = int(order_np[hg, i, want])
+            assert 0 <= extra <= i and extra not in set(ref_order[hr, i, :want].tolist())
+    return off
 
 
 def run_osk(q, k, v, order, count, tb, skip_scale, impl=0, causal=True):
@@ -130,6 +155,43 @@ def test_kap_lists_bit_exact_small(small, stride, budget, impl):
     ref_order, ref_count = O.kap_select(qf, kf, s=stride, budget=budget, order_stride=order.shape[-1])
     assert np.array_equal(_np(count), ref_count)
     assert np.array_equal(_np(order), ref_order)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("top_p,budget", [(0.5, 1.0), (0.9, 1.0), (0.95, 1.0), (1.0, 1.0), (0.95, 0.3)])
+def test_kap_topp_small(small, impl, top_p, budget):
+    q, k, _ = small["dev"]
+    qf, kf, _ = small["f64"]
+    for stride in (8, 32):
+        order, count = run_kap(q, k, budget, stride, impl=impl, top_p=top_p)
+        ref_order, ref_count, audit = O.kap_select(qf, kf, s=stride, budget=budget, order_stride=order.shape[-1],
+                                                   top_p=top_p, audit=True)
+        pairs = [(h, h, i) for h in range(qf.shape[0]) for i in range(qf.shape[1] // 128)]
+        check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs)
+        if top_p == 1.0:
+            assert np.array_equal(_np(count), ref_count)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_kap_topp_4k(cfg1, impl):
+    q, k, _ = cfg1["dev"]
+    qf, kf, _ = cfg1["f64"]
+    w = cfg1["w"]
+    order, count = run_kap(q, k, 1.0, w.stride, impl=impl, top_p=0.95)
+    ref_order, ref_count, audit = O.kap_select(qf, kf, s=w.stride, budget=1.0, order_stride=order.shape[-1],
+                                               top_p=0.95, audit=True)
+    pairs = [(h, h, i) for h in range(w.hq) for i in range(w.n_blocks)]
+    off = check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs)
+    assert off <= 2
+    assert (ref_count < np.arange(1, w.n_blocks + 1)[None, :]).any()      # Top-p does drop blocks on this workload
+
+
+def test_kap_topp_rejects_bad_p(small):
+    q, k, _ = small["dev"]
+    order, count = alloc_lists(q.shape[1], q.shape[2] // 128, None)
+    for bad in (-0.1, 1.5, float("nan")):
+        with pytest.raises(cosa.CosaError):
+            cosa.cosa_kap_select(q, k, 1.0, order, count, opt=cosa.default_options(top_p=bad))
 
 
 @pytest.mark.parametrize("impl", IMPLS)
