@@ -258,6 +258,51 @@ def kap_select(q, k, s=8, budget=0.25, causal=True, block=128, heads=None, query
 
 
 # ----------------------------------------------------------------------------
+# List utilities for the remapping analysis (Sec. 5.3 "Effect of remapping") and the
+# logical-mask comparison (Sec. D "Kernel Microbenchmark")
+# ----------------------------------------------------------------------------
+def lists_reordered(order, count, descending=False):
+    """The same kept sets visited in natural page order (ascending block id: execution
+    "without remapping") or in descending id order; padding stays -1."""
+    out = np.full_like(order, -1)
+    for h in range(order.shape[0]):
+        for i in range(order.shape[1]):
+            ids = sorted(int(x) for x in order[h, i, :count[h, i]])
+            if descending:
+                ids.reverse()
+            out[h, i, :len(ids)] = ids
+    return out
+
+
+def lists_to_mask(order, count, n_kblocks):
+    """The binary block mask of Eq. (3) for the kept sets: uint32 words [Hq,nQB,ceil(nKB/32)],
+    block j is bit (j mod 32) of word (j div 32)."""
+    words = (n_kblocks + 31) // 32
+    mask = np.zeros(order.shape[:2] + (words,), np.uint32)
+    for h in range(order.shape[0]):
+        for i in range(order.shape[1]):
+            for j in order[h, i, :count[h, i]]:
+                mask[h, i, int(j) // 32] |= np.uint32(1 << (int(j) % 32))
+    return mask
+
+
+def mask_to_lists(mask, n_kblocks, causal=True, order_stride=None):
+    """The visiting sequence of a kernel that walks the candidates j = 0, 1, ... and skips the
+    ones whose mask bit is clear ("logical skipping"): the kept ids in ascending order.  Bits of
+    non-candidates (j > i when causal, j >= nKB) are ignored."""
+    hq, nqb, _ = mask.shape
+    order_stride = order_stride or n_kblocks
+    order = np.full((hq, nqb, order_stride), -1, np.int32)
+    count = np.zeros((hq, nqb), np.int32)
+    for h in range(hq):
+        for i in range(nqb):
+            ids = [j for j in range(n_candidates(i, n_kblocks, causal)) if (int(mask[h, i, j // 32]) >> (j % 32)) & 1]
+            order[h, i, :len(ids)] = ids
+            count[h, i] = len(ids)
+    return order, count
+
+
+# ----------------------------------------------------------------------------
 # OSK: ordered traversal with the in-kernel skip
 # ----------------------------------------------------------------------------
 def skip_threshold(skip_scale: float, n: int) -> float:

@@ -419,6 +419,54 @@ def test_kap_select_with_topp(small):
     assert (ccap == np.minimum(count, cb)).all()
 
 
+# ---------------------------------------------------------------- list utilities (remapping analysis, logical mask)
+def test_list_utilities_against_hand_example_and_bruteforce():
+    order = np.array([[[0, -1, -1, -1], [1, 0, -1, -1], [2, 0, 1, -1]]], np.int32)      # causal lists, nQB = 3
+    count = np.array([[1, 2, 3]], np.int32)
+    assert O.lists_reordered(order, count).tolist() == [[[0, -1, -1, -1], [0, 1, -1, -1], [0, 1, 2, -1]]]
+    assert O.lists_reordered(order, count, descending=True).tolist() == [[[0, -1, -1, -1], [1, 0, -1, -1], [2, 1, 0, -1]]]
+    # bit packing: block 33 is bit 1 of word 1, block 5 is bit 5 of word 0
+    big = np.full((1, 40, 40), -1, np.int32)
+    cnt = np.ones((1, 40), np.int32)
+    big[0, :, 0] = 0
+    big[0, 39, :3] = [33, 0, 5]
+    cnt[0, 39] = 3
+    mask = O.lists_to_mask(big, cnt, 40)
+    assert mask.shape == (1, 40, 2) and mask[0, 39].tolist() == [0x21, 0x2] and mask[0, 7].tolist() == [1, 0]
+    # round trip on random causal sets: mask -> walk gives the ascending list; non-candidate bits are ignored
+    rng = np.random.default_rng(3)
+    nqb = 70
+    order = np.full((2, nqb, nqb), -1, np.int32)
+    count = np.zeros((2, nqb), np.int32)
+    for h in range(2):
+        for i in range(nqb):
+            ids = rng.permutation(i + 1)[:rng.integers(1, i + 2)]
+            order[h, i, :len(ids)] = ids
+            count[h, i] = len(ids)
+    mask = O.lists_to_mask(order, count, nqb)
+    for h in range(2):
+        for i in range(nqb):
+            assert {j for j in range(nqb) if (int(mask[h, i, j // 32]) >> (j % 32)) & 1} == set(order[h, i, :count[h, i]].tolist())
+    noisy = mask.copy()
+    noisy[:, :5, 2] = 0xffffffff                                             # blocks 64.. are no candidates of rows 0..4
+    back, bcount = O.mask_to_lists(noisy, nqb)
+    assert np.array_equal(back, O.lists_reordered(order, count)) and np.array_equal(bcount, count)
+
+
+def test_natural_order_keeps_the_set_but_changes_the_decisions(small):
+    """Order invariance (Eq. 4) holds with Stage 2 off; with the skip rule on, the visiting order matters
+    (Sec. 3.3, Limitation 2): the remapping analysis rests on exactly this."""
+    q, k, v, _ = small
+    order, count = O.kap_select(q, k, s=8, budget=0.75)
+    nat = O.lists_reordered(order, count)
+    a = O.osk_attention(q, k, v, order, count, tightened_budget=1.0)
+    b = O.osk_attention(q, k, v, nat, count, tightened_budget=1.0)
+    assert np.abs(a["out"] - b["out"]).max() < 1e-12
+    c = O.osk_attention(q, k, v, order, count, skip_scale=300.0, tightened_budget=0.999)
+    d = O.osk_attention(q, k, v, nat, count, skip_scale=300.0, tightened_budget=0.999)
+    assert c["visited"].sum() < d["visited"].sum()          # HRM-first order lets more blocks fall below the threshold
+
+
 def test_planted_structure_is_recalled():
     q, k, v, planted = _inputs(seed=11, hq=4, hkv=1, n=2048, needles=3)
     order, count = O.kap_select(q, k, s=8, budget=0.35)
