@@ -86,6 +86,13 @@ typedef struct {
                               scores sum to >= top_p * (sum over all candidates), never more than
                               the budget count (pass budget = 1 for Top-p alone); must be <= 1.
                               0: the budget count alone (default)                                 */
+  const uint32_t* logical_mask; /* OSK only.  Non-NULL: instead of the order lists the kernel walks this binary
+                              block mask (Eq. 3) [B,Hq,nQB,ceil(nQB/32)], block j = bit (j mod 32) of
+                              word (j div 32): candidates are tested one by one in ascending order and
+                              the blocks whose bit is clear are stepped over ("logical skipping", the
+                              execution style OSK's index-driven jumping is compared with in Sec. D).
+                              `order` and `count` may then be NULL; list positions in the outputs
+                              are ranks among the kept blocks                                       */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);
@@ -181,6 +188,19 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
                           const int32_t* order, const int32_t* count, float tightened_budget,
                           void* out, float* out_lse, int32_t* out_visited, void* stream,
                           const cosa_options* opt);
+
+/*
+ * List rearrangements for the remapping analysis (Sec. 5.3 "Effect of remapping") and the logical-mask
+ * comparison (Sec. D).  Device pointers, enqueue-only.
+ *   cosa_reorder_lists  sorts the first count ids of every list by block id in place: descending == 0
+ *                       gives natural page order (execution without remapping), != 0 the reverse.
+ *   cosa_lists_to_mask  writes the binary block mask of Eq. (3) of the kept sets to out_mask
+ *                       [B,Hq,nQB,ceil(nQB/32)] (layout as cosa_options.logical_mask).
+ */
+int cosa_reorder_lists(int32_t* order, const int32_t* count, const cosa_shape* shape, int32_t order_stride,
+                       int32_t descending, void* stream);
+int cosa_lists_to_mask(const int32_t* order, const int32_t* count, const cosa_shape* shape, int32_t order_stride,
+                       uint32_t* out_mask, void* stream);
 
 /*
  * Read-only check of caller-built lists (Eq. 14 encoding): every id at a position < count is

@@ -28,7 +28,7 @@ COSA_ERR_BAD_ORDER = -6
 
 EXPORTS = (
     "cosa_default_options", "cosa_workspace_bytes", "cosa_budget_count", "cosa_kap_select",
-    "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_validate_order",
+    "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_reorder_lists", "cosa_lists_to_mask", "cosa_validate_order",
     "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status",
     "cosa_last_cuda_error", "cosa_status_string", "cosa_version",
 )
@@ -43,7 +43,7 @@ class CosaOptions(Structure):
     _fields_ = [("stride", c_int32), ("skip_scale", c_float), ("softmax_scale", c_float),
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
-                ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float)]
+                ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p)]
 
 
 class CosaError(RuntimeError):
@@ -82,6 +82,8 @@ def _load():
                                        c_void_p, c_void_p, c_void_p, c_void_p]
     lib.cosa_osk_attention_ex.argtypes = lib.cosa_osk_attention.argtypes + [POINTER(CosaOptions)]
     lib.cosa_validate_order.argtypes = [c_void_p, c_void_p, POINTER(CosaShape), c_int32, c_void_p, c_void_p]
+    lib.cosa_reorder_lists.argtypes = [c_void_p, c_void_p, POINTER(CosaShape), c_int32, c_int32, c_void_p]
+    lib.cosa_lists_to_mask.argtypes = [c_void_p, c_void_p, POINTER(CosaShape), c_int32, c_void_p, c_void_p]
     lib.cosa_host_call_workspace_bytes.argtypes = [POINTER(CosaShape), POINTER(CosaOptions)]
     lib.cosa_host_call_workspace_bytes.restype = c_size_t
     lib.cosa_prefill_host.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(CosaShape), c_float, c_float, c_void_p,
@@ -91,7 +93,7 @@ def _load():
     lib.cosa_status_string.argtypes = [c_int]
     lib.cosa_status_string.restype = c_char_p
     for name in ("cosa_kap_select", "cosa_kap_select_ex", "cosa_osk_attention", "cosa_osk_attention_ex",
-                 "cosa_validate_order", "cosa_prefill_host", "cosa_device_status", "cosa_version"):
+                 "cosa_validate_order", "cosa_reorder_lists", "cosa_lists_to_mask", "cosa_prefill_host", "cosa_device_status", "cosa_version"):
         getattr(lib, name).restype = c_int
     _lib = lib
     return lib
@@ -197,7 +199,7 @@ def cosa_osk_attention(q, k, v, order, count, tightened_budget: float, out, out_
             raise ValueError("without options the order tensor must have pitch nQB")
         _check(lib.cosa_osk_attention(*args), "cosa_osk_attention")
     else:
-        if opt.order_stride == 0:
+        if opt.order_stride == 0 and order is not None:
             opt.order_stride = order.shape[-1]
         _check(lib.cosa_osk_attention_ex(*args, byref(opt)), "cosa_osk_attention_ex")
 
@@ -206,6 +208,20 @@ def cosa_validate_order(order, count, shape: CosaShape, status_word: torch.Tenso
     _check(_load().cosa_validate_order(_dev_ptr(order, torch.int32, "order"), _dev_ptr(count, torch.int32, "count"),
                                        byref(shape), order.shape[-1], _dev_ptr(status_word, torch.int32, "status"),
                                        _stream_ptr(stream)), "cosa_validate_order")
+
+
+def cosa_reorder_lists(order, count, shape: CosaShape, descending=False, stream=None):
+    """Sorts the kept ids of every list by block id in place (ascending = natural page order)."""
+    _check(_load().cosa_reorder_lists(_dev_ptr(order, torch.int32, "order"), _dev_ptr(count, torch.int32, "count"),
+                                      byref(shape), order.shape[-1], 1 if descending else 0, _stream_ptr(stream)),
+           "cosa_reorder_lists")
+
+
+def cosa_lists_to_mask(order, count, shape: CosaShape, out_mask, stream=None):
+    """Binary block mask [B,Hq,nQB,ceil(nQB/32)] (int32 tensor holding the uint32 words) of the kept sets."""
+    _check(_load().cosa_lists_to_mask(_dev_ptr(order, torch.int32, "order"), _dev_ptr(count, torch.int32, "count"),
+                                      byref(shape), order.shape[-1], _dev_ptr(out_mask, torch.int32, "out_mask"),
+                                      _stream_ptr(stream)), "cosa_lists_to_mask")
 
 
 def cosa_host_call_workspace_bytes(shape: CosaShape, opt: CosaOptions | None = None) -> int:

@@ -203,16 +203,18 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
                           int32_t* out_visited, void* stream, const cosa_options* opt) {
   int rc = check_shape(shape);
   if (rc != COSA_OK) return rc;
-  if (!q || !k || !v || !order || !count || !out) return COSA_ERR_INVALID_ARG;
+  if (!q || !k || !v || !out) return COSA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return COSA_ERR_INVALID_ARG;
   if (!(tightened_budget > 0.f)) return COSA_ERR_INVALID_ARG;
   cosa_options o = resolve_options(opt);
+  if (!o.logical_mask && (!order || !count)) return COSA_ERR_INVALID_ARG;
   const int nqb = shape->n / kBlock;
   OskParams p{};
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.k = static_cast<const __nv_bfloat16*>(k);
   p.v = static_cast<const __nv_bfloat16*>(v);
-  p.order = order; p.count = count;
+  p.order = o.logical_mask ? nullptr : order; p.count = o.logical_mask ? nullptr : count;
+  p.mask = o.logical_mask;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = out_lse; p.visited = out_visited;
   p.scored = o.out_scored; p.decisions = o.out_decisions;
@@ -247,6 +249,30 @@ int cosa_validate_order(const int32_t* order, const int32_t* count, const cosa_s
   cudaError_t e = launch_validate_order(order, count, shape->batch * shape->hq * nqb, nqb, shape->causal ? 1 : 0,
                                         order_stride, out_status_dev, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return cuda_fail(e, "validate launch");
+  return COSA_OK;
+}
+
+int cosa_reorder_lists(int32_t* order, const int32_t* count, const cosa_shape* shape, int32_t order_stride,
+                       int32_t descending, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!order || !count || order_stride < 1) return COSA_ERR_INVALID_ARG;
+  const int nqb = shape->n / kBlock;
+  cudaError_t e = launch_reorder_lists(order, count, shape->batch * shape->hq * nqb, order_stride, descending ? 1 : 0,
+                                       static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "reorder launch");
+  return COSA_OK;
+}
+
+int cosa_lists_to_mask(const int32_t* order, const int32_t* count, const cosa_shape* shape, int32_t order_stride,
+                       uint32_t* out_mask, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != COSA_OK) return rc;
+  if (!order || !count || !out_mask || order_stride < 1) return COSA_ERR_INVALID_ARG;
+  const int nqb = shape->n / kBlock;
+  cudaError_t e = launch_lists_to_mask(order, count, shape->batch * shape->hq * nqb, order_stride, nqb, out_mask,
+                                       static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "mask launch");
   return COSA_OK;
 }
 

@@ -52,6 +52,7 @@ struct OskParams {
   const __nv_bfloat16* v;
   const int32_t* order;
   const int32_t* count;
+  const uint32_t* mask;  // non-null: logical-mask walk instead of the lists (order and count unused)
   __nv_bfloat16* out;
   float* lse;            // optional
   int32_t* visited;      // optional
@@ -65,6 +66,40 @@ struct OskParams {
   long long cap_fx;      // floor(tightened_budget_f32 * 2^20)
   float theta;           // ln(Delta / N)
   float scale;           // softmax scale
+};
+
+// Where the kk-th visited key block of one (head, query block) comes from.  List mode: the order list, read
+// directly ("physical jumping", Sec. 4.3).  Mask mode: a binary block mask (Eq. 3) walked candidate by
+// candidate in ascending order, skipping the blocks whose bit is clear ("logical skipping", the execution
+// style OSK is compared with in Sec. D).  Positions must be asked for in increasing order.
+struct BlockWalk {
+  const int32_t* list;
+  const uint32_t* mask;
+  int nqb, J, j, rank;
+  __device__ __forceinline__ void init(const OskParams& p, size_t row, int candidates) {
+    list = p.order ? p.order + row * p.order_stride : nullptr;
+    mask = p.mask ? p.mask + row * (size_t)((p.nqb + 31) / 32) : nullptr;
+    nqb = p.nqb; J = candidates; j = 0; rank = 0;
+  }
+  // number of kept candidates (mask mode)
+  __device__ __forceinline__ int kept() const {
+    int c = 0;
+    for (int w = 0; w * 32 < J; ++w) {
+      uint32_t v = mask[w];
+      if ((w + 1) * 32 > J) v &= (1u << (J - w * 32)) - 1u;
+      c += __popc(v);
+    }
+    return c;
+  }
+  __device__ __forceinline__ int at(int kk) {
+    if (!mask) return min(max(list[kk], 0), nqb - 1);
+    while (j < J) {
+      const bool keep = (mask[j >> 5] >> (j & 31)) & 1u;
+      ++j;
+      if (keep && rank++ == kk) return j - 1;
+    }
+    return J - 1;   // asked for more positions than the mask keeps: stay inside the tensor
+  }
 };
 
 // ceil(fx * candidates / 2^20) clamped to [1, candidates]  (rounding of Eq. 14's K_i = B x J)
@@ -92,6 +127,10 @@ cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float
 size_t kap_exact_smem_bytes(int rows, int nqb);
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
+cudaError_t launch_reorder_lists(int32_t* order, const int32_t* count, int total_qb, int order_stride, int descending,
+                                 cudaStream_t st);
+cudaError_t launch_lists_to_mask(const int32_t* order, const int32_t* count, int total_qb, int order_stride, int nkb,
+                                 uint32_t* mask, cudaStream_t st);
 cudaError_t launch_validate_order(const int32_t* order, const int32_t* count, int total_qb, int nqb,
                                   int causal, int order_stride, int32_t* status, cudaStream_t st);
 

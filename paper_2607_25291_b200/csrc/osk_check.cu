@@ -26,9 +26,10 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
   const int g = h / (p.hq / p.hkv);
   const int t = threadIdx.x;  // query row inside the tile
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  const int cnt = max(0, min(p.count[row], p.order_stride));
-  const int32_t* list = p.order + row * p.order_stride;
   const int J = p.causal ? i + 1 : p.nqb;
+  BlockWalk walk;
+  walk.init(p, row, J);
+  const int cnt = p.mask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
   const int dec_words = (p.order_stride + 31) / 32;
 
@@ -53,7 +54,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
 
   for (int kk = 0; kk < cnt; ++kk) {
     if (computed == cap) break;  // uniform over the CTA
-    const int j = min(max(list[kk], 0), p.nqb - 1);
+    const int j = walk.at(kk);
     __syncthreads();
     for (int e = t; e < kBlock * kHeadDim / 8; e += kRows) {
       reinterpret_cast<uint4*>(Ksm)[e] = kbase[(size_t)j * (kBlock * kHeadDim / 8) + e];

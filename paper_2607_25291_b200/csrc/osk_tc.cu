@@ -84,6 +84,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
+// list-driven kernel carries none of the walk's state
+template <bool kMask>
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
@@ -111,9 +114,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const int i = p.nqb - 1 - (wk % per_kv) / G;
   const int h = g * G + (wk % per_kv) % G;
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  const int cnt = max(0, min(p.count[row], p.order_stride));
-  const int32_t* list = p.order + row * p.order_stride;
   const int J = p.causal ? i + 1 : p.nqb;
+  const int32_t* list = p.order + row * p.order_stride;   // unused when kMask
+  BlockWalk walk;                         // (kMask only) every thread that needs block ids walks on its own
+  if (kMask) walk.init(p, row, J);
+  const int cnt = kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
   const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N, d] view
   const int kv_row0 = (b * p.hkv + g) * p.n;              // first row of this KV head
@@ -125,8 +130,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   int poisoned_early = 0;
   if (threadIdx.x == 0) {
     poisoned_early = *reinterpret_cast<volatile int32_t*>(status);
+    if (kMask) {
+      for (int kk = 0; kk < kKStages; ++kk) first_ids[kk] = kk < min(cnt, cap) ? walk.at(kk) : 0;   // exactly the tiles requested below
+    } else {
 #pragma unroll
-    for (int kk = 0; kk < kKStages; ++kk) first_ids[kk] = kk < p.order_stride ? list[kk] : 0;
+      for (int kk = 0; kk < kKStages; ++kk)   // not waiting for the count: entries past it are never used
+        first_ids[kk] = kk < p.order_stride ? list[kk] : 0;
+    }
   }
 
   static_assert(kVStages == 2 && kKStages == 4, "PV product n frees V stage n & 1 together with p_empty[n & 1]");
@@ -208,7 +218,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           if (!*abort_flag) report_timeout(ctl, status);
           break;
         }
-        const int j = min(max(list[kk], 0), p.nqb - 1);
+        const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
         const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
         mbar_expect_tx(bar, kTileBytes);
         tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
@@ -278,7 +288,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     bool alive = true;
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int par = kk & 1;
-      const int j = min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
+      const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
       alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
@@ -362,7 +372,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       mbar_arrive(smem_u32(&ctl->q_full));
     }
     for (int kk = grp; kk < cnt && alive; kk += 2) {
-      const int j = min(max(list[kk], 0), p.nqb - 1);
+      // only "is this the diagonal block" matters here; an ascending mask walk meets it last, if at all
+      const int j = kMask ? ((kk == cnt - 1 && ((walk.mask[i >> 5] >> (i & 31)) & 1u)) ? i : -1)
+                           : min(max(list[kk], 0), p.nqb - 1);
       // wait for S(kk), or learn that the walk ended before this position
       {
         const uint32_t bar = smem_u32(&ctl->k_empty[kk % kKStages]), par = (kk / kKStages) & 1;   // QK^T(kk) finished
@@ -560,7 +572,8 @@ cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
   if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, (uint64_t)p.batch * p.hkv * p.n) ||
       !make_tile_map(&vm, p.v, (uint64_t)p.batch * p.hkv * p.n) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
     return cudaErrorInvalidValue;
-  cudaError_t e = cudaFuncSetAttribute(osk_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  auto kernel = p.mask ? osk_tc_kernel<true> : osk_tc_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
   if (p.decisions) {
     size_t words = (size_t)p.batch * p.hq * p.nqb * ((p.order_stride + 31) / 32);
@@ -569,7 +582,7 @@ cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
   }
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;
-  osk_tc_kernel<<<p.batch * p.hq * p.nqb, kThreads, kSmemBytes, st>>>(qm, km, vm, om, p, status);
+  kernel<<<p.batch * p.hq * p.nqb, kThreads, kSmemBytes, st>>>(qm, km, vm, om, p, status);
   return cudaGetLastError();
 }
 

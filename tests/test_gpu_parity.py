@@ -312,6 +312,78 @@ def test_osk_noncausal(small, impl):
     check_osk_against_oracle(qf, kf, vf, order_np, count_np, bufs, 0.5, 300.0, range(4), range(8), causal=False)
 
 
+# ---------------------------------------------------------------------------------- list tools, logical-mask walk
+def test_list_tools_bit_exact(small, cfg1):
+    for fx, budget in ((small, 0.6), (cfg1, 0.45)):
+        q, k, _ = fx["dev"]
+        order, count = run_kap(q, k, budget)
+        order_np, count_np = _np(order), _np(count)
+        shape = cosa.make_shape(q, k, True)
+        nqb = q.shape[2] // 128
+        mask = torch.full((1, q.shape[1], nqb, (nqb + 31) // 32), -1, dtype=torch.int32, device="cuda")
+        cosa.cosa_lists_to_mask(order, count, shape, mask)
+        assert np.array_equal(_np(mask).view(np.uint32), O.lists_to_mask(order_np, count_np, nqb))
+        for desc in (False, True):
+            o2 = order.clone()
+            cosa.cosa_reorder_lists(o2, count, shape, descending=desc)
+            assert np.array_equal(_np(o2), O.lists_reordered(order_np, count_np, descending=desc))
+    # a list of one, and lists longer than one sorting pass of a warp
+    o3 = torch.tensor([[[[5, -1, -1, -1], [3, 1, 2, 0]]]], dtype=torch.int32, device="cuda").expand(1, 1, 2, 4).contiguous()
+    c3 = torch.tensor([[[1, 4]]], dtype=torch.int32, device="cuda")
+    sh = cosa.CosaShape(1, 1, 1, 256, 128, 128, 128, 0)
+    cosa.cosa_reorder_lists(o3, c3, sh)
+    assert _np(o3).tolist() == [[[5, -1, -1, -1], [0, 1, 2, 3]]]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("tb,skip_scale", [(1.0, 200.0), (0.4, 150.0)])
+def test_osk_logical_mask_walk(small, cfg1, impl, tb, skip_scale):
+    """Walking the binary mask visits the kept blocks in ascending order: same decisions and outputs as the
+    ascending lists (bit for bit on the GPU, within tolerance against the oracle)."""
+    for fx, budget in ((small, 0.6), (cfg1, 0.45)):
+        q, k, v = fx["dev"]
+        qf, kf, vf = fx["f64"]
+        nqb = q.shape[2] // 128
+        order, count = run_kap(q, k, budget)
+        shape = cosa.make_shape(q, k, True)
+        mask = torch.zeros(1, q.shape[1], nqb, (nqb + 31) // 32, dtype=torch.int32, device="cuda")
+        cosa.cosa_lists_to_mask(order, count, shape, mask)
+        mask[0, :, 0, -1] |= 1 << 30                                      # a non-candidate bit must be ignored
+        bufs = alloc_outputs(q, nqb)
+        opt = cosa.default_options(skip_scale=skip_scale, impl=impl, out_scored=bufs["scored"],
+                                   out_decisions=bufs["decisions"], logical_mask=mask, order_stride=nqb)
+        cosa.cosa_osk_attention(q, k, v, None, None, tb, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+        assert cosa.cosa_device_status() == 0
+        ref_order, ref_count = O.mask_to_lists(_np(mask).view(np.uint32), nqb, order_stride=nqb)
+        heads = range(q.shape[1]) if fx is small else [0, q.shape[1] - 1]
+        blocks = range(nqb) if fx is small else [0, 1, 7, 30, 31]
+        check_osk_against_oracle(qf, kf, vf, ref_order, ref_count, bufs, tb, skip_scale, heads, blocks)
+        asc = torch.from_numpy(ref_order).cuda()[None].contiguous()
+        cnt = torch.from_numpy(ref_count).cuda()[None].contiguous()
+        ref = run_osk(q, k, v, asc, cnt, tb, skip_scale, impl)
+        assert torch.equal(ref["out"], bufs["out"]) and torch.equal(ref["visited"], bufs["visited"])
+        assert torch.equal(ref["scored"], bufs["scored"]) and torch.equal(ref["lse"], bufs["lse"])
+
+
+def test_ablation_tables_run_and_show_the_effect_of_order():
+    from paper_2607_25291_b200 import ablation
+    w = WORKLOADS["gqa4_4k"]
+    rows = ablation.remap_table(w, budgets=(1.0, 0.5), deltas=(200.0, 800.0, 3000.0))
+    assert len(rows) == 6
+    for r in rows:
+        assert 0.0 <= r["skip_natural"] <= 1.0 and 0.0 <= r["skip_remap"] <= 1.0
+        assert np.isfinite(r["err_remap"]) and np.isfinite(r["err_natural"])
+    # visiting the HRM blocks first lets more of the rest fall below the threshold (Sec. 5.3)
+    assert sum(r["skip_remap"] for r in rows) > sum(r["skip_natural"] for r in rows)
+    # a larger Delta skips more, in either order
+    for b in (1.0, 0.5):
+        sel = [r for r in rows if r["stage1"] == b]
+        assert sel[0]["skip_remap"] <= sel[1]["skip_remap"] <= sel[2]["skip_remap"]
+        assert sel[0]["skip_natural"] <= sel[1]["skip_natural"] <= sel[2]["skip_natural"]
+    micro = ablation.micro_table([w], budgets=(0.5,), with_sdpa=False)
+    assert len(micro) == 1 and micro[0]["jump_ms"] > 0 and micro[0]["logical_ms"] > 0 and micro[0]["dense_ms"] > 0
+
+
 def test_osk_is_deterministic(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
