@@ -44,6 +44,9 @@ constexpr int kHalfBytes = kTileBytes / 2;         // one TMA box: 128 rows x 64
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kDecRing = 16;
+constexpr int kSpec = 2;   // K tiles fetched and products issued ahead of the blocks that are certain to be scored: when the cap
+                           // binds, certainty grows one block per decision and each block would otherwise wait out a full
+                           // tile fetch + product (at most 2: the S buffer of position kk is freed by position kk-2)
 constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks before this position
 constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
@@ -204,15 +207,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else if (warp == 0) {
     // ------------------------------------------------------------------ K loader
     if (lane == 0) {
-      for (int kk = min(min(cnt, cap), kKStages); kk < cnt; ++kk) {   // the first tiles were requested in the prologue
+      int last_issued = min(min(cnt, cap), kKStages) - 1;
+      for (int kk = last_issued + 1; kk < cnt; ++kk) {   // the first tiles were requested in the prologue
         const long long t0 = clock64();
         bool ok = true;
-        while (kk >= ctl->n_needed) {          // not yet certain that this block will be scored
+        while (kk >= ctl->n_needed + kSpec) {  // at most kSpec tiles beyond the blocks that are certain to be scored
           if (ctl->end_kk >= 0) { ok = false; break; }
           if (*abort_flag || clock64() - t0 > kWaitBudget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           __nanosleep(32);
         }
-        if (!ok && kk >= ctl->n_needed) break;
+        if (!ok || ctl->end_kk >= 0) break;
         const int st = kk % kKStages;
         if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag)) {
           if (!*abort_flag) report_timeout(ctl, status);
@@ -223,7 +227,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         mbar_expect_tx(bar, kTileBytes);
         tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
         tma_load_2d(dst + kHalfBytes, &k_map, 64, kv_row0 + j * kBlock, bar);
+        last_issued = kk;
       }
+      // tiles fetched ahead may never be multiplied: their copies must have landed before the CTA retires
+      for (int kk = max(0, last_issued - (kKStages - 1)); kk <= last_issued; ++kk)
+        if (!mbar_wait(smem_u32(&ctl->k_full[kk % kKStages]), (kk / kKStages) & 1, abort_flag) && !*abort_flag) report_timeout(ctl, status);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ QK issuer
@@ -232,16 +240,18 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
       const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
+      int last_issued = -1;
       for (int kk = 0; kk < cnt && alive; ++kk) {
-        if (kk >= ctl->n_needed) {               // not yet certain that this block will be scored
+        if (kk >= ctl->n_needed + kSpec) {       // at most kSpec products beyond the blocks that are certain to be scored
           const long long t0 = clock64();
           bool ended = false;
-          while (kk >= ctl->n_needed) {
-            if (ctl->end_kk >= 0) { ended = kk >= ctl->n_needed; break; }
+          while (kk >= ctl->n_needed + kSpec) {
+            if (ctl->end_kk >= 0) { ended = true; break; }
             if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
           if (ended || !alive) break;
         }
+        if (ctl->end_kk >= 0 && kk > ctl->end_kk) break;
         const int st = kk % kKStages, sb = kk & 1;
         alive = mbar_wait(smem_u32(&ctl->k_full[st]), (kk / kKStages) & 1, abort_flag) &&
                 mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
@@ -251,7 +261,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
             tmem_s[sb], tmem_q, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk, false);
         mma_commit(smem_u32(&ctl->k_empty[st]));
+        last_issued = kk;
       }
+      // a product issued ahead of the walk's end may still be running: it must finish before TMEM is released
+      if (alive && last_issued >= 0 &&
+          !mbar_wait(smem_u32(&ctl->k_empty[last_issued % kKStages]), (last_issued / kKStages) & 1, abort_flag) && !*abort_flag)
+        report_timeout(ctl, status);
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------------ PV issuer
@@ -408,6 +423,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
       }
       const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
+      // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
+      //      walk gets here at all (n_needed only grows: an old value merely costs this wait)
+      if (kk >= ctl->n_needed) {
+        alive = mbar_wait(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        if (ctl->dec[(kk - 1) % kDecRing] & kDecEnd) break;
+      }
       // ---- running maximum before this position comes from the other group
       float m_in = -INFINITY;
       if (kk > 0) {
