@@ -227,8 +227,8 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   p.cap_fx = budget_to_fx(tightened_budget);
   p.theta = p.use_threshold ? (float)log((double)o.skip_scale / (double)shape->n) : 0.f;
   p.scale = o.softmax_scale > 0.f ? o.softmax_scale : (float)(1.0 / sqrt((double)shape->d));
-  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, static_cast<cudaStream_t>(stream))
-                                : launch_osk_tc(p, static_cast<cudaStream_t>(stream));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : launch_osk_tc(p, st);
   if (e != cudaSuccess) return cuda_fail(e, "osk launch");
   return COSA_OK;
 }

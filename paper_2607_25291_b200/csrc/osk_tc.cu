@@ -65,6 +65,7 @@ struct __align__(8) Control {
   volatile int n_needed;          // list positions [0, n_needed) are certain to be scored
   volatile int n_dec;             // decisions published so far
   volatile int end_kk;            // last scored position, -1 until known
+  volatile int k_loaded;          // K tiles the loader requested; -1 until it has stopped requesting
   volatile int final_computed;
   volatile int abort_flag;
   int poisoned;
@@ -160,6 +161,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
     ctl->end_kk = -1;
+    ctl->k_loaded = -1;
     ctl->final_computed = 0;
     ctl->abort_flag = 0;
     mbar_fence_init();
@@ -229,6 +231,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         tma_load_2d(dst + kHalfBytes, &k_map, 64, kv_row0 + j * kBlock, bar);
         last_issued = kk;
       }
+      ctl->k_loaded = last_issued + 1;       // the QK issuer must not wait for a tile beyond these
       // tiles fetched ahead may never be multiplied: their copies must have landed before the CTA retires
       for (int kk = max(0, last_issued - (kKStages - 1)); kk <= last_issued; ++kk)
         if (!mbar_wait(smem_u32(&ctl->k_full[kk % kKStages]), (kk / kKStages) & 1, abort_flag) && !*abort_flag) report_timeout(ctl, status);
@@ -253,8 +256,20 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         }
         if (ctl->end_kk >= 0 && kk > ctl->end_kk) break;
         const int st = kk % kKStages, sb = kk & 1;
-        alive = mbar_wait(smem_u32(&ctl->k_full[st]), (kk / kKStages) & 1, abort_flag) &&
-                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
+        {   // the tile, unless the loader stopped short of it (a position beyond the walk's end)
+          const uint32_t bar = smem_u32(&ctl->k_full[st]), par = (kk / kKStages) & 1;
+          bool none = false;
+          if (!mbar_try_wait(bar, par)) {
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar, par)) {
+              const int kl = ctl->k_loaded;
+              if (kl >= 0 && kk >= kl) { none = true; break; }
+              if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+            }
+          }
+          if (none || !alive) break;
+        }
+        alive = mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
         // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
