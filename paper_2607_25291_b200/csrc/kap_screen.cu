@@ -29,17 +29,20 @@ using namespace ptx;
 constexpr int kStages = 4;
 constexpr int kTileBytes = 128 * kHeadDim * 2;
 constexpr int kHalfBytes = kTileBytes / 2;
-constexpr int kThreads = 320;        // producer warp, MMA warp, 2 x 4 epilogue warps
-constexpr int kTmemCols = 256;
+constexpr int kParts = 4;             // column parts of a tile, one epilogue warp per part and sub-partition
+constexpr int kPartCols = 128 / kParts;
+constexpr int kThreads = 64 + 128 * kParts;   // producer warp, MMA warp, kParts x 4 epilogue warps
+constexpr int kAccs = 4;              // logit tiles in tensor memory (products run this far ahead of the epilogue)
+constexpr int kTmemCols = 128 * kAccs;
 
 struct __align__(8) ScreenCtl {
   unsigned long long a_full, k_full[kStages];
   unsigned long long k_empty[kStages];  // the tile's MMAs finished: stage free and logits ready
-  unsigned long long s_empty[2], x_bar;
+  unsigned long long s_empty[kAccs], x_bar;
   uint32_t tmem_base;
   volatile int abort_flag;
-  float xt[2][3][128];                  // pass-1 exchange between the two column halves: top-3 block maxima
-  int xj[2][2][128];                    // ... and the blocks holding the two largest
+  float xt[kParts][3][128];             // pass-1 exchange between the column parts: top-3 block maxima
+  int xj[kParts][2][128];               // ... and the blocks holding the two largest
 };
 constexpr size_t kScreenSmem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(ScreenCtl);
 
@@ -83,8 +86,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     if (blockIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
     mbar_init(smem_u32(&ctl->a_full), 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
-    for (int s = 0; s < 2; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), 256);
-    mbar_init(smem_u32(&ctl->x_bar), 256);
+    for (int s = 0; s < kAccs; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), 128 * kParts);
+    mbar_init(smem_u32(&ctl->x_bar), 128 * kParts);
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -126,9 +129,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       bool alive = mbar_wait(smem_u32(&ctl->a_full), 0, abort_flag);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
       for (int t = 0; t < 2 * n_tiles && alive; ++t) {
-        const int st = t % kStages, sb = t & 1;
+        const int st = t % kStages, sb = t % kAccs;
         alive = mbar_wait(smem_u32(&ctl->k_full[st]), (t / kStages) & 1, abort_flag) &&
-                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t >> 1) & 1) ^ 1, abort_flag);
+                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t / kAccs) & 1) ^ 1, abort_flag);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         tc_fence_after();
         const uint32_t kt = k_sm + st * kTileBytes;
@@ -138,10 +141,10 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       }
     }
   } else {
-    // ---------------------------------------------------------------- two threads per sampled query row
-    // (one per 64-column half of every tile: two epilogue warps per SM sub-partition overlap their latencies)
+    // ---------------------------------------------------------------- kParts threads per sampled query row
+    // (one per column part of every tile: kParts epilogue warps per SM sub-partition overlap their latencies)
     const int sub = warp & 3;
-    const int half = (warp - 2) >> 2;
+    const int half = (warp - 2) >> 2;        // column part
     const int row = sub * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
     const int grp = row / R, r = row % R;
@@ -158,7 +161,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     float* srow = p.scores + ((size_t)(b * p.hq + h) * p.nqb + (row_ok ? i : 0)) * p.nqb;
     bool alive = true;
     for (int t = 0; t < 2 * n_tiles && alive; ++t) {
-      const int sb = t & 1, jt = t % n_tiles, st = t % kStages;
+      const int sb = t % kAccs, jt = t % n_tiles, st = t % kStages;
       const bool pass2 = t >= n_tiles;
       if (t == n_tiles) {
         // end of pass 1: merge the two halves' top-3 block maxima of every row
@@ -168,12 +171,16 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         alive = mbar_wait(smem_u32(&ctl->x_bar), 0, abort_flag);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
 #pragma unroll
-        for (int q = 0; q < 3; ++q) {
-          const float m = ctl->xt[half ^ 1][q][row];
-          const int jb = q < 2 ? ctl->xj[half ^ 1][q][row] : 0;
-          if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
-          else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
-          else if (m > top3) top3 = m;
+        for (int other = 1; other < kParts; ++other) {
+          const int op = (half + other) % kParts;
+#pragma unroll
+          for (int q = 0; q < 3; ++q) {
+            const float m = ctl->xt[op][q][row];
+            const int jb = q < 2 ? ctl->xj[op][q][row] : 0;
+            if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
+            else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
+            else if (m > top3) top3 = m;
+          }
         }
         // the row's best block, and whether the runner-up is too close to call
         const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
@@ -193,15 +200,15 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       alive = mbar_wait(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag);   // this tile's MMAs finished
       if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
       tc_fence_after();
-      const int col0 = jt * 128 + half * 64;
-      uint32_t v[2][32];
-      tmem_ld32(tmem + sb * 128 + lane_addr + half * 64, v[0]);
-      tmem_ld32(tmem + sb * 128 + lane_addr + half * 64 + 32, v[1]);
+      const int col0 = jt * 128 + half * kPartCols;
+      uint32_t v[kPartCols / 32][32];
+#pragma unroll
+      for (int c2 = 0; c2 < kPartCols / 32; ++c2) tmem_ld32(tmem + sb * 128 + lane_addr + half * kPartCols + c2 * 32, v[c2]);
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->s_empty[sb]));
 #pragma unroll
-      for (int c2 = 0; c2 < 2; ++c2) {
+      for (int c2 = 0; c2 < kPartCols / 32; ++c2) {
         const int cbase = col0 + c2 * 32;
         float mb[BPC];
 #pragma unroll
