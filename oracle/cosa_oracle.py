@@ -258,6 +258,21 @@ def kap_select(q, k, s=8, budget=0.25, causal=True, block=128, heads=None, query
 
 
 # ----------------------------------------------------------------------------
+# Paged K/V (Sec. C.1: a logical block of b = 128 tokens is resolved through one or more
+# physical pages of b_p tokens)
+# ----------------------------------------------------------------------------
+def paged_view(pool, table, n):
+    """The logical [Hkv, N, d] tensor behind a page pool [P, Hkv, b_p, d] and a page table
+    [N / b_p]: token t of KV head g is pool[table[t div b_p], g, t mod b_p].  Everything the
+    method computes is defined on this view."""
+    page_size = pool.shape[2]
+    out = np.empty((pool.shape[1], n, pool.shape[3]), pool.dtype)
+    for t in range(n // page_size):
+        out[:, t * page_size:(t + 1) * page_size] = pool[int(table[t])]
+    return out
+
+
+# ----------------------------------------------------------------------------
 # List utilities for the remapping analysis (Sec. 5.3 "Effect of remapping") and the
 # logical-mask comparison (Sec. D "Kernel Microbenchmark")
 # ----------------------------------------------------------------------------

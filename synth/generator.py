@@ -132,3 +132,19 @@ def make_qkv(seed: int, hq: int, hkv: int, n: int, d: int = 128, block: int = 12
         planted["needle_key_blocks"].append(jn)
         planted["needle_targets"].append(tn)
     return q, k, v, planted
+
+
+def scatter_to_pages(x_bits: np.ndarray, page_size: int, seed: int, spare_pages: int = 3):
+    """Lay a dense [Hkv, N, d] tensor out as a paged pool (layout only, no arithmetic).
+
+    Returns (pool [P, Hkv, page_size, d] uint16, table [N / page_size] int32): logical page t of every
+    KV head lives in physical page table[t]; the pages are a seeded random permutation and the
+    pool holds a few unused pages filled with a recognisable bit pattern."""
+    hkv, n, d = x_bits.shape
+    assert n % page_size == 0
+    n_pages = n // page_size
+    rng = np.random.Generator(np.random.Philox(key=[seed, 77]))
+    phys = rng.permutation(n_pages + spare_pages)[:n_pages].astype(np.int32)
+    pool = np.full((n_pages + spare_pages, hkv, page_size, d), 0x7FC0, np.uint16)   # bf16 NaN in unused pages
+    pool[phys] = x_bits.reshape(hkv, n_pages, page_size, d).transpose(1, 0, 2, 3)
+    return pool, phys

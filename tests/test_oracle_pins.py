@@ -419,6 +419,22 @@ def test_kap_select_with_topp(small):
     assert (ccap == np.minimum(count, cb)).all()
 
 
+# ---------------------------------------------------------------- paged K/V
+def test_paged_view_hand_example_and_round_trip():
+    from synth.generator import scatter_to_pages
+    # two KV heads, four tokens, page size 2: logical page 0 -> physical 2, logical page 1 -> physical 0
+    pool = np.arange(3 * 2 * 2 * 1).reshape(3, 2, 2, 1)
+    view = O.paged_view(pool, np.array([2, 0]), 4)
+    assert view[:, :, 0].tolist() == [[8, 9, 0, 1], [10, 11, 2, 3]]
+    rng = np.random.default_rng(1)
+    x = rng.integers(0, 2 ** 16, size=(3, 1024, 8), dtype=np.uint16)
+    for page_size in (16, 64, 128, 256):
+        pool, table = scatter_to_pages(x, page_size, seed=5)
+        assert len(set(table.tolist())) == 1024 // page_size and pool.shape[0] == 1024 // page_size + 3
+        assert np.array_equal(O.paged_view(pool, table, 1024), x)
+        assert not np.array_equal(table, np.arange(1024 // page_size))          # really permuted
+
+
 # ---------------------------------------------------------------- list utilities (remapping analysis, logical mask)
 def test_list_utilities_against_hand_example_and_bruteforce():
     order = np.array([[[0, -1, -1, -1], [1, 0, -1, -1], [2, 0, 1, -1]]], np.int32)      # causal lists, nQB = 3
