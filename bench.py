@@ -42,6 +42,8 @@ def parse():
     ap.add_argument("--no-comparators", action="store_true", help="skip the dense-path and SDPA timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--page-size", type=int, default=0,
+                    help="K and V as page pools of this many tokens per page behind a shuffled page table (Sec. C.1); not the headline config")
     ap.add_argument("--top-p", type=float, default=0.0,
                     help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
     return ap.parse_args()
@@ -222,10 +224,22 @@ def main():
     opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=scored,
                                top_p=args.top_p)
     stream = torch.cuda.current_stream()
+    k_in, v_in = k, v
+    if args.page_size > 0:
+        # the same K and V as page pools behind a shuffled page table (layout only: a device-side copy)
+        from synth.generator import scatter_to_pages
+        kpool, table = scatter_to_pages(kb, args.page_size, seed=w.seed + 31)
+        vpool, _ = scatter_to_pages(vb, args.page_size, seed=w.seed + 31)
+        k_in = torch.from_numpy(kpool.view(np.int16)).view(torch.bfloat16).to(dev)
+        v_in = torch.from_numpy(vpool.view(np.int16)).view(torch.bfloat16).to(dev)
+        page_table = torch.from_numpy(table).to(dev)[None].contiguous()
+        opt.kv_page_table = page_table.data_ptr()
+        opt.kv_page_size = args.page_size
+        opt.kv_num_pages = kpool.shape[0]
 
     def step():
-        cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt, stream=stream)
-        cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_osk_attention(q, k_in, v_in, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
 
     def sync_all():
         if world > 1:
@@ -249,9 +263,9 @@ def main():
     t_wall = time.perf_counter()
     for s in range(args.steps):
         ev[s][0].record(stream)
-        cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream)
         ev[s][1].record(stream)
-        cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
+        cosa.cosa_osk_attention(q, k_in, v_in, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
         ev[s][2].record(stream)
     sync_all()
     t_wall = time.perf_counter() - t_wall
@@ -356,7 +370,7 @@ def main():
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
-                           "kap_budget": kap_budget, "top_p": args.top_p or None, "osk_budget": w.osk_budget, "stride": w.stride,
+                           "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "osk_budget": w.osk_budget, "stride": w.stride,
                            "skip_scale": w.skip_scale, "parallelism": f"layer-per-rank x{world}",
                            "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
                            "blocks_scored": n_scored, "blocks_computed": n_computed,

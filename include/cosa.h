@@ -15,7 +15,8 @@
  *   - All tensors are dense, row-major, innermost dimension contiguous, base pointers
  *     16-byte aligned.  Layouts:
  *         q, out              [B, Hq,  N, d]   bf16
- *         k, v                [B, Hkv, N, d]   bf16      (query head h reads KV head h / (Hq/Hkv))
+ *         k, v                [B, Hkv, N, d]   bf16      (query head h reads KV head h / (Hq/Hkv));
+ *                                                       or page pools, see cosa_options.kv_page_table
  *         order               [B, Hq, nQB, order_stride] int32   0-based key-block ids, then -1
  *         count, visited,
  *         scored              [B, Hq, nQB]     int32
@@ -93,6 +94,14 @@ typedef struct {
                               execution style OSK's index-driven jumping is compared with in Sec. D).
                               `order` and `count` may then be NULL; list positions in the outputs
                               are ranks among the kept blocks                                       */
+  const int32_t* kv_page_table; /* Non-NULL: k and v are page pools [kv_num_pages, Hkv, kv_page_size, d] and
+                              this device table [B, N / kv_page_size] names the physical page of every
+                              logical page (Sec. C.1: a logical block of 128 tokens is resolved through
+                              one or more physical pages when the page size differs).  NULL: k and v are
+                              the dense [B, Hkv, N, d] tensors (page = block, identity table)        */
+  int32_t kv_page_size;    /* tokens per physical page: a power of two in [8, N] that divides N and, for
+                              KAP, is a multiple of the stride                                       */
+  int32_t kv_num_pages;    /* pages in the pools                                                     */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);

@@ -43,7 +43,8 @@ class CosaOptions(Structure):
     _fields_ = [("stride", c_int32), ("skip_scale", c_float), ("softmax_scale", c_float),
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
-                ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p)]
+                ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p), ("kv_page_table", c_void_p),
+                ("kv_page_size", c_int32), ("kv_num_pages", c_int32)]
 
 
 class CosaError(RuntimeError):

@@ -67,6 +67,23 @@ int check_shape(const cosa_shape* s) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Paging arguments of a call: COSA_OK and *pg filled (table == nullptr when the tensors are dense).
+int resolve_paging(const cosa_shape* s, const cosa_options& o, int stride, KvPaging* pg) {
+  *pg = KvPaging{};
+  if (!o.kv_page_table) return COSA_OK;
+  const int ps = o.kv_page_size;
+  if (ps < 8 || (ps & (ps - 1)) != 0 || ps > s->n || s->n % ps != 0 || o.kv_num_pages < s->n / ps) return COSA_ERR_INVALID_ARG;
+  if (stride > 0 && ps % stride != 0) return COSA_ERR_UNSUPPORTED;
+  if ((long long)o.kv_num_pages * s->hkv * ps > 0x7fffffffLL) return COSA_ERR_UNSUPPORTED;   // tensor-map row coordinates
+  pg->table = o.kv_page_table;
+  pg->page_size = ps;
+  pg->page_shift = 0;
+  while ((1 << pg->page_shift) < ps) ++pg->page_shift;
+  pg->pages_per_seq = s->n / ps;
+  pg->num_pages = o.kv_num_pages;
+  return COSA_OK;
+}
+
 cosa_options resolve_options(const cosa_options* opt) {
   cosa_options o;
   cosa_default_options(&o);
@@ -84,8 +101,10 @@ struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, total; };
 static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
   KapScratch L{};
   const int stride = o.stride > 0 ? o.stride : 8;
+  KvPaging pg{};
+  if (resolve_paging(s, o, stride, &pg) != COSA_OK) return L;
   const size_t nqb = s->n / kBlock, heads = (size_t)s->batch * s->hq;
-  if (o.impl == 1 || stride < 1 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv)) return L;  // exact kernel: none
+  if (o.impl == 1 || stride < 1 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv, stride, pg)) return L;  // exact kernel: none
   size_t off = 0;
   L.scores = off; off += align_up(heads * nqb * nqb * 4, 256);
   L.jstar = off; off += align_up(heads * (s->n / stride) * 8, 256);
@@ -152,6 +171,8 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   p.budget_fx = budget_to_fx(budget);
   p.scale = o.softmax_scale > 0.f ? (double)o.softmax_scale : 1.0 / sqrt((double)shape->d);
   p.top_p = (double)o.top_p;
+  rc = resolve_paging(shape, o, s, &p.pg);
+  if (rc != COSA_OK) return rc;
   // the list of the longest row must fit the pitch
   if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
   if (kap_exact_smem_bytes(p.rows, nqb) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
@@ -184,6 +205,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.causal = p.causal; sp.stride = s;
   sp.scale = (float)p.scale;
   sp.tau_row = 1e-4f;
+  sp.pg = p.pg;
   cudaError_t e = launch_kap_screen(sp, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");
   e = launch_kap_sort(p, sp, 1.220703125e-4f, st);
@@ -215,6 +237,8 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   p.v = static_cast<const __nv_bfloat16*>(v);
   p.order = o.logical_mask ? nullptr : order; p.count = o.logical_mask ? nullptr : count;
   p.mask = o.logical_mask;
+  rc = resolve_paging(shape, o, 0, &p.pg);
+  if (rc != COSA_OK) return rc;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = out_lse; p.visited = out_visited;
   p.scored = o.out_scored; p.decisions = o.out_decisions;
@@ -330,6 +354,7 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
   o.workspace = ws + L.scratch;
   o.workspace_bytes = L.total - L.scratch;
   o.kap_scores = nullptr; o.kap_flags = nullptr; o.out_scored = nullptr; o.out_decisions = nullptr;
+  o.kv_page_table = nullptr;   // the host buffers are dense tensors
   rc = cosa_kap_select_ex(ws + L.q, ws + L.k, shape, budget, reinterpret_cast<int32_t*>(ws + L.order),
                           reinterpret_cast<int32_t*>(ws + L.count), stream, &o);
   if (rc != COSA_OK) return rc;

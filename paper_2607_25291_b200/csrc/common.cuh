@@ -12,6 +12,23 @@ namespace cosa {
 constexpr int kBlock = 128;  // logical query/key block b (Sec. C.1: b = 128)
 constexpr int kHeadDim = 128;
 
+// Paged K/V (Sec. C.1): k and v are page pools [P, Hkv, b_p, d]; token t of KV head g of batch item b lives in row
+// t mod b_p of pool[table[b, t div b_p], g].  table == nullptr: k and v are the dense [B, Hkv, N, d] tensors.
+struct KvPaging {
+  const int32_t* table;   // [B, N / b_p]
+  int page_size;          // b_p, a power of two
+  int page_shift;         // log2 b_p
+  int pages_per_seq;      // N / b_p
+  int num_pages;          // P
+};
+
+// Row of the [rows, d] view of k / v that holds `token` of KV head g of batch item b.
+__host__ __device__ inline long long kv_row(const KvPaging& pg, int b, int hkv, int g, int n, int token) {
+  if (!pg.table) return ((long long)b * hkv + g) * n + token;
+  const int page = pg.table[(long long)b * pg.pages_per_seq + (token >> pg.page_shift)];
+  return ((long long)page * hkv + g) * pg.page_size + (token & (pg.page_size - 1));
+}
+
 // Resolved call parameters handed to the kernels.
 struct KapParams {
   const __nv_bfloat16* q;
@@ -28,6 +45,7 @@ struct KapParams {
   long long budget_fx;   // floor(budget_f32 * 2^20)
   double scale;          // softmax scale applied to the sampled logits
   double top_p;          // > 0: Top-p retention, capped by the budget count; 0: budget count alone
+  KvPaging pg;
 };
 
 // The float32 screen of the KAP fast path (tensor cores) and what it leaves for the sort stage.
@@ -44,6 +62,7 @@ struct KapScreenParams {
   int stride;
   float scale;
   float tau_row;         // two block maxima of a row closer than this (scaled logits) are "too close to call"
+  KvPaging pg;
 };
 
 struct OskParams {
@@ -66,6 +85,7 @@ struct OskParams {
   long long cap_fx;      // floor(tightened_budget_f32 * 2^20)
   float theta;           // ln(Delta / N)
   float scale;           // softmax scale
+  KvPaging pg;
 };
 
 // Where the kk-th visited key block of one (head, query block) comes from.  List mode: the order list, read
@@ -120,7 +140,7 @@ int32_t* device_status_word();
 
 // redo_list == nullptr: every (head, query block); else only the listed ones (count in [0])
 cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st);
-bool kap_screen_supported(int rows, int group);
+bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
 // sorts the screened scores, recomputes near-ties in double precision, writes the lists
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st);

@@ -54,7 +54,6 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
   unsigned* ids = reinterpret_cast<unsigned*>(keys + sort_cap);
 
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
-  const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
 
   // sampled query rows of block i: tokens (i*R + r) * s
   for (int e = tid; e < R * kHeadDim; e += kThreads) {
@@ -68,8 +67,8 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
     __syncthreads();
     for (int e = tid; e < nb * R * kHeadDim; e += kThreads) {
       int c = e / kHeadDim, d = e % kHeadDim;  // c: sampled key within this group of blocks
-      size_t tok = (size_t)(j0 * R + c) * p.stride;
-      Ks[c * kPad + d] = (double)__bfloat162float(kh[tok * kHeadDim + d]);
+      const int tok = (j0 * R + c) * p.stride;
+      Ks[c * kPad + d] = (double)__bfloat162float(p.k[(size_t)kv_row(p.pg, b, p.hkv, g, p.n, tok) * kHeadDim + d]);
     }
     __syncthreads();
     for (int e = tid; e < nb * R * R; e += kThreads) {

@@ -110,17 +110,46 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         tma_load_2d(a_sm + grp * R * 128, &q_map, 0, row, smem_u32(&ctl->a_full));
         tma_load_2d(a_sm + kHalfBytes + grp * R * 128, &q_map, 64, row, smem_u32(&ctl->a_full));
       }
-      const int krow0 = (b * p.hkv + g) * ns;
+      if (!p.pg.table) {
+        const int krow0 = (b * p.hkv + g) * ns;
+        for (int t = 0; t < 2 * n_tiles; ++t) {
+          const int st = t % kStages, jt = t % n_tiles;
+          if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag)) {
+            if (!*abort_flag) screen_timeout(ctl, status);
+            break;
+          }
+          const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
+          mbar_expect_tx(bar, kTileBytes);
+          tma_load_2d(dst, &k_map, 0, krow0 + jt * 128, bar);
+          tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + jt * 128, bar);
+        }
+      }
+    }
+    if (p.pg.table) {
+      // paged keys: the 128 sampled keys of a tile come from 128 / spp pages (spp sampled rows each) or from one page;
+      // one lane per page looks its page up and issues its two boxes.  Sampled keys past the sequence are masked
+      // later: any valid page will do for them.
+      const int spp = min(128, p.pg.page_size / p.stride);
+      const int parts = 128 / spp;
       for (int t = 0; t < 2 * n_tiles; ++t) {
         const int st = t % kStages, jt = t % n_tiles;
-        if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag)) {
-          if (!*abort_flag) screen_timeout(ctl, status);
-          break;
-        }
         const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
-        mbar_expect_tx(bar, kTileBytes);
-        tma_load_2d(dst, &k_map, 0, krow0 + jt * 128, bar);
-        tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + jt * 128, bar);
+        int ok = 1;
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag) ? 1 : 0;
+          if (!ok && !*abort_flag) screen_timeout(ctl, status);
+          if (ok) mbar_expect_tx(bar, kTileBytes);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane < parts) {
+          int tok = (jt * 128 + lane * spp) * p.stride;
+          if (tok >= p.n) tok = 0;
+          const int srow = (int)(kv_row(p.pg, b, p.hkv, g, p.n, tok) / p.stride);
+          tma_load_2d(dst + lane * spp * 128, &k_map, 0, srow, bar);
+          tma_load_2d(dst + kHalfBytes + lane * spp * 128, &k_map, 64, srow, bar);
+        }
+        __syncwarp();
       }
     }
   } else if (warp == 1) {
@@ -290,16 +319,20 @@ bool make_strided_map(CUtensorMap* map, const void* basep, uint64_t sampled_rows
 
 }  // namespace
 
-bool kap_screen_supported(int rows, int group) {
-  return (rows == 8 || rows == 16 || rows == 32) && group * rows <= 128 && 128 % (group * rows) == 0;
+bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg) {
+  if (!((rows == 8 || rows == 16 || rows == 32) && group * rows <= 128 && 128 % (group * rows) == 0)) return false;
+  // paged keys: a page must hold at least 8 sampled rows (boxes land on 1024-byte boundaries of the swizzled tile)
+  return !pg.table || pg.page_size / stride >= 8;
 }
 
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st) {
   const int R = 128 / p.stride, G = p.hq / p.hkv;
   const uint64_t ns = (uint64_t)p.n / p.stride;
   CUtensorMap qm, km;
+  const uint64_t k_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * (p.pg.page_size / p.stride) : (uint64_t)p.batch * p.hkv * ns;
+  const int k_box = p.pg.table ? ((p.pg.page_size / p.stride) < 128 ? p.pg.page_size / p.stride : 128) : 128;
   if (!make_strided_map(&qm, p.q, (uint64_t)p.batch * p.hq * ns, p.stride, R) ||
-      !make_strided_map(&km, p.k, (uint64_t)p.batch * p.hkv * ns, p.stride, 128))
+      !make_strided_map(&km, p.k, k_rows, p.stride, k_box))
     return cudaErrorInvalidValue;
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;

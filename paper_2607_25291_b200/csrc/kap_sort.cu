@@ -33,14 +33,14 @@ struct Tied { int pos; unsigned id; double s; };
 
 // dest[r] = max over the visible sampled keys c of block jb[r] of (Q~[r] . K~[jb[r]*R + c]) * scale, in double
 // precision; rows with jb[r] < 0 are left alone.  All threads of the CTA call it.
-__device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, const __nv_bfloat16* kh, int i, int R,
+__device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, int b, int g, int i, int R,
                               const int* jb, double* dest, int tid) {
   for (int e = tid; e < R * R; e += kThreads) {
     const int r = e / R, c = e % R;
     double z = -INFINITY;
     const int kc = jb[r] * R + c;  // sampled key index
     if (jb[r] >= 0 && (!p.causal || kc <= i * R + r)) {
-      const uint4* src = reinterpret_cast<const uint4*>(kh + ((size_t)kc * p.stride) * kHeadDim);
+      const uint4* src = reinterpret_cast<const uint4*>(p.k + (size_t)kv_row(p.pg, b, p.hkv, g, p.n, kc * p.stride) * kHeadDim);
       const double* qr = Qs + r * kPad;
       double acc = 0.0;
 #pragma unroll 4
@@ -91,7 +91,6 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   }
   const unsigned amb = sp.ambmask[row];
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
-  const __nv_bfloat16* kh = p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim;
 
   const float* srow = sp.scores + row * p.nqb;
   int P2 = 2;
@@ -118,7 +117,7 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     }
     if (tid < R) jb[tid] = j1[tid];
     __syncthreads();
-    f64_block_max(p, Qs, Z, kh, i, R, jb, Mstar, tid);
+    f64_block_max(p, Qs, Z, b, g, i, R, jb, Mstar, tid);
     have_mstar = true;
   };
   __syncthreads();
@@ -128,7 +127,7 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     load_q_and_mstar();
     if (tid < R) { jb[tid] = ((amb >> tid) & 1u) ? j2[tid] : -1; Msecond[tid] = -INFINITY; }
     __syncthreads();
-    f64_block_max(p, Qs, Z, kh, i, R, jb, Msecond, tid);
+    f64_block_max(p, Qs, Z, b, g, i, R, jb, Msecond, tid);
     if (tid == 0) {
       for (int r = 0; r < R; ++r) {
         if (!((amb >> r) & 1u)) continue;
@@ -300,7 +299,7 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     for (int round = 0; round < nt; ++round) {
       if (tid < R) jb[tid] = (int)tied[round].id;
       __syncthreads();
-      f64_block_max(p, Qs, Z, kh, i, R, jb, Mrow, tid);
+      f64_block_max(p, Qs, Z, b, g, i, R, jb, Mrow, tid);
       if (tid == 0) {
         double s = 0.0;
         for (int r = 0; r < R; ++r) s += exp(Mrow[r] - Mstar[r]);

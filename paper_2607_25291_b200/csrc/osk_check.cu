@@ -49,16 +49,18 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
   float m = -INFINITY, l = 0.f;
   int computed = 0, scored = 0;
 
-  const uint4* kbase = reinterpret_cast<const uint4*>(p.k + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim);
-  const uint4* vbase = reinterpret_cast<const uint4*>(p.v + ((size_t)(b * p.hkv + g) * p.n) * kHeadDim);
+  const uint4* kbase = reinterpret_cast<const uint4*>(p.k);
+  const uint4* vbase = reinterpret_cast<const uint4*>(p.v);
 
   for (int kk = 0; kk < cnt; ++kk) {
     if (computed == cap) break;  // uniform over the CTA
     const int j = walk.at(kk);
     __syncthreads();
     for (int e = t; e < kBlock * kHeadDim / 8; e += kRows) {
-      reinterpret_cast<uint4*>(Ksm)[e] = kbase[(size_t)j * (kBlock * kHeadDim / 8) + e];
-      reinterpret_cast<uint4*>(Vsm)[e] = vbase[(size_t)j * (kBlock * kHeadDim / 8) + e];
+      // row e / 16 of the block, 16-byte chunk e % 16 of that row, through the page table if there is one
+      const size_t src = (size_t)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock + e / (kHeadDim / 8)) * (kHeadDim / 8) + e % (kHeadDim / 8);
+      reinterpret_cast<uint4*>(Ksm)[e] = kbase[src];
+      reinterpret_cast<uint4*>(Vsm)[e] = vbase[src];
     }
     __syncthreads();
     // S = Q_i K_j^T * scale, m_loc = rowmax S

@@ -88,6 +88,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&t);
 }
 
+// One 128-row K or V block into a tile buffer.  Dense tensors, or pages that hold whole blocks: one pair of boxes
+// (128 rows x 64 columns each).  Pages smaller than a block (Sec. C.1: a logical block resolved through several
+// physical pages): one pair of boxes of b_p rows per page, looked up in the page table.
+__device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensorMap* map, uint32_t dst, int b, int g, int j,
+                                              uint32_t bar) {
+  if (!p.pg.table || p.pg.page_size >= kBlock) {
+    const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock);
+    tma_load_2d(dst, map, 0, row, bar);
+    tma_load_2d(dst + kHalfBytes, map, 64, row, bar);
+  } else {
+    const int ps = p.pg.page_size;
+    for (int part = 0; part < kBlock / ps; ++part) {
+      const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock + part * ps);
+      tma_load_2d(dst + part * ps * 128, map, 0, row, bar);
+      tma_load_2d(dst + kHalfBytes + part * ps * 128, map, 64, row, bar);
+    }
+  }
+}
+
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
 // list-driven kernel carries none of the walk's state
 template <bool kMask>
@@ -125,7 +144,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const int cnt = kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
   const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N, d] view
-  const int kv_row0 = (b * p.hkv + g) * p.n;              // first row of this KV head
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -176,8 +194,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const int j = min(max(first_ids[kk], 0), p.nqb - 1);
         const uint32_t dst = k_sm + kk * kTileBytes, bar = smem_u32(&ctl->k_full[kk]);
         mbar_expect_tx(bar, kTileBytes);
-        tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
-        tma_load_2d(dst + kHalfBytes, &k_map, 64, kv_row0 + j * kBlock, bar);
+        load_kv_block(p, &k_map, dst, b, g, j, bar);
       }
     }
   }
@@ -227,8 +244,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
         const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
         mbar_expect_tx(bar, kTileBytes);
-        tma_load_2d(dst, &k_map, 0, kv_row0 + j * kBlock, bar);
-        tma_load_2d(dst + kHalfBytes, &k_map, 64, kv_row0 + j * kBlock, bar);
+        load_kv_block(p, &k_map, dst, b, g, j, bar);
         last_issued = kk;
       }
       ctl->k_loaded = last_issued + 1;       // the QK issuer must not wait for a tile beyond these
@@ -345,8 +361,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           } else {
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
             mbar_expect_tx(bar, kTileBytes);
-            tma_load_2d(dst, &v_map, 0, kv_row0 + j * kBlock, bar);
-            tma_load_2d(dst + kHalfBytes, &v_map, 64, kv_row0 + j * kBlock, bar);
+            load_kv_block(p, &v_map, dst, b, g, j, bar);
           }
           dec_word |= 1u << (kk & 31);
         }
@@ -589,12 +604,12 @@ EncodeTiledFn encode_fn() {
 }
 
 // [rows, 128] bf16 row-major viewed as boxes of 128 rows x 64 columns with the 128-byte swizzle
-bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows) {
+bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows, int box_rows = kBlock) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)kBlock};
+  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(basep), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -606,8 +621,11 @@ bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows) {
 
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
   CUtensorMap qm, km, vm, om;
-  if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, (uint64_t)p.batch * p.hkv * p.n) ||
-      !make_tile_map(&vm, p.v, (uint64_t)p.batch * p.hkv * p.n) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
+  // K and V: the dense tensors, or the page pools (boxes of one page when a page is smaller than a block)
+  const uint64_t kv_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * p.pg.page_size : (uint64_t)p.batch * p.hkv * p.n;
+  const int kv_box = (p.pg.table && p.pg.page_size < kBlock) ? p.pg.page_size : kBlock;
+  if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, kv_rows, kv_box) ||
+      !make_tile_map(&vm, p.v, kv_rows, kv_box) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
     return cudaErrorInvalidValue;
   auto kernel = p.mask ? osk_tc_kernel<true> : osk_tc_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

@@ -8,7 +8,7 @@ import torch
 import paper_2607_25291_b200 as cosa
 from oracle import cosa_oracle as O
 from synth.configs import SWEEP_STAGE1, SWEEP_STAGE2_MULT, WORKLOADS
-from synth.generator import bf16_bits_to_f64
+from synth.generator import bf16_bits_to_f64, scatter_to_pages
 from tests.helpers import to_dev
 from tests.test_gpu_parity import TOPP_MARGIN, _np, check_osk_against_oracle, check_topp_lists
 
@@ -127,6 +127,36 @@ def test_qwen3_32k_and_128k_topp_sampled():
         pairs = w.hq * w.n_blocks * (w.n_blocks + 1) // 2
         assert stats["listed"] < pairs
         print(name, "top-p 0.95", stats, "listed fraction", stats["listed"] / pairs)
+
+
+def test_qwen3_32k_paged_equals_dense():
+    """Page pools of 64- and 256-token pages (Sec. C.1) against the dense tensors they hold, whole workload."""
+    w = WORKLOADS["qwen3_32k"]
+    qb, kb, vb, _ = w.make()
+    q, k, v = (to_dev(x) for x in (qb, kb, vb))
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(w.kap_budget, nqb) + 7) // 8 * 8
+
+    def run(kk, vv, **paging):
+        order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+        count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+        out = torch.empty_like(q)
+        vis = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+        opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, **paging)
+        cosa.cosa_kap_select(q, kk, w.kap_budget, order, count, opt=opt)
+        cosa.cosa_osk_attention(q, kk, vv, order, count, w.osk_budget, out, None, vis, opt=opt)
+        assert cosa.cosa_device_status() == 0
+        return order, count, out, vis
+
+    dense = run(k, v)
+    for page_size in (64, 256):
+        kpool, table = scatter_to_pages(kb, page_size, seed=12)
+        vpool, _ = scatter_to_pages(vb, page_size, seed=12)
+        dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda().contiguous()
+        paged = run(dev(kpool), dev(vpool), kv_page_table=torch.from_numpy(table).cuda()[None].contiguous(),
+                    kv_page_size=page_size, kv_num_pages=kpool.shape[0])
+        for a, b in zip(dense, paged):
+            assert torch.equal(a, b)
 
 
 def test_llama31_64k_budget_sweep_sampled():

@@ -14,6 +14,7 @@ import torch
 import paper_2607_25291_b200 as cosa
 from oracle import cosa_oracle as O
 from synth.configs import WORKLOADS, tiny
+from synth.generator import scatter_to_pages
 from tests.helpers import alloc_lists, alloc_outputs, to_dev, widen
 
 pytestmark = pytest.mark.gpu
@@ -382,6 +383,73 @@ def test_ablation_tables_run_and_show_the_effect_of_order():
         assert sel[0]["skip_natural"] <= sel[1]["skip_natural"] <= sel[2]["skip_natural"]
     micro = ablation.micro_table([w], budgets=(0.5,), with_sdpa=False)
     assert len(micro) == 1 and micro[0]["jump_ms"] > 0 and micro[0]["logical_ms"] > 0 and micro[0]["dense_ms"] > 0
+
+
+# ---------------------------------------------------------------------------------- paged K/V
+def _pools(w, page_size):
+    """K and V of the workload as page pools that share one seeded page table."""
+    _, kb, vb, _ = w.make()
+    kpool, table = scatter_to_pages(kb, page_size, seed=9)
+    vpool, table_v = scatter_to_pages(vb, page_size, seed=9)
+    assert np.array_equal(table, table_v)
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda().contiguous()
+    return dev(kpool), dev(vpool), torch.from_numpy(table).cuda()[None].contiguous(), kpool.shape[0]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("page_size", [16, 64, 128, 256])
+def test_paged_kv_small(small, impl, page_size):
+    """Pools + page table give the lists and outputs of the dense tensors behind them (Sec. C.1)."""
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    nqb = q.shape[2] // 128
+    kpool, vpool, table, n_pages = _pools(small["w"], page_size)
+    for stride in (8, 16):
+        paging = dict(kv_page_table=table, kv_page_size=page_size, kv_num_pages=n_pages)
+        order, count = alloc_lists(q.shape[1], nqb)
+        cosa.cosa_kap_select(q, kpool, 0.6, order, count, opt=cosa.default_options(stride=stride, impl=impl, **paging))
+        assert cosa.cosa_device_status() == 0
+        ref_order, ref_count = O.kap_select(qf, kf, s=stride, budget=0.6, order_stride=nqb)
+        assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    for tb, skip_scale in ((1.0, 200.0), (0.4, 150.0)):
+        bufs = alloc_outputs(q, nqb)
+        opt = cosa.default_options(skip_scale=skip_scale, impl=impl, out_scored=bufs["scored"],
+                                   out_decisions=bufs["decisions"], **paging)
+        cosa.cosa_osk_attention(q, kpool, vpool, order, count, tb, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+        assert cosa.cosa_device_status() == 0
+        check_osk_against_oracle(qf, kf, vf, ref_order, ref_count, bufs, tb, skip_scale, range(q.shape[1]), range(nqb))
+        dense = run_osk(q, k, v, order, count, tb, skip_scale, impl)
+        assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
+        assert torch.equal(dense["lse"], bufs["lse"])
+
+
+def test_paged_kv_4k(cfg1):
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    for page_size in (64, 512):
+        kpool, vpool, table, n_pages = _pools(w, page_size)
+        paging = dict(kv_page_table=table, kv_page_size=page_size, kv_num_pages=n_pages)
+        order, count = alloc_lists(w.hq, w.n_blocks)
+        cosa.cosa_kap_select(q, kpool, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride, **paging))
+        d_order, d_count = run_kap(q, k, w.kap_budget, w.stride)
+        assert torch.equal(order, d_order) and torch.equal(count, d_count)
+        bufs = alloc_outputs(q, w.n_blocks)
+        opt = cosa.default_options(skip_scale=w.skip_scale, out_scored=bufs["scored"], out_decisions=bufs["decisions"], **paging)
+        cosa.cosa_osk_attention(q, kpool, vpool, order, count, w.osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+        assert cosa.cosa_device_status() == 0
+        dense = run_osk(q, k, v, order, count, w.osk_budget, w.skip_scale)
+        assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
+
+
+def test_paged_kv_rejects_bad_arguments(small):
+    q, _, _ = small["dev"]
+    kpool, vpool, table, n_pages = _pools(small["w"], 64)
+    order, count = alloc_lists(q.shape[1], q.shape[2] // 128)
+    for bad in (dict(kv_page_size=48), dict(kv_page_size=4), dict(kv_num_pages=3), dict(kv_page_size=4096)):
+        args = dict(kv_page_table=table, kv_page_size=64, kv_num_pages=n_pages)
+        args.update(bad)
+        with pytest.raises(cosa.CosaError):
+            cosa.cosa_kap_select(q, kpool, 0.5, order, count, opt=cosa.default_options(**args))
 
 
 def test_osk_is_deterministic(cfg1):
