@@ -225,6 +225,9 @@ int cosa_validate_order(const int32_t* order, const int32_t* count, const cosa_s
  * pointers (pinned memory gives asynchronous copies); `device_workspace` is a DEVICE buffer of
  * at least cosa_host_call_workspace_bytes() bytes.  Outputs are valid after the stream is
  * synchronised.  out_lse_host and out_visited_host may be NULL.
+ * The call works through the (batch item, KV head) slices one after the other; the copies to and from the
+ * device run on two internal streams (created once per device) so that they overlap the kernels of the other
+ * slices; `stream` is ordered after all of them.  opt->kv_page_table and opt->logical_mask are ignored.
  */
 size_t cosa_host_call_workspace_bytes(const cosa_shape* shape, const cosa_options* opt);
 int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host,

@@ -302,6 +302,22 @@ int cosa_lists_to_mask(const int32_t* order, const int32_t* count, const cosa_sh
 
 // ---- whole path on host buffers ----
 namespace {
+// Two non-blocking streams per device for the host call's transfers (created on first use, kept).
+bool copy_streams(cudaStream_t* up, cudaStream_t* down) {
+  static cudaStream_t streams[64][2];
+  static bool made[64];
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!made[dev]) {
+    if (cudaStreamCreateWithFlags(&streams[dev][0], cudaStreamNonBlocking) != cudaSuccess) return false;
+    if (cudaStreamCreateWithFlags(&streams[dev][1], cudaStreamNonBlocking) != cudaSuccess) return false;
+    made[dev] = true;
+  }
+  *up = streams[dev][0]; *down = streams[dev][1];
+  return true;
+}
 struct HostCallLayout {
   size_t q, k, v, out, lse, order, count, visited, scratch, total;
   size_t q_bytes, kv_bytes, lse_bytes, order_bytes, cnt_bytes;
@@ -347,24 +363,62 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
   char* ws = static_cast<char*>(device_workspace);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(ws + L.q, q_host, L.q_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D q");
-  if ((e = cudaMemcpyAsync(ws + L.k, k_host, L.kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D k");
-  if ((e = cudaMemcpyAsync(ws + L.v, v_host, L.kv_bytes, cudaMemcpyHostToDevice, st)) != cudaSuccess) return cuda_fail(e, "H2D v");
   o.order_stride = L.order_stride;
   o.workspace = ws + L.scratch;
   o.workspace_bytes = L.total - L.scratch;
   o.kap_scores = nullptr; o.kap_flags = nullptr; o.out_scored = nullptr; o.out_decisions = nullptr;
   o.kv_page_table = nullptr;   // the host buffers are dense tensors
-  rc = cosa_kap_select_ex(ws + L.q, ws + L.k, shape, budget, reinterpret_cast<int32_t*>(ws + L.order),
-                          reinterpret_cast<int32_t*>(ws + L.count), stream, &o);
-  if (rc != COSA_OK) return rc;
-  rc = cosa_osk_attention_ex(ws + L.q, ws + L.k, ws + L.v, shape, reinterpret_cast<int32_t*>(ws + L.order),
-                             reinterpret_cast<int32_t*>(ws + L.count), tightened_budget, ws + L.out,
-                             reinterpret_cast<float*>(ws + L.lse), reinterpret_cast<int32_t*>(ws + L.visited), stream, &o);
-  if (rc != COSA_OK) return rc;
-  if ((e = cudaMemcpyAsync(out_host, ws + L.out, L.q_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H out");
-  if (out_lse_host && (e = cudaMemcpyAsync(out_lse_host, ws + L.lse, L.lse_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H lse");
-  if (out_visited_host && (e = cudaMemcpyAsync(out_visited_host, ws + L.visited, L.cnt_bytes, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e, "D2H visited");
+  o.logical_mask = nullptr;
+
+  // One chunk per (batch item, KV head): its query heads, lists and outputs are contiguous slices of every tensor,
+  // so the chunks run as independent calls.  Copies to the device go on a second stream and copies back on a third,
+  // so that the transfers of the other chunks overlap a chunk's kernels; `stream` waits for the last copy back.
+  const int G = shape->hq / shape->hkv, chunks = shape->batch * shape->hkv;
+  const size_t nqb = shape->n / kBlock;
+  const size_t q_chunk = L.q_bytes / chunks, kv_chunk = L.kv_bytes / chunks, lse_chunk = L.lse_bytes / chunks;
+  const size_t order_chunk = L.order_bytes / chunks, cnt_chunk = L.cnt_bytes / chunks;
+  cudaStream_t up = nullptr, down = nullptr;
+  if (!copy_streams(&up, &down)) return cuda_fail(cudaGetLastError(), "copy streams");
+  cosa_shape sub = *shape;
+  sub.batch = 1; sub.hq = G; sub.hkv = 1;
+  cudaEvent_t ev = nullptr;
+  auto order_after = [&](cudaStream_t later, cudaStream_t earlier) -> bool {   // later waits for what earlier holds now
+    if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return false;
+    e = cudaEventRecord(ev, earlier);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(later, ev, 0);
+    cudaEventDestroy(ev);   // released once the recorded work has completed
+    return e == cudaSuccess;
+  };
+  if (!order_after(up, st)) return cuda_fail(e, "stream order");   // the workspace may still be in use on `stream`
+  if (!order_after(down, st)) return cuda_fail(e, "stream order");
+  (void)nqb;
+  for (int c = 0; c < chunks; ++c) {
+    const char* qh = static_cast<const char*>(q_host) + c * q_chunk;
+    const char* kh = static_cast<const char*>(k_host) + c * kv_chunk;
+    const char* vh = static_cast<const char*>(v_host) + c * kv_chunk;
+    char* qd = ws + L.q + c * q_chunk; char* kd = ws + L.k + c * kv_chunk; char* vd = ws + L.v + c * kv_chunk;
+    char* od = ws + L.out + c * q_chunk;
+    if ((e = cudaMemcpyAsync(kd, kh, kv_chunk, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e, "H2D k");
+    if ((e = cudaMemcpyAsync(qd, qh, q_chunk, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e, "H2D q");
+    if ((e = cudaMemcpyAsync(vd, vh, kv_chunk, cudaMemcpyHostToDevice, up)) != cudaSuccess) return cuda_fail(e, "H2D v");
+    if (!order_after(st, up)) return cuda_fail(e, "stream order");
+    int32_t* order_d = reinterpret_cast<int32_t*>(ws + L.order + c * order_chunk);
+    int32_t* count_d = reinterpret_cast<int32_t*>(ws + L.count + c * cnt_chunk);
+    int32_t* visited_d = reinterpret_cast<int32_t*>(ws + L.visited + c * cnt_chunk);
+    float* lse_d = reinterpret_cast<float*>(ws + L.lse + c * lse_chunk);
+    rc = cosa_kap_select_ex(qd, kd, &sub, budget, order_d, count_d, stream, &o);
+    if (rc != COSA_OK) return rc;
+    rc = cosa_osk_attention_ex(qd, kd, vd, &sub, order_d, count_d, tightened_budget, od, lse_d, visited_d, stream, &o);
+    if (rc != COSA_OK) return rc;
+    if (!order_after(down, st)) return cuda_fail(e, "stream order");
+    if ((e = cudaMemcpyAsync(static_cast<char*>(out_host) + c * q_chunk, od, q_chunk, cudaMemcpyDeviceToHost, down)) != cudaSuccess)
+      return cuda_fail(e, "D2H out");
+    if (out_lse_host && (e = cudaMemcpyAsync(reinterpret_cast<char*>(out_lse_host) + c * lse_chunk, lse_d, lse_chunk,
+                                             cudaMemcpyDeviceToHost, down)) != cudaSuccess) return cuda_fail(e, "D2H lse");
+    if (out_visited_host && (e = cudaMemcpyAsync(reinterpret_cast<char*>(out_visited_host) + c * cnt_chunk, visited_d, cnt_chunk,
+                                                 cudaMemcpyDeviceToHost, down)) != cudaSuccess) return cuda_fail(e, "D2H visited");
+  }
+  if (!order_after(st, down)) return cuda_fail(e, "stream order");   // outputs are valid once `stream` is synchronised
   return COSA_OK;
 }
 
