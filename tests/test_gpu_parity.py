@@ -452,6 +452,52 @@ def test_paged_kv_rejects_bad_arguments(small):
             cosa.cosa_kap_select(q, kpool, 0.5, order, count, opt=cosa.default_options(**args))
 
 
+# ---------------------------------------------------------------------------------- batch > 1
+@pytest.mark.parametrize("impl", IMPLS)
+def test_batch_of_two_equals_single_items(impl):
+    """Two different sequences in one call give exactly the results of two calls (dense and paged)."""
+    items = []
+    for seed in (31, 32):
+        w = tiny(seed=seed, hq=4, hkv=2, n=1024, needles=2)
+        qb, kb, vb, _ = w.make()
+        items.append((w, qb, kb, vb))
+    stack = lambda idx: torch.cat([to_dev(it[idx]) for it in items], dim=0).contiguous()
+    q2, k2, v2 = stack(1), stack(2), stack(3)
+    nqb = 8
+
+    def run(q, k, v, batch, **paging):
+        order = torch.full((batch, 4, nqb, nqb), -7, dtype=torch.int32, device="cuda")
+        count = torch.full((batch, 4, nqb), -7, dtype=torch.int32, device="cuda")
+        out = torch.empty_like(q)
+        lse = torch.empty(batch, 4, 1024, dtype=torch.float32, device="cuda")
+        vis = torch.empty(batch, 4, nqb, dtype=torch.int32, device="cuda")
+        opt = cosa.default_options(impl=impl, skip_scale=200.0, **paging)
+        cosa.cosa_kap_select(q, k, 0.6, order, count, opt=opt)
+        cosa.cosa_osk_attention(q, k, v, order, count, 0.4, out, lse, vis, opt=opt)
+        assert cosa.cosa_device_status() == 0
+        return order, count, out, lse, vis
+
+    both = run(q2, k2, v2, 2)
+    for b in range(2):
+        one = run(q2[b:b + 1].contiguous(), k2[b:b + 1].contiguous(), v2[b:b + 1].contiguous(), 1)
+        for x, y in zip(both, one):
+            assert torch.equal(x[b:b + 1], y)
+    # the same through page pools: both sequences share one pool, each with its own row of the page table
+    page_size = 64
+    pools, tables = [], []
+    for _, _, kb, vb in items:
+        kp, tab = scatter_to_pages(kb, page_size, seed=4)
+        vp, _ = scatter_to_pages(vb, page_size, seed=4)
+        tables.append(tab + sum(p_[0].shape[0] for p_ in pools))
+        pools.append((kp, vp))
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda().contiguous()
+    kpool = dev(np.concatenate([p_[0] for p_ in pools])); vpool = dev(np.concatenate([p_[1] for p_ in pools]))
+    table = torch.from_numpy(np.stack(tables).astype(np.int32)).cuda().contiguous()
+    paged = run(q2, kpool, vpool, 2, kv_page_table=table, kv_page_size=page_size, kv_num_pages=kpool.shape[0])
+    for x, y in zip(both, paged):
+        assert torch.equal(x, y)
+
+
 def test_osk_is_deterministic(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
