@@ -177,6 +177,59 @@ def kap_scores_literal(q, k, h, i, s=8, block=128, causal=True):
     return scores, flags
 
 
+def kap_scores_wide(q, k, h, big, s=8, block=128, tiles=2, causal=True):
+    """Scores and flags of a query block of tiles*block rows against key blocks of `block`
+    rows (Sec. C.1 names b = 128 for both; this is the wider-query variant): Eqs. (8)-(12)
+    with the sum of Eq. (11) and the "some row" of Eq. (12) running over all sampled rows of
+    the wide block.  Candidates when causal: the key blocks holding a key that some row of
+    the block may see, j < tiles * (big + 1).  Returns (scores [J], flags [J], M [tiles*R, J])."""
+    G = q.shape[0] // k.shape[0]
+    n, d = q.shape[1], q.shape[2]
+    R = block // s
+    rows = tiles * R
+    J = tiles * (big + 1) if causal else n // block
+    r = np.arange(big * rows, (big + 1) * rows)
+    c = np.arange(J * R)
+    z = (q[h, r * s] @ k[h // G, c * s].T) * (1.0 / math.sqrt(d))
+    if causal:
+        z = np.where(c[None, :] <= r[:, None], z, NEG_INF)
+    M = z.reshape(rows, J, R).max(axis=2)
+    Mstar = M.max(axis=1)
+    Pbar = np.exp(M - Mstar[:, None])             # 0 where a row sees nothing of block j
+    scores = np.zeros(J)
+    for rr in range(rows):
+        scores += Pbar[rr]
+    flags = (M == Mstar[:, None]).any(axis=0)
+    return scores, flags, M
+
+
+def kap_select_wide(q, k, s=8, budget=0.25, causal=True, block=128, tiles=2, order_stride=None, heads=None,
+                    wide_blocks=None):
+    """Stage-1 lists when one ranking is made per query block of tiles*block rows and shared by
+    its `tiles` row tiles of `block` rows (the block_q = 256 variant).  The wide block keeps the
+    first K = budget_count(budget, candidates) entries of its flag-grouped order; row tile t of
+    the block gets those entries in that order minus the key blocks that lie wholly after it
+    (when causal).  Returns per-tile (order [Hq, N/block, order_stride], count [Hq, N/block])."""
+    hq, n, _ = q.shape
+    nqb = n // block
+    nbig = nqb // tiles
+    if order_stride is None:
+        order_stride = nqb
+    order = np.full((hq, nqb, order_stride), -1, np.int32)
+    count = np.zeros((hq, nqb), np.int32)
+    for h in (range(hq) if heads is None else heads):
+        for big in (range(nbig) if wide_blocks is None else wide_blocks):
+            scores, flags, _ = kap_scores_wide(q, k, h, big, s, block, tiles, causal)
+            rho = flag_grouped_order(scores, flags)
+            kept = rho[:budget_count(budget, len(rho))]
+            for t in range(tiles):
+                i = big * tiles + t
+                ids = [j for j in kept if (not causal) or j <= i]
+                order[h, i, :len(ids)] = ids
+                count[h, i] = len(ids)
+    return order, count
+
+
 def flag_grouped_order(scores, flags):
     """rho_i of Eq. (13): HRM blocks first, each group by descending score.
     Equal scores inside a group are ordered by ascending block id (this build's

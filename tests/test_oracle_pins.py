@@ -419,6 +419,46 @@ def test_kap_select_with_topp(small):
     assert (ccap == np.minimum(count, cb)).all()
 
 
+# ---------------------------------------------------------------- wide query blocks (block_q = 256 variant)
+def test_wide_block_scores_are_the_sum_over_its_row_tiles(small):
+    """The sum over sampled rows of Eq. (11) splits over the two 128-row tiles, the flag of Eq. (12) is their OR;
+    a key block wholly after a tile gets nothing from it."""
+    q, k, _, _ = small
+    for h in range(q.shape[0]):
+        for big in range(q.shape[1] // 256):
+            scores, flags, M = O.kap_scores_wide(q, k, h, big, 8)
+            s0, f0, _ = O.kap_scores(q, k, h, 2 * big, 8)
+            s1, f1, _ = O.kap_scores(q, k, h, 2 * big + 1, 8)
+            assert len(scores) == 2 * big + 2
+            assert np.abs(scores - (np.append(s0, 0.0) + s1)).max() < 1e-12
+            assert np.array_equal(flags, np.append(f0, False) | f1)
+            assert np.isneginf(M[:16, 2 * big + 1]).all()                    # the first tile never sees the last block
+    # with a single tile the wide routine is the ordinary one
+    sw, fw, _ = O.kap_scores_wide(q, k, 1, 5, 8, tiles=1)
+    sn, fn, _ = O.kap_scores(q, k, 1, 5, 8)
+    assert np.array_equal(sw, sn) and np.array_equal(fw, fn)
+
+
+def test_wide_block_lists(small):
+    q, k, _, _ = small
+    nqb = q.shape[1] // 128
+    order, count = O.kap_select_wide(q, k, s=8, budget=0.6)
+    for h in range(q.shape[0]):
+        for big in range(nqb // 2):
+            scores, flags, _ = O.kap_scores_wide(q, k, h, big, 8)
+            # the ranking by brute force: HRM group first, then by score, ties by id
+            J = 2 * big + 2
+            rank = sorted(range(J), key=lambda j: (not flags[j], -scores[j], j))[:O.budget_count(0.6, J)]
+            hi = order[h, 2 * big + 1, :count[h, 2 * big + 1]].tolist()
+            lo = order[h, 2 * big, :count[h, 2 * big]].tolist()
+            assert hi == rank
+            assert lo == [j for j in rank if j != 2 * big + 1] and all(j <= 2 * big for j in lo)
+    # one tile per block: the ordinary lists
+    o1, c1 = O.kap_select_wide(q, k, s=8, budget=0.6, tiles=1)
+    o0, c0 = O.kap_select(q, k, s=8, budget=0.6, order_stride=nqb)
+    assert np.array_equal(o1, o0) and np.array_equal(c1, c0)
+
+
 # ---------------------------------------------------------------- paged K/V
 def test_paged_view_hand_example_and_round_trip():
     from synth.generator import scatter_to_pages
