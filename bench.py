@@ -44,6 +44,8 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--page-size", type=int, default=0,
                     help="K and V as page pools of this many tokens per page behind a shuffled page table (Sec. C.1); not the headline config")
+    ap.add_argument("--block-q", type=int, default=128, choices=[128, 256],
+                    help="256: one Stage-1 ranking per 256-row query block shared by its two row tiles; not the headline config")
     ap.add_argument("--top-p", type=float, default=0.0,
                     help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
     return ap.parse_args()
@@ -238,7 +240,7 @@ def main():
         opt.kv_num_pages = kpool.shape[0]
 
     def step():
-        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream, block_q=args.block_q)
         cosa.cosa_osk_attention(q, k_in, v_in, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
 
     def sync_all():
@@ -263,7 +265,7 @@ def main():
     t_wall = time.perf_counter()
     for s in range(args.steps):
         ev[s][0].record(stream)
-        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream)
+        cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream, block_q=args.block_q)
         ev[s][1].record(stream)
         cosa.cosa_osk_attention(q, k_in, v_in, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
         ev[s][2].record(stream)
@@ -370,7 +372,7 @@ def main():
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
-                           "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "osk_budget": w.osk_budget, "stride": w.stride,
+                           "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "kap_block_q": args.block_q, "osk_budget": w.osk_budget, "stride": w.stride,
                            "skip_scale": w.skip_scale, "parallelism": f"layer-per-rank x{world}",
                            "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
                            "blocks_scored": n_scored, "blocks_computed": n_computed,

@@ -58,7 +58,8 @@ typedef struct {
   int32_t hkv;        /* Hkv, divides Hq */
   int32_t n;          /* N, sequence length, multiple of 128 */
   int32_t d;          /* head dimension, must be 128 */
-  int32_t block_q;    /* must be 128 */
+  int32_t block_q;    /* 128; cosa_kap_select also takes 256: one ranking per 256-row query block,
+                         shared by its two 128-row tiles (see cosa_kap_select) */
   int32_t block_k;    /* must be 128 */
   int32_t causal;     /* 1: candidates of query block i are key blocks j <= i (Algorithm A step 5)
                          and the diagonal block is masked per token; 0: all key blocks */
@@ -130,6 +131,13 @@ int32_t cosa_budget_count(float budget, int32_t candidates);
  *   out_order   out  device int32 [B,Hq,nQB,order_stride]; positions >= count are set to -1;
  *                    order_stride must be >= the largest K_i
  *   out_count   out  device int32 [B,Hq,nQB]
+ * shape->block_q = 256 (a variant; N a multiple of 256): the scores and flags of a query block are taken over the
+ * sampled rows of both of its 128-row tiles, the candidates are the key blocks j <= 2I + 1, and K_I is counted
+ * over them; the kept entries are then written as two lists, still one per 128-row tile: the second tile's list
+ * is the ranking itself, the first tile's leaves out key block 2I + 1, which lies wholly after it.  out_order
+ * and out_count keep their per-tile shapes, so cosa_osk_attention is called on them with block_q = 128 as usual;
+ * the two tiles of a block then walk the same K/V tiles in the same order.  kap_scores / kap_flags are not
+ * available in this mode.
  * Scores are evaluated so that the list equals the one exact arithmetic would give whenever
  * neighbouring scores differ by more than ~1e-9 relative.  With top_p the prefix sums are taken over
  * float32 scores (relative error < 2^-15): K_i equals the exact count unless a prefix sum lies

@@ -149,10 +149,13 @@ def cosa_workspace_bytes(op: int, shape: CosaShape, opt: CosaOptions | None = No
     return int(_load().cosa_workspace_bytes(op, byref(shape), byref(opt) if opt is not None else None))
 
 
-def cosa_kap_select(q, k, budget: float, out_order, out_count, causal=True, stream=None, opt: CosaOptions | None = None):
-    """Stage 1: fills out_order [B,Hq,nQB,order_stride] / out_count [B,Hq,nQB] (int32)."""
+def cosa_kap_select(q, k, budget: float, out_order, out_count, causal=True, stream=None, opt: CosaOptions | None = None,
+                    block_q: int = 128):
+    """Stage 1: fills out_order [B,Hq,nQB,order_stride] / out_count [B,Hq,nQB] (int32); block_q = 256 makes one ranking
+    per 256-row query block (the lists stay per 128-row tile, see cosa.h)."""
     lib = _load()
     shape = make_shape(q, k, causal)
+    shape.block_q = block_q
     args = (_dev_ptr(q, torch.bfloat16, "q"), _dev_ptr(k, torch.bfloat16, "k"), byref(shape), c_float(budget),
             _dev_ptr(out_order, torch.int32, "out_order"), _dev_ptr(out_count, torch.int32, "out_count"),
             _stream_ptr(stream))

@@ -56,12 +56,14 @@ int own_scratch(size_t need, void** out) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-int check_shape(const cosa_shape* s) {
+// wide_q_ok: the caller accepts query blocks of 256 rows (KAP's shared-ranking variant)
+int check_shape(const cosa_shape* s, bool wide_q_ok = false) {
   if (!s) return COSA_ERR_INVALID_ARG;
   if (s->batch < 1 || s->hq < 1 || s->hkv < 1 || s->n < 1) return COSA_ERR_INVALID_ARG;
   if (s->hq % s->hkv != 0) return COSA_ERR_INVALID_ARG;
-  if (s->d != kHeadDim || s->block_q != kBlock || s->block_k != kBlock) return COSA_ERR_UNSUPPORTED;
-  if (s->n % kBlock != 0) return COSA_ERR_UNSUPPORTED;
+  if (s->d != kHeadDim || s->block_k != kBlock) return COSA_ERR_UNSUPPORTED;
+  if (s->block_q != kBlock && !(wide_q_ok && s->block_q == 2 * kBlock)) return COSA_ERR_UNSUPPORTED;
+  if (s->n % s->block_q != 0) return COSA_ERR_UNSUPPORTED;
   return COSA_OK;
 }
 
@@ -135,7 +137,7 @@ int32_t cosa_budget_count(float budget, int32_t candidates) {
 }
 
 size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt) {
-  if (check_shape(shape) != COSA_OK) return 0;
+  if (check_shape(shape, op == 0) != COSA_OK) return 0;
   cosa_options o = resolve_options(opt);
   size_t a = align_up(kap_scratch_bytes(shape, o), 256), b = align_up(osk_scratch_bytes(shape, o), 256);
   if (op == 0) return a;
@@ -145,7 +147,7 @@ size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options*
 
 int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, float budget, int32_t* out_order,
                        int32_t* out_count, void* stream, const cosa_options* opt) {
-  int rc = check_shape(shape);
+  int rc = check_shape(shape, true);
   if (rc != COSA_OK) return rc;
   if (!q || !k || !out_order || !out_count) return COSA_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k)) return COSA_ERR_INVALID_ARG;
@@ -171,11 +173,14 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   p.budget_fx = budget_to_fx(budget);
   p.scale = o.softmax_scale > 0.f ? (double)o.softmax_scale : 1.0 / sqrt((double)shape->d);
   p.top_p = (double)o.top_p;
+  p.qtiles = shape->block_q / kBlock;
+  if (p.qtiles == 2 && (o.kap_scores || o.kap_flags)) return COSA_ERR_UNSUPPORTED;   // the exports are per 128-row block
+  if (p.qtiles == 2 && p.rows * 2 > 64) return COSA_ERR_UNSUPPORTED;                  // stride 2 and below
   rc = resolve_paging(shape, o, s, &p.pg);
   if (rc != COSA_OK) return rc;
   // the list of the longest row must fit the pitch
   if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
-  if (kap_exact_smem_bytes(p.rows, nqb) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
+  if (kap_exact_smem_bytes(p.rows, nqb, p.qtiles) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const KapScratch L = kap_scratch_layout(shape, o);
   if (L.total == 0) {   // double precision throughout

@@ -45,6 +45,7 @@ struct KapParams {
   long long budget_fx;   // floor(budget_f32 * 2^20)
   double scale;          // softmax scale applied to the sampled logits
   double top_p;          // > 0: Top-p retention, capped by the budget count; 0: budget count alone
+  int qtiles;            // 1, or 2: one ranking per query block of 2 x 128 rows, shared by its two row tiles
   KvPaging pg;
 };
 
@@ -144,7 +145,7 @@ bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
 // sorts the screened scores, recomputes near-ties in double precision, writes the lists
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st);
-size_t kap_exact_smem_bytes(int rows, int nqb);
+size_t kap_exact_smem_bytes(int rows, int nqb, int qtiles);
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
 cudaError_t launch_reorder_lists(int32_t* order, const int32_t* count, int total_qb, int order_stride, int descending,

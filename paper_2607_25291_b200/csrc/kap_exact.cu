@@ -17,12 +17,13 @@ __device__ __forceinline__ bool sorts_before(unsigned long long ka, unsigned ia,
   return ka > kb || (ka == kb && ia < ib);
 }
 
-// smem: Qs[R][kPad] | Ks[KB*R][kPad] | Z[KB*R*R] | M[R][Jpad] | Mstar[R] | sort keys | sort ids
-__device__ void kap_exact_item(const KapParams& p, int b, int h, int i, int kb_per_iter, int sort_cap);
+// smem: Qs[R][kPad] | Ks[KB*R][kPad] | Z[KB*R*R] | M[R][Jpad] | Mstar[R] | score[Jpad] | sort keys | sort ids | flag[Jpad]
+// i_lo: the first row tile of the query block (the block has p.qtiles row tiles of 128 rows)
+__device__ void kap_exact_item(const KapParams& p, int b, int h, int i_lo, int kb_per_iter, int sort_cap);
 
 // grid (nQB, Hq, B): one CTA per (head, query block)
 __global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb_per_iter, int sort_cap) {
-  kap_exact_item(p, blockIdx.z, blockIdx.y, p.nqb - 1 - (int)blockIdx.x, kb_per_iter, sort_cap);
+  kap_exact_item(p, blockIdx.z, blockIdx.y, (p.nqb / p.qtiles - 1 - (int)blockIdx.x) * p.qtiles, kb_per_iter, sort_cap);
 }
 
 // 1-d grid: the CTAs share out the entries of a redo list (usually empty)
@@ -32,14 +33,16 @@ __global__ void __launch_bounds__(kThreads) kap_exact_list_kernel(KapParams p, c
   for (int e = blockIdx.x; e < n; e += gridDim.x) {
     const int flat = redo_list[1 + e];
     const int i = flat % p.nqb, bh = flat / p.nqb;
-    kap_exact_item(p, bh / p.hq, bh % p.hq, i, kb_per_iter, sort_cap);
+    kap_exact_item(p, bh / p.hq, bh % p.hq, i, kb_per_iter, sort_cap);   // i: first row tile of the block
     __syncthreads();
   }
 }
 
-__device__ void kap_exact_item(const KapParams& p, const int b, const int h, const int i, int kb_per_iter, int sort_cap) {
+__device__ void kap_exact_item(const KapParams& p, const int b, const int h, const int i_lo, int kb_per_iter, int sort_cap) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int R = p.rows;
+  const int R = p.rows;                 // sampled rows per row tile = sampled keys per key block
+  const int T = p.qtiles;               // row tiles of the query block
+  const int i = i_lo + T - 1;           // its last row tile
   const int g = h / (p.hq / p.hkv);
   const int J = p.causal ? i + 1 : p.nqb;
   const int Jpad = p.nqb | 1;
@@ -50,55 +53,72 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
   double* Z = Ks + (size_t)kb_per_iter * R * kPad;
   double* M = Z + (size_t)kb_per_iter * R * R;
   double* Mstar = M + (size_t)R * Jpad;
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(Mstar + R);
+  double* score = Mstar + R;                                   // [Jpad] sums over the rows of all tiles
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(score + Jpad);
   unsigned* ids = reinterpret_cast<unsigned*>(keys + sort_cap);
+  unsigned char* flag = reinterpret_cast<unsigned char*>(ids + sort_cap);   // [Jpad]
 
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+  for (int j = tid; j < J; j += kThreads) { score[j] = 0.0; flag[j] = 0; }
 
-  // sampled query rows of block i: tokens (i*R + r) * s
-  for (int e = tid; e < R * kHeadDim; e += kThreads) {
-    int r = e / kHeadDim, d = e % kHeadDim;
-    size_t tok = (size_t)(i * R + r) * p.stride;
-    Qs[r * kPad + d] = (double)__bfloat162float(qh[tok * kHeadDim + d]);
-  }
-
-  for (int j0 = 0; j0 < J; j0 += kb_per_iter) {
-    const int nb = min(kb_per_iter, J - j0);
+  // one row tile after the other: its block maxima M[r,j], its row maxima M*[r], its share of the sums of Eq. (11)
+  for (int tile = 0; tile < T; ++tile) {
+    const int row0 = (i_lo + tile) * R;          // index of the tile's first sampled row in its head
     __syncthreads();
-    for (int e = tid; e < nb * R * kHeadDim; e += kThreads) {
-      int c = e / kHeadDim, d = e % kHeadDim;  // c: sampled key within this group of blocks
-      const int tok = (j0 * R + c) * p.stride;
-      Ks[c * kPad + d] = (double)__bfloat162float(p.k[(size_t)kv_row(p.pg, b, p.hkv, g, p.n, tok) * kHeadDim + d]);
+    for (int e = tid; e < R * kHeadDim; e += kThreads) {
+      int r = e / kHeadDim, d = e % kHeadDim;
+      size_t tok = (size_t)(row0 + r) * p.stride;
+      Qs[r * kPad + d] = (double)__bfloat162float(qh[tok * kHeadDim + d]);
     }
-    __syncthreads();
-    for (int e = tid; e < nb * R * R; e += kThreads) {
-      int c = e % (nb * R), r = e / (nb * R);
-      const double* qr = Qs + r * kPad;
-      const double* kc = Ks + c * kPad;
-      double acc = 0.0;
+    for (int j0 = 0; j0 < J; j0 += kb_per_iter) {
+      const int nb = min(kb_per_iter, J - j0);
+      __syncthreads();
+      for (int e = tid; e < nb * R * kHeadDim; e += kThreads) {
+        int c = e / kHeadDim, d = e % kHeadDim;  // c: sampled key within this group of blocks
+        const int tok = (j0 * R + c) * p.stride;
+        Ks[c * kPad + d] = (double)__bfloat162float(p.k[(size_t)kv_row(p.pg, b, p.hkv, g, p.n, tok) * kHeadDim + d]);
+      }
+      __syncthreads();
+      for (int e = tid; e < nb * R * R; e += kThreads) {
+        int c = e % (nb * R), r = e / (nb * R);
+        const double* qr = Qs + r * kPad;
+        const double* kc = Ks + c * kPad;
+        double acc = 0.0;
 #pragma unroll 8
-      for (int d = 0; d < kHeadDim; ++d) acc = fma(qr[d], kc[d], acc);
-      Z[(size_t)r * (kb_per_iter * R) + c] = acc * p.scale;
+        for (int d = 0; d < kHeadDim; ++d) acc = fma(qr[d], kc[d], acc);
+        Z[(size_t)r * (kb_per_iter * R) + c] = acc * p.scale;
+      }
+      __syncthreads();
+      for (int e = tid; e < nb * R; e += kThreads) {
+        int jj = e % nb, r = e / nb;
+        int j = j0 + jj;
+        const double* zr = Z + (size_t)r * (kb_per_iter * R) + jj * R;
+        int cmax = R;  // sampled keys of this block the row may see: key j*R + c <= row0 + r
+        if (p.causal) cmax = max(0, min(R, row0 + r - j * R + 1));
+        double m = -INFINITY;
+        for (int c = 0; c < cmax; ++c) m = fmax(m, zr[c]);
+        M[(size_t)r * Jpad + j] = m;
+      }
     }
     __syncthreads();
-    for (int e = tid; e < nb * R; e += kThreads) {
-      int jj = e % nb, r = e / nb;
-      int j = j0 + jj;
-      const double* zr = Z + (size_t)r * (kb_per_iter * R) + jj * R;
-      int cmax = R;  // valid sampled keys of this block for this row
-      if (p.causal && j == i) cmax = r + 1;
-      double m = zr[0];
-      for (int c = 1; c < cmax; ++c) m = fmax(m, zr[c]);
-      M[(size_t)r * Jpad + j] = m;
+    // M*[r]: the row's maximum over all candidate blocks
+    for (int r = tid / 32; r < R; r += kThreads / 32) {
+      double m = -INFINITY;
+      for (int j = tid % 32; j < J; j += 32) m = fmax(m, M[(size_t)r * Jpad + j]);
+      for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (tid % 32 == 0) Mstar[r] = m;
     }
-  }
-  __syncthreads();
-  // M*[r]: the row's maximum over all candidate blocks
-  for (int r = tid / 32; r < R; r += kThreads / 32) {
-    double m = -INFINITY;
-    for (int j = tid % 32; j < J; j += 32) m = fmax(m, M[(size_t)r * Jpad + j]);
-    for (int o = 16; o > 0; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (tid % 32 == 0) Mstar[r] = m;
+    __syncthreads();
+    for (int j = tid; j < J; j += kThreads) {
+      double sj = score[j];
+      bool fj = flag[j] != 0;
+      for (int r = 0; r < R; ++r) {
+        double mv = M[(size_t)r * Jpad + j], ms = Mstar[r];
+        sj += exp(mv - ms);          // 0 for a row that sees nothing of the block
+        fj |= (mv == ms);
+      }
+      score[j] = sj; flag[j] = fj ? 1 : 0;
+    }
   }
   __syncthreads();
   const size_t dbg_row = ((size_t)(b * p.hq + h) * p.nqb + i) * p.nqb;
@@ -106,17 +126,12 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
   while (P2 < J) P2 <<= 1;
   for (int j = tid; j < P2; j += kThreads) {
     if (j < J) {
-      double s = 0.0;
-      bool flag = false;
-      for (int r = 0; r < R; ++r) {
-        double mv = M[(size_t)r * Jpad + j], ms = Mstar[r];
-        s += exp(mv - ms);
-        flag |= (mv == ms);
-      }
-      keys[j] = (unsigned long long)__double_as_longlong(s) | (flag ? (1ULL << 63) : 0ULL);
+      const double sj = score[j];
+      const bool fj = flag[j] != 0;
+      keys[j] = (unsigned long long)__double_as_longlong(sj) | (fj ? (1ULL << 63) : 0ULL);
       ids[j] = (unsigned)j;
-      if (p.dbg_scores) p.dbg_scores[dbg_row + j] = (float)s;
-      if (p.dbg_flags) p.dbg_flags[dbg_row + j] = flag ? 1 : 0;
+      if (p.dbg_scores) p.dbg_scores[dbg_row + j] = (float)sj;
+      if (p.dbg_flags) p.dbg_flags[dbg_row + j] = fj ? 1 : 0;
     } else {
       keys[j] = 0ULL;
       ids[j] = 0xffffffffu;
@@ -143,9 +158,9 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
     }
   }
   int K = budget_count_fx(p.budget_fx, J);
+  __shared__ int k_topp, pos_after;
   if (p.top_p > 0.0) {
     // Top-p retention (text after Eq. 13): prefix sums along the order, sequentially in double precision
-    __shared__ int k_topp;
     if (tid == 0) {
       double total = 0.0;
       for (int t = 0; t < J; ++t) total += __longlong_as_double((long long)(keys[t] & ~(1ULL << 63)));
@@ -160,12 +175,27 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
     }
     __syncthreads();
     K = min(K, k_topp);
-    __syncthreads();   // the list kernel reuses k_topp for its next item
   }
-  const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  int32_t* dst = p.order + row * p.order_stride;
-  for (int t = tid; t < p.order_stride; t += kThreads) dst[t] = (t < K) ? (int32_t)ids[t] : -1;
-  if (tid == 0) p.count[row] = K;
+  // the last row tile takes the kept entries as they are; an earlier tile leaves out the key blocks wholly after it
+  if (tid == 0) pos_after = K;
+  __syncthreads();
+  if (T == 2 && p.causal) {
+    for (int t = tid; t < K; t += kThreads)
+      if ((int)ids[t] == i) pos_after = t;
+    __syncthreads();
+  }
+  const size_t row_lo = (size_t)(b * p.hq + h) * p.nqb + i_lo;
+  for (int tile = 0; tile < T; ++tile) {
+    const bool drop = tile < T - 1 && pos_after < K;
+    const int kept = K - (drop ? 1 : 0);
+    int32_t* dst = p.order + (row_lo + tile) * p.order_stride;
+    for (int t = tid; t < p.order_stride; t += kThreads) {
+      const int src = (drop && t >= pos_after) ? t + 1 : t;
+      dst[t] = (t < kept) ? (int32_t)ids[src] : -1;
+    }
+    if (tid == 0) p.count[row_lo + tile] = kept;
+  }
+  __syncthreads();   // the list kernel reuses the shared words for its next item
 }
 
 int next_pow2(int x) {
@@ -181,16 +211,17 @@ int kb_per_iter_for(int rows) {
 
 }  // namespace
 
-size_t kap_exact_smem_bytes(int rows, int nqb) {
+size_t kap_exact_smem_bytes(int rows, int nqb, int qtiles) {
+  (void)qtiles;   // the row tiles of a block are worked through one after the other in the same buffers
   int kb = kb_per_iter_for(rows);
   int sort_cap = next_pow2(nqb);
   size_t doubles = (size_t)rows * kPad + (size_t)kb * rows * kPad + (size_t)kb * rows * rows +
-                   (size_t)rows * (nqb | 1) + rows;
-  return doubles * 8 + (size_t)sort_cap * 12;
+                   (size_t)rows * (nqb | 1) + rows + (nqb | 1);
+  return doubles * 8 + (size_t)sort_cap * 12 + (size_t)((nqb | 1) + 15) / 16 * 16;
 }
 
 cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st) {
-  size_t smem = kap_exact_smem_bytes(p.rows, p.nqb);
+  size_t smem = kap_exact_smem_bytes(p.rows, p.nqb, p.qtiles);
   if (redo_list) {
     cudaError_t e = cudaFuncSetAttribute(kap_exact_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -199,7 +230,7 @@ cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaS
   }
   cudaError_t e = cudaFuncSetAttribute(kap_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(p.nqb, p.hq, p.batch);
+  dim3 grid(p.nqb / p.qtiles, p.hq, p.batch);
   kap_exact_kernel<<<grid, kThreads, smem, st>>>(p, kb_per_iter_for(p.rows), next_pow2(p.nqb));
   return cudaGetLastError();
 }

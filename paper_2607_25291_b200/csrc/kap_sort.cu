@@ -26,20 +26,21 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kMaxTied = 96;
-constexpr int kMaxRows = 32;
+constexpr int kMaxRows = 64;   // sampled rows of one (possibly two-tile) query block
 constexpr int kPad = kHeadDim + 1;
 
 struct Tied { int pos; unsigned id; double s; };
 
 // dest[r] = max over the visible sampled keys c of block jb[r] of (Q~[r] . K~[jb[r]*R + c]) * scale, in double
-// precision; rows with jb[r] < 0 are left alone.  All threads of the CTA call it.
-__device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, int b, int g, int i, int R,
+// precision, for the `rows` sampled rows of the query block whose first sampled row has index row0 in its head
+// (-inf when the row sees nothing of the block); rows with jb[r] < 0 are left alone.  All threads of the CTA call it.
+__device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, int b, int g, int row0, int rows, int R,
                               const int* jb, double* dest, int tid) {
-  for (int e = tid; e < R * R; e += kThreads) {
+  for (int e = tid; e < rows * R; e += kThreads) {
     const int r = e / R, c = e % R;
     double z = -INFINITY;
     const int kc = jb[r] * R + c;  // sampled key index
-    if (jb[r] >= 0 && (!p.causal || kc <= i * R + r)) {
+    if (jb[r] >= 0 && (!p.causal || kc <= row0 + r)) {
       const uint4* src = reinterpret_cast<const uint4*>(p.k + (size_t)kv_row(p.pg, b, p.hkv, g, p.n, kc * p.stride) * kHeadDim);
       const double* qr = Qs + r * kPad;
       double acc = 0.0;
@@ -58,7 +59,7 @@ __device__ void f64_block_max(const KapParams& p, const double* Qs, double* Z, i
     Z[r * R + c] = z;
   }
   __syncthreads();
-  if (tid < R && jb[tid] >= 0) {
+  if (tid < rows && jb[tid] >= 0) {
     double m = Z[tid * R];
     for (int c = 1; c < R; ++c) m = fmax(m, Z[tid * R + c]);
     dest[tid] = m;
@@ -71,53 +72,69 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
   unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);        // [tie_bytes]
-  double* Qs = reinterpret_cast<double*>(tie + tie_bytes);                       // [R][kPad]
-  double* Z = Qs + (size_t)p.rows * kPad;                                        // [R][R]
+  double* Qs = reinterpret_cast<double*>(tie + tie_bytes);                       // [R * tiles][kPad]
+  double* Z = Qs + (size_t)p.rows * p.qtiles * kPad;                             // [R * tiles][R]
   __shared__ Tied tied[kMaxTied];
   __shared__ double Mrow[kMaxRows], Mstar[kMaxRows], Msecond[kMaxRows];
   __shared__ int jb[kMaxRows], j1[kMaxRows], j2[kMaxRows];
   __shared__ int n_tied, tail_end;
 
-  const int R = p.rows;
-  const int i = p.nqb - 1 - (int)blockIdx.x;
+  const int R = p.rows;                       // sampled rows per 128-row tile
+  const int T = p.qtiles;                     // row tiles that share this ranking
+  const int RT = R * T;
+  const int big = p.nqb / T - 1 - (int)blockIdx.x;
+  const int i_lo = big * T, i = i_lo + T - 1; // first and last row tile of the query block
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.hq / p.hkv);
-  const int J = p.causal ? i + 1 : p.nqb;
+  const int J = p.causal ? i + 1 : p.nqb;     // candidates: key blocks some row of the block may see
   const int tid = threadIdx.x;
-  const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  if (sp.hard[row]) {  // left to the double-precision kernel
-    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row;
+  const size_t row_lo = (size_t)(b * p.hq + h) * p.nqb + i_lo;
+  const size_t row = row_lo + (T - 1);
+  bool hard = false;
+  unsigned long long amb = 0ULL;              // bit r: sampled row r of the block was too close to call
+  for (int t = 0; t < T; ++t) {
+    hard = hard || sp.hard[row_lo + t];
+    amb |= (unsigned long long)sp.ambmask[row_lo + t] << (t * R);
+  }
+  if (hard) {  // left to the double-precision kernel
+    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
     return;
   }
-  const unsigned amb = sp.ambmask[row];
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
 
-  const float* srow = sp.scores + row * p.nqb;
+  // scores of the block = sum over its row tiles (the sum of Eq. 11 splits over the rows), flags = OR; a tile has
+  // no score for key blocks wholly after it
   int P2 = 2;
   while (P2 < J) P2 <<= 1;
   for (int j = tid; j < P2; j += kThreads) {
     unsigned long long key = 0ULL;
     if (j < J) {
-      const float v = srow[j];
-      const unsigned hi = (__float_as_uint(fabsf(v))) | (v < 0.f ? 0x80000000u : 0u);
-      key = ((unsigned long long)hi << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
+      float sum = 0.f;
+      unsigned flag = 0u;
+      for (int t = 0; t < T; ++t) {
+        if (p.causal && j > i_lo + t) continue;
+        const float v = sp.scores[(row_lo + t) * p.nqb + j];
+        sum += fabsf(v);
+        flag |= (v < 0.f) ? 0x80000000u : 0u;
+      }
+      key = ((unsigned long long)(__float_as_uint(sum) | flag) << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
     }
     keys[j] = key;
   }
   if (tid == 0) { n_tied = 0; tail_end = 0; }
-  if (tid < R) {
-    const int2 js = reinterpret_cast<const int2*>(sp.jstar)[(size_t)(b * p.hq + h) * (p.n / p.stride) + (size_t)i * R + tid];
+  if (tid < RT) {
+    const int2 js = reinterpret_cast<const int2*>(sp.jstar)[(size_t)(b * p.hq + h) * (p.n / p.stride) + (size_t)i_lo * R + tid];
     j1[tid] = js.x; j2[tid] = js.y;
   }
   bool have_mstar = false;
   auto load_q_and_mstar = [&]() {
-    for (int e = tid; e < R * kHeadDim; e += kThreads) {
+    for (int e = tid; e < RT * kHeadDim; e += kThreads) {
       const int r = e / kHeadDim, d = e % kHeadDim;
-      Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i * R + r) * p.stride) * kHeadDim + d]);
+      Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i_lo * R + r) * p.stride) * kHeadDim + d]);
     }
-    if (tid < R) jb[tid] = j1[tid];
+    if (tid < RT) jb[tid] = j1[tid];
     __syncthreads();
-    f64_block_max(p, Qs, Z, b, g, i, R, jb, Mstar, tid);
+    f64_block_max(p, Qs, Z, b, g, i_lo * R, RT, R, jb, Mstar, tid);
     have_mstar = true;
   };
   __syncthreads();
@@ -125,17 +142,17 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   if (amb) {
     // ---- 1. settle the rows the screen could not call
     load_q_and_mstar();
-    if (tid < R) { jb[tid] = ((amb >> tid) & 1u) ? j2[tid] : -1; Msecond[tid] = -INFINITY; }
+    if (tid < RT) { jb[tid] = ((amb >> tid) & 1ULL) ? j2[tid] : -1; Msecond[tid] = -INFINITY; }
     __syncthreads();
-    f64_block_max(p, Qs, Z, b, g, i, R, jb, Msecond, tid);
+    f64_block_max(p, Qs, Z, b, g, i_lo * R, RT, R, jb, Msecond, tid);
     if (tid == 0) {
-      for (int r = 0; r < R; ++r) {
-        if (!((amb >> r) & 1u)) continue;
+      for (int r = 0; r < RT; ++r) {
+        if (!((amb >> r) & 1ULL)) continue;
         for (int which = 0; which < 2; ++which) {       // the HRM flag of both of the row's contenders
           const int j = which ? j2[r] : j1[r];
           bool flag = false;
-          for (int q = 0; q < R && !flag; ++q) {
-            if ((amb >> q) & 1u) {
+          for (int q = 0; q < RT && !flag; ++q) {
+            if ((amb >> q) & 1ULL) {
               const double best = fmax(Mstar[q], Msecond[q]);
               flag = (j == j1[q] && Mstar[q] == best) || (j == j2[q] && Msecond[q] == best);
             } else {
@@ -145,8 +162,8 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
           keys[j] = (keys[j] & 0x7fffffffffffffffULL) | (flag ? 0x8000000000000000ULL : 0ULL);
         }
       }
-      for (int r = 0; r < R; ++r)
-        if ((amb >> r) & 1u) Mstar[r] = fmax(Mstar[r], Msecond[r]);
+      for (int r = 0; r < RT; ++r)
+        if ((amb >> r) & 1ULL) Mstar[r] = fmax(Mstar[r], Msecond[r]);
     }
     __syncthreads();
   }
@@ -291,18 +308,20 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
   __syncthreads();
   const int nt = n_tied;
   if (nt > kMaxTied) {  // pathological: too many near ties
-    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row;
+    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
     return;
   }
   if (nt > 0) {
     if (!have_mstar) load_q_and_mstar();
     for (int round = 0; round < nt; ++round) {
-      if (tid < R) jb[tid] = (int)tied[round].id;
+      if (tid < RT) jb[tid] = (int)tied[round].id;
       __syncthreads();
-      f64_block_max(p, Qs, Z, b, g, i, R, jb, Mrow, tid);
+      if (tid < RT) Mrow[tid] = -INFINITY;
+      __syncthreads();
+      f64_block_max(p, Qs, Z, b, g, i_lo * R, RT, R, jb, Mrow, tid);
       if (tid == 0) {
         double s = 0.0;
-        for (int r = 0; r < R; ++r) s += exp(Mrow[r] - Mstar[r]);
+        for (int r = 0; r < RT; ++r) s += exp(Mrow[r] - Mstar[r]);   // exp(-inf) = 0: the row sees nothing of the block
         tied[round].s = s;
       }
       __syncthreads();
@@ -338,10 +357,26 @@ __global__ void __launch_bounds__(kThreads) kap_sort_kernel(KapParams p, KapScre
     }
     __syncthreads();
   }
-  int32_t* dst = p.order + row * p.order_stride;
-  for (int t = tid; t < p.order_stride; t += kThreads)
-    dst[t] = (t < K) ? (int32_t)(0xffffffffu - (unsigned)(keys[t] & 0xffffffffu)) : -1;
-  if (tid == 0) p.count[row] = K;
+  // the last row tile of the block takes the kept entries as they are; an earlier tile leaves out the key blocks that
+  // lie wholly after it (with two tiles: the one block i), keeping the order
+  __shared__ int pos_after;
+  if (tid == 0) pos_after = K;
+  __syncthreads();
+  if (T == 2 && p.causal) {
+    for (int t = tid; t < K; t += kThreads)
+      if ((int)(0xffffffffu - (unsigned)(keys[t] & 0xffffffffu)) == i) pos_after = t;
+    __syncthreads();
+  }
+  for (int tile = 0; tile < T; ++tile) {
+    const bool drop = tile < T - 1 && pos_after < K;      // this tile leaves one entry out
+    const int kept = K - (drop ? 1 : 0);
+    int32_t* dst = p.order + (row_lo + tile) * p.order_stride;
+    for (int t = tid; t < p.order_stride; t += kThreads) {
+      const int src = (drop && t >= pos_after) ? t + 1 : t;
+      dst[t] = (t < kept) ? (int32_t)(0xffffffffu - (unsigned)(keys[src] & 0xffffffffu)) : -1;
+    }
+    if (tid == 0) p.count[row_lo + tile] = kept;
+  }
 }
 
 int next_pow2(int x) {
@@ -353,13 +388,14 @@ int next_pow2(int x) {
 }  // namespace
 
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st) {
-  if (p.rows > kMaxRows) return cudaErrorInvalidValue;
+  if (p.rows * p.qtiles > kMaxRows || p.nqb % p.qtiles != 0 || p.qtiles < 1 || p.qtiles > 2) return cudaErrorInvalidValue;
   const int cap = next_pow2(p.nqb);
   const int tie_bytes = (cap + 15) / 16 * 16;
-  size_t smem = (size_t)cap * 8 + tie_bytes + ((size_t)p.rows * kPad + (size_t)p.rows * p.rows) * 8;
+  const size_t rt = (size_t)p.rows * p.qtiles;
+  size_t smem = (size_t)cap * 8 + tie_bytes + (rt * kPad + rt * p.rows) * 8;
   cudaError_t e = cudaFuncSetAttribute(kap_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid(p.nqb, p.hq, p.batch);
+  dim3 grid(p.nqb / p.qtiles, p.hq, p.batch);
   kap_sort_kernel<<<grid, kThreads, smem, st>>>(p, sp, tau_score, cap, tie_bytes);
   return cudaGetLastError();
 }

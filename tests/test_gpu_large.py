@@ -159,6 +159,37 @@ def test_qwen3_32k_paged_equals_dense():
             assert torch.equal(a, b)
 
 
+def test_qwen3_32k_wide_query_blocks_sampled():
+    """block_q = 256 lists at 32K against the oracle on sampled blocks, and OSK on them."""
+    w = WORKLOADS["qwen3_32k"]
+    qb, kb, vb, _ = w.make()
+    q, k, v = (to_dev(x) for x in (qb, kb, vb))
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(w.kap_budget, nqb) + 7) // 8 * 8
+    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+    bufs = dict(out=torch.empty_like(q), lse=torch.empty(1, w.hq, w.n, dtype=torch.float32, device="cuda"),
+                visited=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                scored=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                decisions=torch.zeros(1, w.hq, nqb, (pitch + 31) // 32, dtype=torch.int32, device="cuda"))
+    opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch,
+                               out_scored=bufs["scored"], out_decisions=bufs["decisions"])
+    cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=opt, block_q=256)
+    cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+    assert cosa.cosa_device_status() == 0
+    order_np, count_np = _np(order), _np(count)
+    wide = sorted(set(b // 2 for b in sample_blocks(nqb)))
+    hv = HeadView(qb, kb, vb)
+    for h in range(0, w.hq, 3):
+        qf, kf, vf = hv.get(h)
+        ref_order, ref_count = O.kap_select_wide(qf, kf, s=w.stride, budget=w.kap_budget, order_stride=pitch, wide_blocks=wide)
+        tiles = [2 * b + t for b in wide for t in (0, 1)]
+        for i in tiles:
+            assert ref_count[0, i] == count_np[h, i] and np.array_equal(ref_order[0, i], order_np[h, i]), (h, i)
+        one = {k_: t[:, h:h + 1] for k_, t in bufs.items()}
+        check_osk_against_oracle(qf, kf, vf, order_np[h:h + 1], count_np[h:h + 1], one, w.osk_budget, w.skip_scale, [0], tiles[::3])
+
+
 def test_llama31_64k_budget_sweep_sampled():
     w = WORKLOADS["llama31_64k_sweep"]
     qb, kb, vb, _ = w.make()

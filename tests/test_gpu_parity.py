@@ -385,6 +385,45 @@ def test_ablation_tables_run_and_show_the_effect_of_order():
     assert len(micro) == 1 and micro[0]["jump_ms"] > 0 and micro[0]["logical_ms"] > 0 and micro[0]["dense_ms"] > 0
 
 
+# ---------------------------------------------------------------------------------- block_q = 256 variant
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("budget", [0.3, 0.6, 1.0])
+def test_kap_wide_query_blocks_small(small, impl, budget):
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    nqb = q.shape[2] // 128
+    for stride in (8, 16):
+        order, count = alloc_lists(q.shape[1], nqb)
+        cosa.cosa_kap_select(q, k, budget, order, count, opt=cosa.default_options(stride=stride, impl=impl), block_q=256)
+        assert cosa.cosa_device_status() == 0
+        ref_order, ref_count = O.kap_select_wide(qf, kf, s=stride, budget=budget, order_stride=nqb)
+        assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    # the per-tile lists are ordinary lists: OSK runs on them unchanged
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cosa.cosa_validate_order(order, count, cosa.make_shape(q, k, True), status)
+    assert int(status.item()) == 0
+    bufs = run_osk(q, k, v, order, count, 0.4, 150.0, impl)
+    check_osk_against_oracle(qf, kf, vf, ref_order, ref_count, bufs, 0.4, 150.0, range(q.shape[1]), range(nqb))
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_kap_wide_query_blocks_4k(cfg1, impl):
+    w = cfg1["w"]
+    q, k, _ = cfg1["dev"]
+    qf, kf, _ = cfg1["f64"]
+    order, count = alloc_lists(w.hq, w.n_blocks)
+    cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride, impl=impl, top_p=0.0),
+                         block_q=256)
+    ref_order, ref_count = O.kap_select_wide(qf, kf, s=w.stride, budget=w.kap_budget, order_stride=w.n_blocks)
+    assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    # both tiles of a block share the ranking: the first tile's list is the second's minus the last key block
+    o, c = _np(order), _np(count)
+    for h in range(w.hq):
+        for big in range(w.n_blocks // 2):
+            hi = o[h, 2 * big + 1, :c[h, 2 * big + 1]].tolist()
+            assert o[h, 2 * big, :c[h, 2 * big]].tolist() == [j for j in hi if j != 2 * big + 1]
+
+
 # ---------------------------------------------------------------------------------- paged K/V
 def _pools(w, page_size):
     """K and V of the workload as page pools that share one seeded page table."""
