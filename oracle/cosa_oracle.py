@@ -204,7 +204,7 @@ def kap_scores_wide(q, k, h, big, s=8, block=128, tiles=2, causal=True):
 
 
 def kap_select_wide(q, k, s=8, budget=0.25, causal=True, block=128, tiles=2, order_stride=None, heads=None,
-                    wide_blocks=None):
+                    wide_blocks=None, top_p=None):
     """Stage-1 lists when one ranking is made per query block of tiles*block rows and shared by
     its `tiles` row tiles of `block` rows (the block_q = 256 variant).  The wide block keeps the
     first K = budget_count(budget, candidates) entries of its flag-grouped order; row tile t of
@@ -221,7 +221,10 @@ def kap_select_wide(q, k, s=8, budget=0.25, causal=True, block=128, tiles=2, ord
         for big in (range(nbig) if wide_blocks is None else wide_blocks):
             scores, flags, _ = kap_scores_wide(q, k, h, big, s, block, tiles, causal)
             rho = flag_grouped_order(scores, flags)
-            kept = rho[:budget_count(budget, len(rho))]
+            n_keep = budget_count(budget, len(rho))
+            if top_p is not None:
+                n_keep = min(n_keep, topp_count(scores[rho], top_p)[0])
+            kept = rho[:n_keep]
             for t in range(tiles):
                 i = big * tiles + t
                 ids = [j for j in kept if (not causal) or j <= i]

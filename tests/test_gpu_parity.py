@@ -407,6 +407,29 @@ def test_kap_wide_query_blocks_small(small, impl, budget):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+def test_kap_wide_query_blocks_noncausal_and_top_p(small, impl):
+    q, k, _ = small["dev"]
+    qf, kf, _ = small["f64"]
+    nqb = q.shape[2] // 128
+    order, count = alloc_lists(q.shape[1], nqb)
+    cosa.cosa_kap_select(q, k, 0.5, order, count, causal=False, opt=cosa.default_options(impl=impl), block_q=256)
+    ref_order, ref_count = O.kap_select_wide(qf, kf, s=8, budget=0.5, causal=False, order_stride=nqb)
+    assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    assert (ref_count[:, 0::2] == ref_count[:, 1::2]).all()          # nothing lies after a tile: both lists are the ranking
+    # Top-p on the summed scores: p = 1 keeps every candidate, a vanishing p the first entry
+    cosa.cosa_kap_select(q, k, 1.0, order, count, opt=cosa.default_options(impl=impl, top_p=1.0), block_q=256)
+    ref_order, ref_count = O.kap_select_wide(qf, kf, s=8, budget=1.0, order_stride=nqb, top_p=1.0)
+    assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
+    cosa.cosa_kap_select(q, k, 1.0, order, count, opt=cosa.default_options(impl=impl, top_p=1e-9), block_q=256)
+    c = _np(count)
+    assert (c[:, 1::2] == 1).all() and (c[:, 0::2] <= 1).all()
+    # shapes the variant cannot take
+    with pytest.raises(cosa.CosaError):
+        cosa.cosa_kap_select(q[:, :, :896].contiguous(), k[:, :, :896].contiguous(), 0.5, order, count, block_q=256,
+                             opt=cosa.default_options())
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 def test_kap_wide_query_blocks_4k(cfg1, impl):
     w = cfg1["w"]
     q, k, _ = cfg1["dev"]
