@@ -12,8 +12,12 @@ Two tables, both produced with the library's own kernels only:
   {25, 50, 75} % and 32K / 64K / 128K, with the library's dense path and PyTorch SDPA as the dense
   references.
 
+* ``stack``  the 36-layer stack of 128K layers with layer-varying needle density: attention time of the whole
+  prefill (KAP + OSK per layer, summed) against the library's dense path and PyTorch SDPA.
+
     python -m paper_2607_25291_b200.ablation remap [--workload qwen3_32k]
     python -m paper_2607_25291_b200.ablation micro [--lengths 32k,64k,128k]
+    python -m paper_2607_25291_b200.ablation stack [--workload qwen3_128k_x36] [--dense-every 6]
 """
 import argparse
 
@@ -137,6 +141,49 @@ def micro_table(workloads, budgets=MICRO_BUDGETS, with_sdpa=True):
     return rows
 
 
+def stack_table(workload, dense_every=6):
+    """One row per layer: KAP ms, OSK ms, blocks computed; the dense references are timed on every dense_every-th
+    layer (their time does not depend on the data) and averaged."""
+    rows, dense_ms, sdpa_ms = [], [], []
+    nqb, hq = workload.n_blocks, workload.hq
+    pitch = (cosa.cosa_budget_count(workload.kap_budget, nqb) + 7) // 8 * 8
+    order = torch.empty(1, hq, nqb, pitch, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, hq, nqb, dtype=torch.int32, device="cuda")
+    visited = torch.empty(1, hq, nqb, dtype=torch.int32, device="cuda")
+    opt = cosa.default_options(stride=workload.stride, skip_scale=workload.skip_scale, order_stride=pitch)
+    out = None
+    for layer in range(workload.layers):
+        qb, kb, vb, _ = workload.make(layer=layer)
+        q, k, v = _dev(qb), _dev(kb), _dev(vb)
+        if out is None:
+            out = torch.empty_like(q)
+        kap = _time(lambda: cosa.cosa_kap_select(q, k, workload.kap_budget, order, count, opt=opt), reps=2)
+        osk = _time(lambda: cosa.cosa_osk_attention(q, k, v, order, count, workload.osk_budget, out, None, visited, opt=opt), reps=2)
+        rows.append(dict(layer=layer, kap_ms=kap, osk_ms=osk, listed=int(count.sum()), computed=int(visited.sum())))
+        if layer % dense_every == 0:
+            tri = torch.arange(nqb, device="cuda", dtype=torch.int32)
+            full = torch.where(tri[None, :] <= tri[:, None], tri[None, :].expand(nqb, nqb),
+                               torch.full((), -1, dtype=torch.int32, device="cuda")).expand(1, hq, nqb, nqb).contiguous()
+            fcount = (tri + 1).expand(1, hq, nqb).contiguous()
+            dopt = cosa.default_options(order_stride=nqb)
+            dense_ms.append(_time(lambda: cosa.cosa_osk_attention(q, k, v, full, fcount, 1.0, out, None, None, opt=dopt), reps=1))
+            sdpa_ms.append(_time(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True), reps=1))
+            del full
+        del q, k, v
+    return rows, float(np.mean(dense_ms)), float(np.mean(sdpa_ms))
+
+
+def _print_stack(rows, dense_ms, sdpa_ms):
+    print("| layer | KAP ms | OSK ms | KAP+OSK ms | blocks listed | blocks computed |")
+    print("|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['layer']} | {r['kap_ms']:.2f} | {r['osk_ms']:.2f} | {r['kap_ms'] + r['osk_ms']:.2f} | {r['listed']} | {r['computed']} |")
+    total = sum(r["kap_ms"] + r["osk_ms"] for r in rows)
+    n = len(rows)
+    print(f"\ntotal over {n} layers: {total:.1f} ms; dense path {dense_ms:.1f} ms/layer = {dense_ms * n:.0f} ms "
+          f"({dense_ms * n / total:.2f}x); SDPA {sdpa_ms:.1f} ms/layer = {sdpa_ms * n:.0f} ms ({sdpa_ms * n / total:.2f}x)")
+
+
 def _print_remap(rows):
     print("| stage-1 budget | Delta | skip ratio, KAP order | skip ratio, natural order | rel. error, KAP order | rel. error, natural order |")
     print("|---|---|---|---|---|---|")
@@ -159,11 +206,15 @@ def _print_micro(rows):
 def main():
     from synth.configs import WORKLOADS
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("table", choices=["remap", "micro"])
+    ap.add_argument("table", choices=["remap", "micro", "stack"])
+    ap.add_argument("--dense-every", type=int, default=6)
     ap.add_argument("--workload", default="qwen3_32k")
     ap.add_argument("--lengths", default="32k,64k,128k")
     args = ap.parse_args()
-    if args.table == "remap":
+    if args.table == "stack":
+        wl = WORKLOADS[args.workload if args.workload != "qwen3_32k" else "qwen3_128k_x36"]
+        _print_stack(*stack_table(wl, args.dense_every))
+    elif args.table == "remap":
         _print_remap(remap_table(WORKLOADS[args.workload]))
     else:
         _print_micro(micro_table([WORKLOADS[MICRO_WORKLOADS[x]] for x in args.lengths.split(",")]))
