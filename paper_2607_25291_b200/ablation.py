@@ -12,12 +12,15 @@ Two tables, both produced with the library's own kernels only:
   {25, 50, 75} % and 32K / 64K / 128K, with the library's dense path and PyTorch SDPA as the dense
   references.
 
+* ``sweep``  the 64K budget sweep: Stage-1 {50, 25, 12.5} % x Stage-2 {off, 0.5x, 0.25x}: latencies, blocks listed /
+  scored / computed, distance of the output from dense attention.
 * ``stack``  the 36-layer stack of 128K layers with layer-varying needle density: attention time of the whole
   prefill (KAP + OSK per layer, summed) against the library's dense path and PyTorch SDPA.
 
     python -m paper_2607_25291_b200.ablation remap [--workload qwen3_32k]
     python -m paper_2607_25291_b200.ablation micro [--lengths 32k,64k,128k]
     python -m paper_2607_25291_b200.ablation stack [--workload qwen3_128k_x36] [--dense-every 6]
+    python -m paper_2607_25291_b200.ablation sweep        (the 64K budget sweep)
 """
 import argparse
 
@@ -184,6 +187,41 @@ def _print_stack(rows, dense_ms, sdpa_ms):
           f"({dense_ms * n / total:.2f}x); SDPA {sdpa_ms:.1f} ms/layer = {sdpa_ms * n:.0f} ms ({sdpa_ms * n / total:.2f}x)")
 
 
+def sweep_table(workload, stage1, stage2_mult):
+    """The budget sweep: Stage-1 budget x (Stage-2 budget as a multiple of it; 1.0 = Stage 2 off): latencies, blocks
+    listed / scored / computed, and the relative L2 distance of the output from the library's dense path."""
+    pb = Problem(workload)
+    nqb, hq = pb.nqb, workload.hq
+    tri = torch.arange(nqb, device="cuda", dtype=torch.int32)
+    full = torch.where(tri[None, :] <= tri[:, None], tri[None, :].expand(nqb, nqb),
+                       torch.full((), -1, dtype=torch.int32, device="cuda")).expand(1, hq, nqb, nqb).contiguous()
+    dense = torch.empty_like(pb.q)
+    cosa.cosa_osk_attention(pb.q, pb.k, pb.v, full, (tri + 1).expand(1, hq, nqb).contiguous(), 1.0, dense, None, None,
+                            opt=cosa.default_options(order_stride=nqb))
+    del full
+    dense_norm = float(dense.float().norm())
+    scored = torch.empty_like(pb.visited)
+    rows = []
+    for b1 in stage1:
+        kap = _time(lambda: pb.select(b1))
+        for mult in stage2_mult:
+            tb = 1.0 if mult == 1.0 else b1 * mult
+            opt = cosa.default_options(skip_scale=workload.skip_scale, order_stride=nqb, out_scored=scored)
+            osk = _time(lambda: cosa.cosa_osk_attention(pb.q, pb.k, pb.v, pb.order, pb.count, tb, pb.out, None, pb.visited, opt=opt))
+            err = float((pb.out.float() - dense.float()).norm()) / dense_norm
+            rows.append(dict(stage1=b1, stage2=tb, kap_ms=kap, osk_ms=osk, listed=int(pb.count.sum()), scored=int(scored.sum()),
+                             computed=int(pb.visited.sum()), err=err))
+    return rows
+
+
+def _print_sweep(rows):
+    print("| stage-1 budget | stage-2 budget | KAP ms | OSK ms | blocks listed | scored | computed | rel. L2 distance from dense |")
+    print("|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        s2 = "off" if r["stage2"] >= 1.0 else f"{r['stage2']:.4f}"
+        print(f"| {r['stage1']:.3f} | {s2} | {r['kap_ms']:.2f} | {r['osk_ms']:.2f} | {r['listed']} | {r['scored']} | {r['computed']} | {r['err']:.3e} |")
+
+
 def _print_remap(rows):
     print("| stage-1 budget | Delta | skip ratio, KAP order | skip ratio, natural order | rel. error, KAP order | rel. error, natural order |")
     print("|---|---|---|---|---|---|")
@@ -206,12 +244,15 @@ def _print_micro(rows):
 def main():
     from synth.configs import WORKLOADS
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("table", choices=["remap", "micro", "stack"])
+    ap.add_argument("table", choices=["remap", "micro", "stack", "sweep"])
     ap.add_argument("--dense-every", type=int, default=6)
     ap.add_argument("--workload", default="qwen3_32k")
     ap.add_argument("--lengths", default="32k,64k,128k")
     args = ap.parse_args()
-    if args.table == "stack":
+    if args.table == "sweep":
+        from synth.configs import SWEEP_STAGE1, SWEEP_STAGE2_MULT
+        _print_sweep(sweep_table(WORKLOADS["llama31_64k_sweep"], SWEEP_STAGE1, SWEEP_STAGE2_MULT))
+    elif args.table == "stack":
         wl = WORKLOADS[args.workload if args.workload != "qwen3_32k" else "qwen3_128k_x36"]
         _print_stack(*stack_table(wl, args.dense_every))
     elif args.table == "remap":
