@@ -1,5 +1,6 @@
 // The C ABI declared in include/cosa.h: argument checks, option resolution, kernel dispatch.
 #include <math.h>
+#include <algorithm>
 #include <stdio.h>
 #include <string.h>
 
@@ -99,7 +100,7 @@ cosa_options resolve_options(const cosa_options* opt) {
 }  // namespace
 
 // scratch the kernels of one call need (beyond inputs and outputs)
-struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, total; };
+struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, slot_taken, maxima, total; int slots; };
 static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
   KapScratch L{};
   const int stride = o.stride > 0 ? o.stride : 8;
@@ -113,6 +114,12 @@ static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o)
   L.ambmask = off; off += align_up(heads * nqb * 4, 256);
   L.hard = off; off += align_up(heads * nqb, 256);
   L.redo_list = off; off += align_up((1 + heads * nqb) * 4, 256);
+  // the screen's parked block maxima: one area per CTA that can be resident on the current device
+  L.slots = kap_screen_slots();
+  if (L.slots <= 0) L.slots = 160;   // no usable device (a size query only): the count of the largest sm_100a part, rounded up
+  L.slots = std::min(L.slots, kap_screen_grid(s->batch, s->hq, s->hkv, (int)nqb, stride));
+  L.slot_taken = off; off += align_up((size_t)L.slots * 4, 256);
+  L.maxima = off; off += align_up((size_t)L.slots * kap_screen_slot_bytes(s->n, stride), 256);
   L.total = off;
   return L;
 }
@@ -206,6 +213,9 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.ambmask = reinterpret_cast<uint32_t*>(ws + L.ambmask);
   sp.hard = reinterpret_cast<uint8_t*>(ws + L.hard);
   sp.redo_list = reinterpret_cast<int32_t*>(ws + L.redo_list);
+  sp.slot_taken = reinterpret_cast<int32_t*>(ws + L.slot_taken);
+  sp.maxima = reinterpret_cast<float*>(ws + L.maxima);
+  sp.slots = L.slots;
   sp.batch = p.batch; sp.hq = p.hq; sp.hkv = p.hkv; sp.n = p.n; sp.nqb = nqb;
   sp.causal = p.causal; sp.stride = s;
   sp.scale = (float)p.scale;

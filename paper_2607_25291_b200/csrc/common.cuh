@@ -58,6 +58,9 @@ struct KapScreenParams {
   uint32_t* ambmask;     // [B,Hq,nQB]      bit r: sampled row r's two best blocks are too close to call in float32
   uint8_t* hard;         // [B,Hq,nQB]      1 = three blocks too close on some row: whole query block goes to double precision
   int32_t* redo_list;    // [1 + B*Hq*nQB]  [0] = number of entries, then flat (b*Hq+h)*nQB+i of query blocks to redo
+  float* maxima;         // [slots][key tiles][128 rows x 128/R blocks]  per-row block maxima of the CTA that holds the slot
+  int32_t* slot_taken;   // [slots]  0 = free; zeroed before every launch
+  int slots;             // CTAs that can be resident at once
   int batch, hq, hkv, n, nqb;
   int causal;
   int stride;
@@ -143,6 +146,11 @@ int32_t* device_status_word();
 cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st);
 bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
+// CTAs of the screen kernel that can be resident at once on the current device (0 on failure), and the bytes of
+// block-maxima scratch each of them needs
+int kap_screen_slots();
+int kap_screen_grid(int batch, int hq, int hkv, int nqb, int stride);   // CTAs of the screen kernel
+size_t kap_screen_slot_bytes(int n, int stride);
 // sorts the screened scores, recomputes near-ties in double precision, writes the lists
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st);
 size_t kap_exact_smem_bytes(int rows, int nqb, int qtiles);

@@ -1,16 +1,22 @@
 // KAP fast path, stage A: the proxy scores on the sm_100a tensor cores (Sec. 4.2, Eqs. 8-12;
 // Algorithm A steps 2-4).
 //
-// One CTA owns 128 sampled query rows = the R sampled rows of each of the G query heads of one
-// KV head for 128/(G*R) consecutive query blocks, so that every sampled-key tile fetched once
-// serves all of them.  The sampled logits of 128 rows x 128 sampled keys (= 128/R key blocks)
-// are one tcgen05 MMA tile with a TMEM accumulator; strided TMA boxes gather every s-th row of
-// Q and K directly (the down-sampled matrices are never materialised).
+// One CTA owns 256 sampled query rows = the R sampled rows of each of the G query heads of one
+// KV head for 256/(G*R) consecutive query blocks, so that every sampled-key tile fetched once
+// serves all of them: two row tiles of 128, because with a single one the kernel ran at the
+// speed L2 could deliver key tiles, not at the speed of the tensor pipe.  The sampled logits of
+// 128 rows x 128 sampled keys (= 128/R key blocks) are one tcgen05 MMA tile with a TMEM
+// accumulator; strided TMA boxes gather every s-th row of Q and K directly (the down-sampled
+// matrices are never materialised).
 //
 // The row maximum M*[r] must be known before Pbar[r,j] = exp(M[r,j] - M*[r]) can be summed, and
-// the per-row block maxima of 128 rows do not fit on chip at long context, so the kernel walks
-// the key tiles twice: pass 1 finds, per sampled row, the largest and second largest block
-// maximum and the block holding the largest; pass 2 forms the block scores and HRM flags.
+// the per-row block maxima of 256 rows do not fit on chip at long context.  The contraction is
+// still done once: while the key tiles stream by, every epilogue thread takes its row's block
+// maxima M[r,j] (tracking the three largest and the blocks holding the two largest) and parks
+// them in a scratch area of global memory that the CTA owns while it runs; there are only as
+// many such areas as CTAs can be resident, so they mostly stay in L2.  After the last tile, with
+// M* known, the block scores and HRM flags are formed from the parked maxima, one thread per
+// (row group, key block).
 // Float32 results are a SCREEN: the sort stage recomputes in double precision whatever a
 // rounding error could reorder.  For that it is told, per sampled row, the two blocks with the
 // largest block maxima and whether they are closer than tau_row (the row's HRM flag and M* are
@@ -29,22 +35,31 @@ using namespace ptx;
 constexpr int kStages = 4;
 constexpr int kTileBytes = 128 * kHeadDim * 2;
 constexpr int kHalfBytes = kTileBytes / 2;
-constexpr int kParts = 4;             // column parts of a tile, one epilogue warp per part and sub-partition
+constexpr int kRowTiles = 2;          // 128-row tiles of sampled queries per CTA
+constexpr int kRows = 128 * kRowTiles;
+constexpr int kParts = 2;             // column parts of a tile: one epilogue warp per row tile, part and sub-partition
 constexpr int kPartCols = 128 / kParts;
-constexpr int kThreads = 64 + 128 * kParts;   // producer warp, MMA warp, kParts x 4 epilogue warps
-constexpr int kAccs = 4;              // logit tiles in tensor memory (products run this far ahead of the epilogue)
-constexpr int kTmemCols = 128 * kAccs;
+constexpr int kEpiThreads = 128 * kRowTiles * kParts;
+constexpr int kThreads = 64 + kEpiThreads;    // producer warp, MMA warp, epilogue warps
+constexpr int kSteps = 2;             // key tiles whose logits are in tensor memory at once
+constexpr int kTmemCols = 128 * kRowTiles * kSteps;
+constexpr int kCtasPerSm = 1;
+static_assert(kTmemCols == 512 && kPartCols == 64, "TMEM budget and two 32-column loads per thread and tile");
 
 struct __align__(8) ScreenCtl {
   unsigned long long a_full, k_full[kStages];
   unsigned long long k_empty[kStages];  // the tile's MMAs finished: stage free and logits ready
-  unsigned long long s_empty[kAccs], x_bar;
+  unsigned long long s_empty[kSteps], x_bar;
   uint32_t tmem_base;
   volatile int abort_flag;
-  float xt[kParts][3][128];             // pass-1 exchange between the column parts: top-3 block maxima
-  int xj[kParts][2][128];               // ... and the blocks holding the two largest
+  int slot;                             // scratch area held by this CTA, -1 = none
+  int poisoned;
+  float xt[kParts][3][kRows];           // exchange between the column parts: top-3 block maxima
+  int xj[kParts][2][kRows];             // ... and the blocks holding the two largest
+  float mstar[kRows];                   // M*[r] of every row
 };
-constexpr size_t kScreenSmem = 1024 + (size_t)kTileBytes * (1 + kStages) + sizeof(ScreenCtl);
+constexpr size_t kScreenSmem = 1024 + (size_t)kTileBytes * (kRowTiles + kStages) + sizeof(ScreenCtl);
+static_assert(kScreenSmem <= 232448, "shared memory budget of one CTA");
 
 __device__ __forceinline__ void screen_timeout(ScreenCtl* c, int32_t* status) {
   c->abort_flag = 1;
@@ -52,7 +67,7 @@ __device__ __forceinline__ void screen_timeout(ScreenCtl* c, int32_t* status) {
 }
 
 template <int R>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                   KapScreenParams p, int32_t* status) {
   extern __shared__ unsigned char smem_raw[];
@@ -60,11 +75,13 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* smem = smem_raw + (base - raw);
   const uint32_t a_sm = base;
-  const uint32_t k_sm = base + kTileBytes;
-  ScreenCtl* ctl = reinterpret_cast<ScreenCtl*>(smem + (size_t)kTileBytes * (1 + kStages));
+  const uint32_t k_sm = base + kRowTiles * kTileBytes;
+  ScreenCtl* ctl = reinterpret_cast<ScreenCtl*>(smem + (size_t)kTileBytes * (kRowTiles + kStages));
 
+  constexpr int BPT = 128 / R;                  // key blocks per key tile
+  constexpr int kGroups = kRows / R;            // row groups (one query head of one query block each) per CTA
   const int G = p.hq / p.hkv;
-  const int QB = 128 / (G * R);                 // query blocks per CTA
+  const int QB = kGroups / G;                   // query blocks per CTA
   const int n_iq = (p.nqb + QB - 1) / QB;
   const int w = blockIdx.x;
   const int b = w / (p.hkv * n_iq);
@@ -77,17 +94,34 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   const int n_tiles = (n_keys + 127) / 128;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  __shared__ int s_poisoned;
-  if (threadIdx.x == 0) s_poisoned = *reinterpret_cast<volatile int32_t*>(status);
+  if (threadIdx.x == 0) {
+    // once some CTA has reported a timeout the rest of the grid returns at once
+    int poisoned = *reinterpret_cast<volatile int32_t*>(status);
+    int slot = -1;
+    if (poisoned == 0) {
+      // a scratch area no resident CTA holds: there are as many as CTAs can be resident, so one is free; the
+      // search starts at this SM's number and normally ends at once
+      unsigned smid;
+      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+      for (int s = 0; s < 8 * p.slots && slot < 0; ++s) {
+        const int cand = (int)((smid * kCtasPerSm + s) % (unsigned)p.slots);
+        if (atomicCAS(&p.slot_taken[cand], 0, 1) == 0) slot = cand;
+      }
+      if (slot < 0) { atomicMin(status, (int32_t)COSA_ERR_DEVICE_TIMEOUT); poisoned = 1; }
+      __threadfence();
+    }
+    ctl->slot = slot;
+    ctl->poisoned = poisoned;
+  }
   __syncthreads();
-  if (s_poisoned != 0) return;
+  if (ctl->poisoned != 0) return;
 
   if (threadIdx.x == 0) {
     if (blockIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
     mbar_init(smem_u32(&ctl->a_full), 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
-    for (int s = 0; s < kAccs; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), 128 * kParts);
-    mbar_init(smem_u32(&ctl->x_bar), 128 * kParts);
+    for (int s = 0; s < kSteps; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), kEpiThreads);
+    mbar_init(smem_u32(&ctl->x_bar), kEpiThreads);
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -102,26 +136,27 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
 
   if (warp == 0) {
     if (lane == 0) {
-      // A tile: one strided box of R sampled rows per (query block, query head of the group)
-      mbar_expect_tx(smem_u32(&ctl->a_full), kTileBytes);
-      for (int grp = 0; grp < QB * G; ++grp) {
+      // A tiles: one strided box of R sampled rows per (query block, query head of the group)
+      mbar_expect_tx(smem_u32(&ctl->a_full), kRowTiles * kTileBytes);
+      for (int grp = 0; grp < kGroups; ++grp) {
         const int i = i0 + grp / G, h = g * G + grp % G;
         const int row = (b * p.hq + h) * ns + i * R;   // rows past the tensor are zero-filled
-        tma_load_2d(a_sm + grp * R * 128, &q_map, 0, row, smem_u32(&ctl->a_full));
-        tma_load_2d(a_sm + kHalfBytes + grp * R * 128, &q_map, 64, row, smem_u32(&ctl->a_full));
+        const uint32_t dst = a_sm + (grp * R / 128) * kTileBytes + (grp * R % 128) * 128;
+        tma_load_2d(dst, &q_map, 0, row, smem_u32(&ctl->a_full));
+        tma_load_2d(dst + kHalfBytes, &q_map, 64, row, smem_u32(&ctl->a_full));
       }
       if (!p.pg.table) {
         const int krow0 = (b * p.hkv + g) * ns;
-        for (int t = 0; t < 2 * n_tiles; ++t) {
-          const int st = t % kStages, jt = t % n_tiles;
+        for (int t = 0; t < n_tiles; ++t) {
+          const int st = t % kStages;
           if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag)) {
             if (!*abort_flag) screen_timeout(ctl, status);
             break;
           }
           const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
           mbar_expect_tx(bar, kTileBytes);
-          tma_load_2d(dst, &k_map, 0, krow0 + jt * 128, bar);
-          tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + jt * 128, bar);
+          tma_load_2d(dst, &k_map, 0, krow0 + t * 128, bar);
+          tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + t * 128, bar);
         }
       }
     }
@@ -131,8 +166,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       // later: any valid page will do for them.
       const int spp = min(128, p.pg.page_size / p.stride);
       const int parts = 128 / spp;
-      for (int t = 0; t < 2 * n_tiles; ++t) {
-        const int st = t % kStages, jt = t % n_tiles;
+      for (int t = 0; t < n_tiles; ++t) {
+        const int st = t % kStages;
         const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
         int ok = 1;
         if (lane == 0) {
@@ -143,7 +178,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
         if (lane < parts) {
-          int tok = (jt * 128 + lane * spp) * p.stride;
+          int tok = (t * 128 + lane * spp) * p.stride;
           if (tok >= p.n) tok = 0;
           const int srow = (int)(kv_row(p.pg, b, p.hkv, g, p.n, tok) / p.stride);
           tma_load_2d(dst + lane * spp * 128, &k_map, 0, srow, bar);
@@ -157,67 +192,121 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       const uint32_t idesc = idesc_bf16(128, 128, 0, 0);
       bool alive = mbar_wait(smem_u32(&ctl->a_full), 0, abort_flag);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
-      for (int t = 0; t < 2 * n_tiles && alive; ++t) {
-        const int st = t % kStages, sb = t % kAccs;
+      for (int t = 0; t < n_tiles && alive; ++t) {
+        const int st = t % kStages, sb = t % kSteps;
         alive = mbar_wait(smem_u32(&ctl->k_full[st]), (t / kStages) & 1, abort_flag) &&
-                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t / kAccs) & 1) ^ 1, abort_flag);
+                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t / kSteps) & 1) ^ 1, abort_flag);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         tc_fence_after();
-        const uint32_t kt = k_sm + st * kTileBytes;
-        mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
-            tmem + sb * 128, smem_desc_sw128(a_sm, 16, 1024), smem_desc_sw128(kt, 16, 1024), idesc);
+        const uint64_t kdesc = smem_desc_sw128(k_sm + st * kTileBytes, 16, 1024);
+#pragma unroll
+        for (int rt = 0; rt < kRowTiles; ++rt)
+          mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+              tmem + (sb * kRowTiles + rt) * 128, smem_desc_sw128(a_sm + rt * kTileBytes, 16, 1024), kdesc, idesc);
         mma_commit(smem_u32(&ctl->k_empty[st]));
       }
     }
   } else {
     // ---------------------------------------------------------------- kParts threads per sampled query row
-    // (one per column part of every tile: kParts epilogue warps per SM sub-partition overlap their latencies)
-    const int sub = warp & 3;
-    const int half = (warp - 2) >> 2;        // column part
-    const int row = sub * 32 + lane;
+    const int ew = warp - 2;
+    const int sub = warp & 3;                // the TMEM lanes a warp may read: 32 * (warp % 4)
+    const int rt = (ew >> 2) % kRowTiles;    // row tile
+    const int part = ew / (4 * kRowTiles);   // column part
+    const int row = rt * 128 + sub * 32 + lane;
     const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
     const int grp = row / R, r = row % R;
     const int i = i0 + grp / G, h = g * G + grp % G;
     const bool row_ok = i < p.nqb;
     const int r_glob = i * R + r;                        // index among the head's sampled rows
     const int c_limit = p.causal ? r_glob : ns - 1;      // last sampled key this row may see
-    const int J = p.causal ? i + 1 : p.nqb;
-    constexpr int BPC = 32 / R;                          // key blocks per 32-column chunk
+    constexpr int BPC = kPartCols / R;                   // key blocks per column part
     float top1 = -INFINITY, top2 = -INFINITY, top3 = -INFINITY;
     int jstar = 0, jstar2 = 0;
-    const float kLog2e = 1.4426950408889634f;
-    const float scale2 = p.scale * kLog2e;
-    float* srow = p.scores + ((size_t)(b * p.hq + h) * p.nqb + (row_ok ? i : 0)) * p.nqb;
+    // the CTA's block maxima: [tile][row][block of the tile]
+    constexpr int kTileFloats = kRows * BPT;
+    float* parked = p.maxima + (size_t)ctl->slot * ((size_t)((ns + 127) / 128) * kTileFloats);
+    float* mine = parked + (size_t)row * BPT + part * BPC;
+    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
     bool alive = true;
-    for (int t = 0; t < 2 * n_tiles && alive; ++t) {
-      const int sb = t % kAccs, jt = t % n_tiles, st = t % kStages;
-      const bool pass2 = t >= n_tiles;
-      if (t == n_tiles) {
-        // end of pass 1: merge the two halves' top-3 block maxima of every row
-        ctl->xt[half][0][row] = top1; ctl->xt[half][1][row] = top2; ctl->xt[half][2][row] = top3;
-        ctl->xj[half][0][row] = jstar; ctl->xj[half][1][row] = jstar2;
-        mbar_arrive(smem_u32(&ctl->x_bar));
-        alive = mbar_wait(smem_u32(&ctl->x_bar), 0, abort_flag);
-        if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
+    for (int t = 0; t < n_tiles && alive; ++t) {
+      const int sb = t % kSteps, st = t % kStages;
+      alive = mbar_wait(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag);   // this tile's MMAs finished
+      if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
+      tc_fence_after();
+      uint32_t v[kPartCols / 32][32];
 #pragma unroll
-        for (int other = 1; other < kParts; ++other) {
-          const int op = (half + other) % kParts;
+      for (int c2 = 0; c2 < kPartCols / 32; ++c2)
+        tmem_ld32(tmem + (sb * kRowTiles + rt) * 128 + lane_addr + part * kPartCols + c2 * 32, v[c2]);
+      tmem_wait_ld();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->s_empty[sb]));
+      float mb[BPC];
 #pragma unroll
-          for (int q = 0; q < 3; ++q) {
-            const float m = ctl->xt[op][q][row];
-            const int jb = q < 2 ? ctl->xj[op][q][row] : 0;
-            if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
-            else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
-            else if (m > top3) top3 = m;
+      for (int bb = 0; bb < BPC; ++bb) {
+        const int c0 = bb * R;                              // first column of the block within the part
+        const int cabs = t * 128 + part * kPartCols + c0;   // ... and among the head's sampled keys
+        float m0 = -INFINITY, m1 = -INFINITY;
+        if (cabs + R - 1 <= c_limit) {                      // whole block visible: no masking
+#pragma unroll
+          for (int e = 0; e < R; e += 2) {
+            m0 = fmaxf(m0, __uint_as_float(v[(c0 + e) / 32][(c0 + e) % 32]));
+            m1 = fmaxf(m1, __uint_as_float(v[(c0 + e + 1) / 32][(c0 + e + 1) % 32]));
           }
+        } else {
+#pragma unroll
+          for (int e = 0; e < R; ++e)
+            if (cabs + e <= c_limit) m0 = fmaxf(m0, __uint_as_float(v[(c0 + e) / 32][(c0 + e) % 32]));
         }
-        // the row's best block, and whether the runner-up is too close to call
-        const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
-        const bool amb3 = row_ok && (top1 - top3) * p.scale <= p.tau_row;
-        const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);
-        const int shift = (lane / R) * R;
-        const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << shift);
-        if (row_ok && half == 0) {
+        mb[bb] = fmaxf(m0, m1);
+      }
+      float* dst = mine + (size_t)t * kTileFloats;
+      if (BPC == 8) {
+        st_l2_hint(reinterpret_cast<float4*>(dst), make_float4(mb[0], mb[1 % BPC], mb[2 % BPC], mb[3 % BPC]), keep);
+        st_l2_hint(reinterpret_cast<float4*>(dst) + 1, make_float4(mb[4 % BPC], mb[5 % BPC], mb[6 % BPC], mb[7 % BPC]), keep);
+      } else if (BPC == 4) {
+        st_l2_hint(reinterpret_cast<float4*>(dst), make_float4(mb[0], mb[1 % BPC], mb[2 % BPC], mb[3 % BPC]), keep);
+      } else {
+        st_l2_hint(reinterpret_cast<float2*>(dst), make_float2(mb[0], mb[1 % BPC]), keep);
+      }
+#pragma unroll
+      for (int bb = 0; bb < BPC; ++bb) {
+        const float m = mb[bb];
+        const int jb = t * BPT + part * BPC + bb;
+        if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
+        else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
+        else if (m > top3) top3 = m;
+      }
+    }
+    if (alive) {
+      // all tiles seen: merge the column parts' top-3 block maxima of every row
+      ctl->xt[part][0][row] = top1; ctl->xt[part][1][row] = top2; ctl->xt[part][2][row] = top3;
+      ctl->xj[part][0][row] = jstar; ctl->xj[part][1][row] = jstar2;
+      mbar_arrive(smem_u32(&ctl->x_bar));
+      alive = mbar_wait(smem_u32(&ctl->x_bar), 0, abort_flag);
+      if (!alive && !*abort_flag) screen_timeout(ctl, status);
+    }
+    if (alive) {
+#pragma unroll
+      for (int other = 1; other < kParts; ++other) {
+        const int op = (part + other) % kParts;
+#pragma unroll
+        for (int q = 0; q < 3; ++q) {
+          const float m = ctl->xt[op][q][row];
+          const int jb = q < 2 ? ctl->xj[op][q][row] : 0;
+          if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
+          else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
+          else if (m > top3) top3 = m;
+        }
+      }
+      // the row's best block, and whether the runner-up is too close to call
+      const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
+      const bool amb3 = row_ok && (top1 - top3) * p.scale <= p.tau_row;
+      const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);
+      const int shift = (lane / R) * R;
+      const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << shift);
+      if (part == 0) {
+        ctl->mstar[row] = top1;
+        if (row_ok) {
           int2 js = make_int2(jstar, jstar2);
           reinterpret_cast<int2*>(p.jstar)[(size_t)(b * p.hq + h) * ns + r_glob] = js;
           if (r == 0) {
@@ -226,59 +315,60 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           }
         }
       }
-      alive = mbar_wait(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag);   // this tile's MMAs finished
-      if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
-      tc_fence_after();
-      const int col0 = jt * 128 + half * kPartCols;
-      uint32_t v[kPartCols / 32][32];
+      // every row's M* in shared memory and every parked maximum visible to the whole CTA
+      __threadfence_block();
+      mbar_arrive(smem_u32(&ctl->x_bar));
+      alive = mbar_wait(smem_u32(&ctl->x_bar), 1, abort_flag);
+      if (!alive && !*abort_flag) screen_timeout(ctl, status);
+    }
+    if (alive) {
+      // block scores s_ij = sum over the group's rows of exp(M[r,j] - M*[r]) and HRM flags: one thread per
+      // (row group, key block of a tile), several tiles per sweep of the CTA's threads
+      constexpr int kOutsPerTile = kGroups * BPT;
+      static_assert(kEpiThreads % kOutsPerTile == 0, "whole tiles per sweep");
+      constexpr int kTilesPerSweep = kEpiThreads / kOutsPerTile;
+      const int et = threadIdx.x - 64;
+      const int o = et % kOutsPerTile;
+      const int blk = o % BPT, og = o / BPT;               // consecutive lanes: consecutive key blocks
+      const int oi = i0 + og / G, oh = g * G + og % G;
+      const int J = p.causal ? oi + 1 : p.nqb;
+      const float kLog2e = 1.4426950408889634f;
+      const float scale2 = p.scale * kLog2e;
+      float ms[R];
 #pragma unroll
-      for (int c2 = 0; c2 < kPartCols / 32; ++c2) tmem_ld32(tmem + sb * 128 + lane_addr + half * kPartCols + c2 * 32, v[c2]);
-      tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->s_empty[sb]));
+      for (int rr = 0; rr < R; ++rr) ms[rr] = ctl->mstar[og * R + rr];
+      if (oi < p.nqb) {
+        float* srow = p.scores + ((size_t)(b * p.hq + oh) * p.nqb + oi) * p.nqb;
+        const float* src0 = parked + (size_t)og * R * BPT + blk;
+        // last tile with a candidate block for this thread; the maxima of the next tile are fetched while the
+        // current one is summed
+        const int t_end = J > blk ? min(n_tiles, (J - 1 - blk) / BPT + 1) : 0;
+        int t = et / kOutsPerTile;
+        float x[R];
+        if (t < t_end) {
 #pragma unroll
-      for (int c2 = 0; c2 < kPartCols / 32; ++c2) {
-        const int cbase = col0 + c2 * 32;
-        float mb[BPC];
-#pragma unroll
-        for (int bb = 0; bb < BPC; ++bb) {
-          float m0 = -INFINITY, m1 = -INFINITY;
-          if (cbase + bb * R + R - 1 <= c_limit) {        // whole block visible: no masking
-#pragma unroll
-            for (int e = 0; e < R; e += 2) {
-              m0 = fmaxf(m0, __uint_as_float(v[c2][bb * R + e]));
-              m1 = fmaxf(m1, __uint_as_float(v[c2][bb * R + e + 1]));
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < R; ++e)
-              if (cbase + bb * R + e <= c_limit) m0 = fmaxf(m0, __uint_as_float(v[c2][bb * R + e]));
-          }
-          mb[bb] = fmaxf(m0, m1);
+          for (int rr = 0; rr < R; ++rr) x[rr] = ld_l2_hint(src0 + (size_t)t * kTileFloats + rr * BPT, drop);
         }
-        if (!pass2) {
+        while (t < t_end) {
+          const int tn = t + kTilesPerSweep;
+          float xn[R];
+          if (tn < t_end) {
 #pragma unroll
-          for (int bb = 0; bb < BPC; ++bb) {
-            const float m = mb[bb];
-            const int jb = cbase / R + bb;
-            if (m > top1) { top3 = top2; top2 = top1; jstar2 = jstar; top1 = m; jstar = jb; }
-            else if (m > top2) { top3 = top2; top2 = m; jstar2 = jb; }
-            else if (m > top3) top3 = m;
+            for (int rr = 0; rr < R; ++rr) xn[rr] = ld_l2_hint(src0 + (size_t)tn * kTileFloats + rr * BPT, drop);
           }
-        } else {
+          float e0 = 0.f, e1 = 0.f;
+          bool fl = false;
 #pragma unroll
-          for (int bb = 0; bb < BPC; ++bb) {
-            float e = ex2_approx((mb[bb] - top1) * scale2);   // exp(M[r,j] - M*[r]); 0 for invisible blocks
-            unsigned f = (mb[bb] == top1) ? 1u : 0u;
-            if (!row_ok) { e = 0.f; f = 0u; }
-#pragma unroll
-            for (int o = R / 2; o > 0; o >>= 1) {
-              e += __shfl_xor_sync(0xffffffffu, e, o);
-              f |= __shfl_xor_sync(0xffffffffu, f, o);
-            }
-            const int j = cbase / R + bb;
-            if (r == 0 && row_ok && j < J) srow[j] = f ? -e : e;   // sign bit carries the HRM flag
+          for (int rr = 0; rr < R; rr += 2) {
+            e0 += ex2_approx((x[rr] - ms[rr]) * scale2);       // exp(M[r,j] - M*[r]); 0 for invisible blocks
+            e1 += ex2_approx((x[rr + 1] - ms[rr + 1]) * scale2);
+            fl = fl || x[rr] == ms[rr] || x[rr + 1] == ms[rr + 1];
           }
+          const float e = e0 + e1;
+          srow[t * BPT + blk] = fl ? -e : e;                   // sign bit carries the HRM flag
+#pragma unroll
+          for (int rr = 0; rr < R; ++rr) x[rr] = xn[rr];
+          t = tn;
         }
       }
     }
@@ -286,6 +376,18 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+  {
+    // the parked maxima are dead: let L2 drop the lines instead of writing them back
+    char* area = reinterpret_cast<char*>(p.maxima + (size_t)ctl->slot * ((size_t)((ns + 127) / 128) * (kRows * BPT)));
+    const size_t bytes = (size_t)n_tiles * (kRows * BPT) * sizeof(float);
+    for (size_t off = (size_t)threadIdx.x * 128; off < bytes; off += (size_t)kThreads * 128)
+      asm volatile("discard.global.L2 [%0], 128;" ::"l"(area + off) : "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicExch(&p.slot_taken[ctl->slot], 0);
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -320,13 +422,34 @@ bool make_strided_map(CUtensorMap* map, const void* basep, uint64_t sampled_rows
 }  // namespace
 
 bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg) {
-  if (!((rows == 8 || rows == 16 || rows == 32) && group * rows <= 128 && 128 % (group * rows) == 0)) return false;
+  if (!((rows == 8 || rows == 16 || rows == 32) && group * rows <= kRows && kRows % (group * rows) == 0)) return false;
   // paged keys: a page must hold at least 8 sampled rows (boxes land on 1024-byte boundaries of the swizzled tile)
   return !pg.table || pg.page_size / stride >= 8;
 }
 
+int kap_screen_grid(int batch, int hq, int hkv, int nqb, int stride) {
+  const int QB = kRows / ((hq / hkv) * (128 / stride));
+  return batch * hkv * ((nqb + QB - 1) / QB);
+}
+
+int kap_screen_slots() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return 0;
+  return sms * kCtasPerSm;
+}
+
+size_t kap_screen_slot_bytes(int n, int stride) {
+  const size_t ns = (size_t)n / stride, R = 128 / stride;
+  return ((ns + 127) / 128) * kRows * (128 / R) * sizeof(float);
+}
+
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st) {
-  const int R = 128 / p.stride, G = p.hq / p.hkv;
+  const int R = 128 / p.stride;
+  if (!p.maxima || !p.slot_taken || p.slots <= 0) return cudaErrorInvalidValue;
+  cudaError_t e0 = cudaMemsetAsync(p.slot_taken, 0, (size_t)p.slots * sizeof(int32_t), st);
+  if (e0 != cudaSuccess) return e0;
   const uint64_t ns = (uint64_t)p.n / p.stride;
   CUtensorMap qm, km;
   const uint64_t k_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * (p.pg.page_size / p.stride) : (uint64_t)p.batch * p.hkv * ns;
@@ -336,8 +459,7 @@ cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st) {
     return cudaErrorInvalidValue;
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;
-  const int QB = 128 / (G * R);
-  const int grid = p.batch * p.hkv * ((p.nqb + QB - 1) / QB);
+  const int grid = kap_screen_grid(p.batch, p.hq, p.hkv, p.nqb, p.stride);
   cudaError_t e;
 #define COSA_LAUNCH_SCREEN(RR)                                                                                    \
   e = cudaFuncSetAttribute(kap_screen_kernel<RR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScreenSmem); \

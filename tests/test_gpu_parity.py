@@ -253,6 +253,63 @@ def test_kap_lists_bit_exact_4k(cfg1, impl):
     assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
 
 
+@pytest.fixture(scope="module")
+def mid():
+    w = tiny(seed=33, hq=4, hkv=2, n=16384, needles=6)
+    qb, kb, vb, _ = w.make()
+    return dict(w=w, dev=tuple(to_dev(x) for x in (qb, kb, vb)), f64=widen(qb, kb, vb))
+
+
+MID_BLOCKS = [0, 1, 63, 64, 71, 72, 89, 90, 100, 117, 126, 127]
+
+
+@pytest.mark.parametrize("budget", [0.05, 0.1, 0.25, 0.6])
+def test_kap_16k_head_of_the_order(mid, budget):
+    """At 128 key blocks and a small budget the fast path selects and sorts only the head of the order (kept prefix
+    plus a margin); larger budgets and short candidate lists sort everything.  Both must give the oracle's lists."""
+    q, k, _ = mid["dev"]
+    qf, kf, _ = mid["f64"]
+    order, count = run_kap(q, k, budget, 8)
+    ref_order, ref_count = O.kap_select(qf, kf, s=8, budget=budget, order_stride=order.shape[-1], query_blocks=MID_BLOCKS)
+    for i in MID_BLOCKS:
+        assert np.array_equal(_np(count)[:, i], ref_count[:, i]), i
+        assert np.array_equal(_np(order)[:, i], ref_order[:, i]), i
+
+
+def test_kap_16k_tie_chain_longer_than_the_margin(mid):
+    """Forty identical key blocks score exactly alike: a chain of near ties far longer than the margin kept beyond the
+    prefix, which the head selection must hand over to the full sort, and whose members the double-precision
+    recount must put in ascending-id order."""
+    q, k, _ = mid["dev"]
+    qf, kf, _ = mid["f64"]
+    k2, kf2 = k.clone(), kf.copy()
+    for dst in range(21, 61):
+        k2[0, :, dst * 128:(dst + 1) * 128] = k2[0, :, 20 * 128:21 * 128]
+        kf2[:, dst * 128:(dst + 1) * 128] = kf2[:, 20 * 128:21 * 128]
+    blocks = [64, 90, 110, 127]
+    for budget in (0.1, 0.3):
+        order, count = run_kap(q, k2, budget, 8)
+        ref_order, ref_count = O.kap_select(qf, kf2, s=8, budget=budget, order_stride=order.shape[-1], query_blocks=blocks)
+        for i in blocks:
+            assert np.array_equal(_np(count)[:, i], ref_count[:, i]), (budget, i)
+            assert np.array_equal(_np(order)[:, i], ref_order[:, i]), (budget, i)
+
+
+@pytest.mark.parametrize("stride", [4, 8, 16])
+@pytest.mark.parametrize("hq,hkv", [(8, 1), (16, 2), (2, 2)])
+def test_kap_query_group_sizes(hq, hkv, stride):
+    """Query groups of 8 and 1 heads per KV head (the screen's CTA holds 256 sampled rows however they split
+    into heads and query blocks); combinations the screen does not take fall to the double-precision kernel."""
+    w = tiny(seed=41, hq=hq, hkv=hkv, n=2048, needles=2)
+    qb, kb, vb, _ = w.make()
+    q, k = to_dev(qb), to_dev(kb)
+    qf, kf, _ = widen(qb, kb, vb)
+    order, count = run_kap(q, k, 0.4, stride)
+    ref_order, ref_count = O.kap_select(qf, kf, s=stride, budget=0.4, order_stride=order.shape[-1])
+    assert np.array_equal(_np(count), ref_count)
+    assert np.array_equal(_np(order), ref_order)
+
+
 # ---------------------------------------------------------------------------------- OSK
 @pytest.mark.parametrize("impl", IMPLS)
 def test_osk_dense_path_matches_dense_attention(small, impl):
