@@ -50,6 +50,7 @@ struct __align__(8) ScreenCtl {
   unsigned long long a_full, k_full[kStages];
   unsigned long long k_empty[kStages];  // the tile's MMAs finished: stage free and logits ready
   unsigned long long s_empty[kSteps], x_bar;
+  unsigned long long m_full[kStages], m_empty[kStages];   // parked maxima fetched back into a key stage / read by all
   uint32_t tmem_base;
   volatile int abort_flag;
   int slot;                             // scratch area held by this CTA, -1 = none
@@ -122,6 +123,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < kSteps; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), kEpiThreads);
     mbar_init(smem_u32(&ctl->x_bar), kEpiThreads);
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->m_full[s]), 1); mbar_init(smem_u32(&ctl->m_empty[s]), kEpiThreads); }
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -222,10 +224,11 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     constexpr int BPC = kPartCols / R;                   // key blocks per column part
     float top1 = -INFINITY, top2 = -INFINITY, top3 = -INFINITY;
     int jstar = 0, jstar2 = 0;
-    // the CTA's block maxima: [tile][row][block of the tile]
+    // the CTA's block maxima: [tile][row group][block of the tile][row of the group], so that the R maxima one
+    // score needs are contiguous
     constexpr int kTileFloats = kRows * BPT;
     float* parked = p.maxima + (size_t)ctl->slot * ((size_t)((ns + 127) / 128) * kTileFloats);
-    float* mine = parked + (size_t)row * BPT + part * BPC;
+    float* mine = parked + ((size_t)grp * BPT + part * BPC) * R + r;
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
     bool alive = true;
     for (int t = 0; t < n_tiles && alive; ++t) {
@@ -260,14 +263,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         mb[bb] = fmaxf(m0, m1);
       }
       float* dst = mine + (size_t)t * kTileFloats;
-      if (BPC == 8) {
-        st_l2_hint(reinterpret_cast<float4*>(dst), make_float4(mb[0], mb[1 % BPC], mb[2 % BPC], mb[3 % BPC]), keep);
-        st_l2_hint(reinterpret_cast<float4*>(dst) + 1, make_float4(mb[4 % BPC], mb[5 % BPC], mb[6 % BPC], mb[7 % BPC]), keep);
-      } else if (BPC == 4) {
-        st_l2_hint(reinterpret_cast<float4*>(dst), make_float4(mb[0], mb[1 % BPC], mb[2 % BPC], mb[3 % BPC]), keep);
-      } else {
-        st_l2_hint(reinterpret_cast<float2*>(dst), make_float2(mb[0], mb[1 % BPC]), keep);
-      }
+#pragma unroll
+      for (int bb = 0; bb < BPC; ++bb) st_l2_hint(dst + bb * R, mb[bb], keep);
 #pragma unroll
       for (int bb = 0; bb < BPC; ++bb) {
         const float m = mb[bb];
@@ -322,54 +319,80 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
     }
     if (alive) {
-      // block scores s_ij = sum over the group's rows of exp(M[r,j] - M*[r]) and HRM flags: one thread per
-      // (row group, key block of a tile), several tiles per sweep of the CTA's threads
+      // block scores s_ij = sum over the group's rows of exp(M[r,j] - M*[r]) and HRM flags.  The parked maxima
+      // come back through the key stages, which are idle by now: bulk copies of a stage's worth of tiles, several
+      // in flight (the fetch is a matter of latency, and no thread could hold that many bytes in registers); one
+      // thread per (tile, row group, key block) then reads its R maxima from shared memory.
       constexpr int kOutsPerTile = kGroups * BPT;
-      static_assert(kEpiThreads % kOutsPerTile == 0, "whole tiles per sweep");
-      constexpr int kTilesPerSweep = kEpiThreads / kOutsPerTile;
+      constexpr int kTileBytesM = kTileFloats * 4;
+      constexpr int kTilesPerChunk = kTileBytes / kTileBytesM;
+      static_assert(kTilesPerChunk >= 1 && kTileBytes % kTileBytesM == 0, "a stage holds whole tiles of maxima");
       const int et = threadIdx.x - 64;
-      const int o = et % kOutsPerTile;
-      const int blk = o % BPT, og = o / BPT;               // consecutive lanes: consecutive key blocks
+      const int n_chunks = (n_tiles + kTilesPerChunk - 1) / kTilesPerChunk;
+      auto fetch = [&](int c) {   // thread et == 0 only
+        const int tiles_here = min(kTilesPerChunk, n_tiles - c * kTilesPerChunk);
+        const uint32_t bar = smem_u32(&ctl->m_full[c % kStages]);
+        mbar_expect_tx(bar, tiles_here * kTileBytesM);
+        bulk_load_hint(k_sm + (c % kStages) * kTileBytes, parked + (size_t)c * kTilesPerChunk * kTileFloats,
+                       tiles_here * kTileBytesM, bar, drop);
+      };
+      if (et == 0) {
+        fence_proxy_async_all();   // the maxima were written with ordinary stores
+        for (int c = 0; c < min(n_chunks, kStages - 1); ++c) fetch(c);
+      }
+      const int oo = et % kOutsPerTile;
+      const int blk = oo % BPT, og = oo / BPT;             // consecutive lanes: consecutive key blocks
       const int oi = i0 + og / G, oh = g * G + og % G;
       const int J = p.causal ? oi + 1 : p.nqb;
       const float kLog2e = 1.4426950408889634f;
       const float scale2 = p.scale * kLog2e;
+      // a thread reads its R maxima as R/4 vectors, starting at a vector that depends on the lane so that the
+      // lanes of a quarter warp hit different banks; M* is taken in the same rotated order
+      constexpr int kVecs = R / 4;
+      const int rot = (lane / (8 / kVecs > 0 ? 8 / kVecs : 1)) % kVecs;
       float ms[R];
 #pragma unroll
-      for (int rr = 0; rr < R; ++rr) ms[rr] = ctl->mstar[og * R + rr];
-      if (oi < p.nqb) {
-        float* srow = p.scores + ((size_t)(b * p.hq + oh) * p.nqb + oi) * p.nqb;
-        const float* src0 = parked + (size_t)og * R * BPT + blk;
-        // last tile with a candidate block for this thread; the maxima of the next tile are fetched while the
-        // current one is summed
-        const int t_end = J > blk ? min(n_tiles, (J - 1 - blk) / BPT + 1) : 0;
-        int t = et / kOutsPerTile;
-        float x[R];
-        if (t < t_end) {
+      for (int v4 = 0; v4 < kVecs; ++v4) {
+        const int src = ((v4 + rot) % kVecs) * 4;
 #pragma unroll
-          for (int rr = 0; rr < R; ++rr) x[rr] = ld_l2_hint(src0 + (size_t)t * kTileFloats + rr * BPT, drop);
-        }
-        while (t < t_end) {
-          const int tn = t + kTilesPerSweep;
-          float xn[R];
-          if (tn < t_end) {
-#pragma unroll
-            for (int rr = 0; rr < R; ++rr) xn[rr] = ld_l2_hint(src0 + (size_t)tn * kTileFloats + rr * BPT, drop);
+        for (int q = 0; q < 4; ++q) ms[v4 * 4 + q] = ctl->mstar[og * R + src + q];
+      }
+      float* srow = p.scores + ((size_t)(b * p.hq + oh) * p.nqb + min(oi, p.nqb - 1)) * p.nqb;
+      for (int c = 0; c < n_chunks && alive; ++c) {
+        const int st = c % kStages;
+        if (et == 0 && c + kStages - 1 < n_chunks) {
+          // the stage of chunk c - 1 takes chunk c + kStages - 1 once every thread has read it
+          if (c > 0 && !mbar_wait(smem_u32(&ctl->m_empty[(c - 1) % kStages]), ((c - 1) / kStages) & 1, abort_flag)) {
+            if (!*abort_flag) screen_timeout(ctl, status);
+          } else {
+            fetch(c + kStages - 1);
           }
-          float e0 = 0.f, e1 = 0.f;
-          bool fl = false;
-#pragma unroll
-          for (int rr = 0; rr < R; rr += 2) {
-            e0 += ex2_approx((x[rr] - ms[rr]) * scale2);       // exp(M[r,j] - M*[r]); 0 for invisible blocks
-            e1 += ex2_approx((x[rr + 1] - ms[rr + 1]) * scale2);
-            fl = fl || x[rr] == ms[rr] || x[rr + 1] == ms[rr + 1];
-          }
-          const float e = e0 + e1;
-          srow[t * BPT + blk] = fl ? -e : e;                   // sign bit carries the HRM flag
-#pragma unroll
-          for (int rr = 0; rr < R; ++rr) x[rr] = xn[rr];
-          t = tn;
         }
+        alive = mbar_wait(smem_u32(&ctl->m_full[st]), (c / kStages) & 1, abort_flag);
+        if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
+        const int tiles_here = min(kTilesPerChunk, n_tiles - c * kTilesPerChunk);
+        const float* stage = reinterpret_cast<const float*>(smem + (size_t)kTileBytes * (kRowTiles + st));
+        for (int o = et; o < tiles_here * kOutsPerTile; o += kEpiThreads) {
+          const int tl = o / kOutsPerTile;
+          const int j = (c * kTilesPerChunk + tl) * BPT + blk;
+          if (oi < p.nqb && j < J) {
+            const float4* src = reinterpret_cast<const float4*>(stage + (size_t)tl * kTileFloats + ((size_t)og * BPT + blk) * R);
+            float e0 = 0.f, e1 = 0.f;
+            bool fl = false;
+#pragma unroll
+            for (int v4 = 0; v4 < kVecs; ++v4) {
+              const float4 x = src[(v4 + rot) % kVecs];
+              e0 += ex2_approx((x.x - ms[v4 * 4]) * scale2);       // exp(M[r,j] - M*[r]); 0 for invisible blocks
+              e1 += ex2_approx((x.y - ms[v4 * 4 + 1]) * scale2);
+              e0 += ex2_approx((x.z - ms[v4 * 4 + 2]) * scale2);
+              e1 += ex2_approx((x.w - ms[v4 * 4 + 3]) * scale2);
+              fl = fl || x.x == ms[v4 * 4] || x.y == ms[v4 * 4 + 1] || x.z == ms[v4 * 4 + 2] || x.w == ms[v4 * 4 + 3];
+            }
+            const float e = e0 + e1;
+            srow[j] = fl ? -e : e;                                 // sign bit carries the HRM flag
+          }
+        }
+        mbar_arrive(smem_u32(&ctl->m_empty[st]));
       }
     }
   }

@@ -71,6 +71,16 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// contiguous global bytes -> shared memory (both 16-byte aligned, size a multiple of 16), with an L2 eviction policy
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+      : "memory");
+}
+// orders this thread's view of earlier generic-proxy writes (its own, and those it has synchronised with) before
+// its later async-proxy operations
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 // shared memory tile -> global (tile store); completion is tracked by bulk async-groups
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(reinterpret_cast<uint64_t>(map)),
@@ -177,6 +187,14 @@ __device__ __forceinline__ void st_l2_hint(float4* ptr, float4 a, uint64_t pol) 
   asm volatile("st.global.L1::no_allocate.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(ptr), "f"(a.x), "f"(a.y),
                "f"(a.z), "f"(a.w), "l"(pol)
                : "memory");
+}
+__device__ __forceinline__ float4 ld_l2_hint(const float4* ptr, uint64_t pol) {
+  float4 a;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(a.x), "=f"(a.y), "=f"(a.z), "=f"(a.w)
+               : "l"(ptr), "l"(pol)
+               : "memory");
+  return a;
 }
 __device__ __forceinline__ float ld_l2_hint(const float* ptr, uint64_t pol) {
   float a;
