@@ -276,12 +276,17 @@ __device__ int select_by_pivot(const unsigned long long* a, int n, int want, uns
     if (lane == 0) cnts[wid * kPivots + k] = wsum;
   }
   __syncthreads();
+  if (tid < kPivots) {
+    int total = 0;
+    for (int w2 = 0; w2 < kThreads / 32; ++w2) total += cnts[w2 * kPivots + tid];
+    cnts[(kThreads / 32) * kPivots + tid] = total;
+  }
+  __syncthreads();
   // counts grow with k (the pivots fall): the first pivot with enough keys at or above it, if those still fit
   int pick = -1, total_pick = 0;
 #pragma unroll
   for (int k = 0; k < kPivots; ++k) {
-    int total = 0;
-    for (int w2 = 0; w2 < kThreads / 32; ++w2) total += cnts[w2 * kPivots + k];
+    const int total = cnts[(kThreads / 32) * kPivots + k];
     if (pick < 0 && total >= want) { pick = k; total_pick = total; }
   }
   if (pick < 0 || total_pick > kHeadCap) return 0;   // (uniform over the CTA)
@@ -393,15 +398,11 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
   const int tid = threadIdx.x;
   const size_t row_lo = (size_t)(b * p.hq + h) * p.nqb + i_lo;
   const size_t row = row_lo + (T - 1);
-  bool hard = false;
+  unsigned hard = 0u;                         // (tested only after the scores have been requested: one round trip, not two)
   unsigned long long amb = 0ULL;              // bit r: sampled row r of the block was too close to call
   for (int t = 0; t < T; ++t) {
-    hard = hard || sp.hard[row_lo + t];
+    hard |= sp.hard[row_lo + t];
     amb |= (unsigned long long)sp.ambmask[row_lo + t] << (t * R);
-  }
-  if (hard) {  // left to the double-precision kernel
-    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
-    return;
   }
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
 
@@ -423,6 +424,10 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
       key = ((unsigned long long)(__float_as_uint(sum) | flag) << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
     }
     keys[j] = key;
+  }
+  if (hard) {  // left to the double-precision kernel
+    if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
+    return;
   }
   if (tid == 0) { n_tied = 0; tail_end = 0; }
   if (tid < RT) {
