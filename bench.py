@@ -327,9 +327,10 @@ def main():
                 "unit": "TFLOP/s", "frac": osk_tflops / tensor_peak, "peak_source": peaks["source"] + " (sustained bf16)",
                 "frac_of_burst": osk_tflops / peaks["bf16_tflops"], "frac_of_nominal_2250": osk_tflops / 2250.0,
                 "traffic": (traffic or {}).get("osk_tc_kernel")}
-    # KAP: the screen kernel forms the sampled logits on the tensor cores (twice: two passes over the key tiles),
-    # the sort kernel is ALU work; the algorithmic FLOPs (one pass, causal pairs only) are set against the tensor
-    # peak, and the algorithmic bytes (sampled rows read once, lists written once) against the copy bandwidth
+    # KAP: the screen kernel forms the sampled logits on the tensor cores (one pass over the key tiles; whole tiles,
+    # so somewhat more than the causal pairs), the sort kernel is ALU work; the algorithmic FLOPs (causal pairs only)
+    # are set against the tensor peak, and the algorithmic bytes (sampled rows read once, lists written once)
+    # against the copy bandwidth
     roof_kap = {"kernel": "kap_screen_kernel+kap_sort_kernel", "bound": "tensor", "achieved": kap_tflops, "peak": tensor_peak,
                 "unit": "TFLOP/s", "frac": kap_tflops / tensor_peak, "peak_source": peaks["source"] + " (sustained bf16)",
                 "hbm_gbs_on_algorithmic_bytes": kap_bytes / (kap_ms * 1e-3) / 1e9,
