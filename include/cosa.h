@@ -82,7 +82,11 @@ typedef struct {
   void*   workspace;       /* device scratch; NULL -> the library's own per-device scratch,
                               which is allocated (cudaMalloc) on first use or growth             */
   size_t  workspace_bytes;
-  int32_t impl;            /* 0 = fastest available; 1 = plain CUDA-core check kernels           */
+  int32_t impl;            /* 0 = fastest available; 1 = plain CUDA-core check kernels; 2 and 3 = as 0,
+                              but the sort stage of cosa_kap_select takes the route it otherwise
+                              keeps for the lists its fastest route cannot settle: 2 = the head of
+                              the order selected by radix, 3 = the whole order sorted (same lists,
+                              slower; for tests and comparisons)                                  */
   float   top_p;           /* KAP only.  > 0: Top-p retention (Sec. 4.2, text after Eq. 13; p = 0.95
                               in Sec. C.1): K_i = length of the shortest prefix of the order whose
                               scores sum to >= top_p * (sum over all candidates), never more than

@@ -181,6 +181,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   p.scale = o.softmax_scale > 0.f ? (double)o.softmax_scale : 1.0 / sqrt((double)shape->d);
   p.top_p = (double)o.top_p;
   p.qtiles = shape->block_q / kBlock;
+  p.sort_mode = o.impl == 2 ? 1 : (o.impl == 3 ? 2 : 0);
   if (p.qtiles == 2 && (o.kap_scores || o.kap_flags)) return COSA_ERR_UNSUPPORTED;   // the exports are per 128-row block
   if (p.qtiles == 2 && p.rows * 2 > 64) return COSA_ERR_UNSUPPORTED;                  // stride 2 and below
   rc = resolve_paging(shape, o, s, &p.pg);

@@ -46,6 +46,7 @@ struct KapParams {
   double scale;          // softmax scale applied to the sampled logits
   double top_p;          // > 0: Top-p retention, capped by the budget count; 0: budget count alone
   int qtiles;            // 1, or 2: one ranking per query block of 2 x 128 rows, shared by its two row tiles
+  int sort_mode;         // sort stage of the fast path: 0 = as fast as it can, 1 = head selected by radix, 2 = everything sorted
   KvPaging pg;
 };
 

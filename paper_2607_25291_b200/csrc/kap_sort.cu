@@ -500,12 +500,12 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
   __shared__ int sel_ctl[3];
   __shared__ int need_full;
   const int Kx = min(J, K + kTieMargin);
-  bool select_mode = p.top_p <= 0.0 && Kx <= kHeadCap && 2 * Kx <= J && J >= 64 && p.nqb <= 65536;
+  bool select_mode = p.sort_mode != 2 && p.top_p <= 0.0 && Kx <= kHeadCap && 2 * Kx <= J && J >= 64 && p.nqb <= 65536;
   unsigned long long* srt = keys;   // the sorted order: srt[0 .. L)
   int L = J;
   for (;;) {
     if (select_mode) {
-      int C = select_by_pivot(keys, J, Kx, picked, head, hist, sel_ctl, tid);   // (the head array is free until the sort)
+      int C = p.sort_mode == 1 ? 0 : select_by_pivot(keys, J, Kx, picked, head, hist, sel_ctl, tid);   // (the head array is free until the sort)
       if (C == 0) {
         select_largest(keys, J, Kx, picked, hist, sel_ctl, tid);
         C = Kx;

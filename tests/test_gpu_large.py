@@ -109,6 +109,26 @@ def test_qwen3_32k_full_kap_and_sampled_osk():
     print("32k", stats)
 
 
+def test_qwen3_32k_sort_routes_agree():
+    """The sort stage has three routes to the same list: head by pivot selection (taken here by nearly every list),
+    head by radix selection, everything sorted.  All 8192 lists must come out identical on each (the first one is
+    checked against the oracle, list by list, by the test above)."""
+    w = WORKLOADS["qwen3_32k"]
+    qb, kb, _, _ = w.make()
+    q, k = to_dev(qb), to_dev(kb)
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(w.kap_budget, nqb) + 7) // 8 * 8
+    lists = []
+    for impl in (0, 2, 3):
+        order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+        count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+        cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride, order_stride=pitch, impl=impl))
+        assert cosa.cosa_device_status() == 0
+        lists.append((order, count))
+    for order, count in lists[1:]:
+        assert torch.equal(count, lists[0][1]) and torch.equal(order, lists[0][0])
+
+
 def test_qwen3_128k_sampled():
     w = WORKLOADS["qwen3_128k"]
     qb, kb, vb, _ = w.make()

@@ -263,13 +263,14 @@ def mid():
 MID_BLOCKS = [0, 1, 63, 64, 71, 72, 89, 90, 100, 117, 126, 127]
 
 
+@pytest.mark.parametrize("impl", [0, 2, 3])
 @pytest.mark.parametrize("budget", [0.05, 0.1, 0.25, 0.6])
-def test_kap_16k_head_of_the_order(mid, budget):
+def test_kap_16k_head_of_the_order(mid, budget, impl):
     """At 128 key blocks and a small budget the fast path selects and sorts only the head of the order (kept prefix
     plus a margin); larger budgets and short candidate lists sort everything.  Both must give the oracle's lists."""
     q, k, _ = mid["dev"]
     qf, kf, _ = mid["f64"]
-    order, count = run_kap(q, k, budget, 8)
+    order, count = run_kap(q, k, budget, 8, impl=impl)   # 2, 3: the sort stage's fall-back routes, forced
     ref_order, ref_count = O.kap_select(qf, kf, s=8, budget=budget, order_stride=order.shape[-1], query_blocks=MID_BLOCKS)
     for i in MID_BLOCKS:
         assert np.array_equal(_np(count)[:, i], ref_count[:, i]), i
@@ -287,8 +288,8 @@ def test_kap_16k_tie_chain_longer_than_the_margin(mid):
         k2[0, :, dst * 128:(dst + 1) * 128] = k2[0, :, 20 * 128:21 * 128]
         kf2[:, dst * 128:(dst + 1) * 128] = kf2[:, 20 * 128:21 * 128]
     blocks = [64, 90, 110, 127]
-    for budget in (0.1, 0.3):
-        order, count = run_kap(q, k2, budget, 8)
+    for budget, impl in ((0.1, 0), (0.3, 0), (0.1, 2), (0.3, 3)):
+        order, count = run_kap(q, k2, budget, 8, impl=impl)
         ref_order, ref_count = O.kap_select(qf, kf2, s=8, budget=budget, order_stride=order.shape[-1], query_blocks=blocks)
         for i in blocks:
             assert np.array_equal(_np(count)[:, i], ref_count[:, i]), (budget, i)
