@@ -111,7 +111,10 @@ typedef struct {
 
 void cosa_default_options(cosa_options* opt);
 
-/* Scratch bytes a call with explicit workspace needs.  op: 0 = KAP, 1 = OSK, 2 = both. */
+/* Scratch bytes a call with explicit workspace needs.  op: 0 = KAP, 1 = OSK, 2 = both.  The KAP figure covers the
+ * screened scores ([B,Hq,nQB,nQB] floats) and one area of parked block maxima per CTA of the screen kernel that can be
+ * resident at once, so it depends on the SM count of the current device (160 is assumed when there is none): ask
+ * with the device current on which the call will run. */
 size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt);
 
 /* Number of blocks kept out of `candidates` under a budget fraction: ceil(budget*candidates)
