@@ -107,6 +107,16 @@ typedef struct {
   int32_t kv_page_size;    /* tokens per physical page: a power of two in [8, N] that divides N and, for
                               KAP, is a multiple of the stride                                       */
   int32_t kv_num_pages;    /* pages in the pools                                                     */
+  const int32_t* seq_lens; /* Non-NULL: device array [B]; batch item b holds seq_lens[b] tokens, a multiple
+                              of 128 in [128, N] (a batch of prompts of different lengths, padded to N;
+                              Sec. C.1 runs inside a paged serving engine, where this is the rule).  Rows
+                              past the length are padding: they are never read as keys, their query
+                              blocks get empty lists (count 0) from cosa_kap_select and all-zero out,
+                              lse = -inf and visited = 0 from cosa_osk_attention, and candidate
+                              counts (budget counts, the Stage-2 cap) and the N of the skip rule
+                              (Eq. 5; skip_scale must stay below the shortest length) follow the
+                              item's own length: every item comes out as in a call of its own.
+                              Not with block_q = 256, not in cosa_prefill_host                      */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);

@@ -44,7 +44,7 @@ class CosaOptions(Structure):
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p), ("kv_page_table", c_void_p),
-                ("kv_page_size", c_int32), ("kv_num_pages", c_int32)]
+                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p)]
 
 
 class CosaError(RuntimeError):

@@ -73,6 +73,8 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // Paging arguments of a call: COSA_OK and *pg filled (table == nullptr when the tensors are dense).
 int resolve_paging(const cosa_shape* s, const cosa_options& o, int stride, KvPaging* pg) {
   *pg = KvPaging{};
+  pg->seq_lens = o.seq_lens;
+  if (o.seq_lens && s->block_q != kBlock) return COSA_ERR_UNSUPPORTED;   // lengths are multiples of 128, not of 256
   if (!o.kv_page_table) return COSA_OK;
   const int ps = o.kv_page_size;
   if (ps < 8 || (ps & (ps - 1)) != 0 || ps > s->n || s->n % ps != 0 || o.kv_num_pages < s->n / ps) return COSA_ERR_INVALID_ARG;
@@ -266,6 +268,7 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   if (p.use_threshold && !(o.skip_scale < (float)shape->n)) return COSA_ERR_INVALID_ARG;
   p.cap_fx = budget_to_fx(tightened_budget);
   p.theta = p.use_threshold ? (float)log((double)o.skip_scale / (double)shape->n) : 0.f;
+  p.skip_scale = o.skip_scale;
   p.scale = o.softmax_scale > 0.f ? o.softmax_scale : (float)(1.0 / sqrt((double)shape->d));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : launch_osk_tc(p, st);
@@ -374,6 +377,7 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
   if (rc != COSA_OK) return rc;
   if (!q_host || !k_host || !v_host || !out_host || !device_workspace) return COSA_ERR_INVALID_ARG;
   cosa_options o = resolve_options(opt);
+  if (o.seq_lens) return COSA_ERR_UNSUPPORTED;   // the slices of this call are whole sequences
   HostCallLayout L = host_layout(shape, o);
   if (device_workspace_bytes < L.total || !aligned16(device_workspace)) return COSA_ERR_WORKSPACE;
   char* ws = static_cast<char*>(device_workspace);

@@ -14,13 +14,28 @@ constexpr int kHeadDim = 128;
 
 // Paged K/V (Sec. C.1): k and v are page pools [P, Hkv, b_p, d]; token t of KV head g of batch item b lives in row
 // t mod b_p of pool[table[b, t div b_p], g].  table == nullptr: k and v are the dense [B, Hkv, N, d] tensors.
+// seq_lens (with or without pages): batch item b holds seq_lens[b] <= N tokens, a multiple of the block size; the rest
+// of its rows is padding that no kernel reads as a key and for which no list or output is produced.
 struct KvPaging {
   const int32_t* table;   // [B, N / b_p]
   int page_size;          // b_p, a power of two
   int page_shift;         // log2 b_p
   int pages_per_seq;      // N / b_p
   int num_pages;          // P
+  const int32_t* seq_lens;   // [B] or nullptr: every item has N tokens
 };
+
+// 128-token blocks of batch item b (nqb: blocks of a full-length item)
+__device__ __forceinline__ int item_blocks(const KvPaging& pg, int b, int nqb) {
+  return pg.seq_lens ? max(0, min(nqb, pg.seq_lens[b] / kBlock)) : nqb;
+}
+
+// ln(Delta / N) of batch item b: N is the item's own length when the batch carries lengths (Eq. 5's N is the
+// length of the context the query attends to), else the host's value for the common length
+__device__ __forceinline__ float item_theta(const KvPaging& pg, int b, float theta_common, float skip_scale, int blocks_b) {
+  if (!pg.seq_lens || blocks_b <= 0) return theta_common;
+  return (float)log((double)skip_scale / (double)(blocks_b * kBlock));
+}
 
 // Row of the [rows, d] view of k / v that holds `token` of KV head g of batch item b.
 __host__ __device__ inline long long kv_row(const KvPaging& pg, int b, int hkv, int g, int n, int token) {
@@ -89,6 +104,7 @@ struct OskParams {
   int use_threshold;     // stage2 && Delta > 0
   long long cap_fx;      // floor(tightened_budget_f32 * 2^20)
   float theta;           // ln(Delta / N)
+  float skip_scale;      // Delta (for items whose own length replaces N, see item_theta)
   float scale;           // softmax scale
   KvPaging pg;
 };

@@ -44,9 +44,18 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
   const int T = p.qtiles;               // row tiles of the query block
   const int i = i_lo + T - 1;           // its last row tile
   const int g = h / (p.hq / p.hkv);
-  const int J = p.causal ? i + 1 : p.nqb;
+  const int nqb_b = item_blocks(p.pg, b, p.nqb);   // the item's own length in blocks
+  const int J = p.causal ? i + 1 : nqb_b;
   const int Jpad = p.nqb | 1;
   const int tid = threadIdx.x;
+  if (i >= nqb_b) {                     // padding past the item's length: empty lists
+    for (int tile = 0; tile < T; ++tile) {
+      const size_t lrow = (size_t)(b * p.hq + h) * p.nqb + i_lo + tile;
+      for (int t = tid; t < p.order_stride; t += kThreads) p.order[lrow * p.order_stride + t] = -1;
+      if (tid == 0) p.count[lrow] = 0;
+    }
+    return;
+  }
 
   double* Qs = reinterpret_cast<double*>(smem_raw);
   double* Ks = Qs + (size_t)R * kPad;

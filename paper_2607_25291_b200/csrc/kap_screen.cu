@@ -89,12 +89,16 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   const int g = (w / n_iq) % p.hkv;
   const int iq = n_iq - 1 - (w % n_iq);         // longest first
   const int i0 = iq * QB;
-  const int i_max = min(i0 + QB, p.nqb) - 1;
-  const int ns = p.n / p.stride;                // sampled rows per head
-  const int n_keys = p.causal ? (i_max + 1) * R : ns;
+  const int nqb_b = item_blocks(p.pg, b, p.nqb);      // the item's own length in blocks
+  const int i_max = min(i0 + QB, nqb_b) - 1;
+  const int ns = p.n / p.stride;                // sampled rows per head (tensor pitch)
+  const int ns_b = nqb_b * R;                   // ... that the item really has
+  const int n_keys = p.causal ? (i_max + 1) * R : ns_b;
   const int n_tiles = (n_keys + 127) / 128;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
+  if (i0 >= nqb_b) return;                        // all of this CTA's query blocks are padding
   if (threadIdx.x == 0) {
     // once some CTA has reported a timeout the rest of the grid returns at once
     int poisoned = *reinterpret_cast<volatile int32_t*>(status);
@@ -118,7 +122,6 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   if (ctl->poisoned != 0) return;
 
   if (threadIdx.x == 0) {
-    if (blockIdx.x == 0) p.redo_list[0] = 0;   // the sort stage (a later launch) appends to it
     mbar_init(smem_u32(&ctl->a_full), 1);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < kSteps; ++s) mbar_init(smem_u32(&ctl->s_empty[s]), kEpiThreads);
@@ -181,7 +184,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (!ok) break;
         if (lane < parts) {
           int tok = (t * 128 + lane * spp) * p.stride;
-          if (tok >= p.n) tok = 0;
+          if (tok >= nqb_b * kBlock) tok = 0;      // past the item's length: masked later, any valid page will do
           const int srow = (int)(kv_row(p.pg, b, p.hkv, g, p.n, tok) / p.stride);
           tma_load_2d(dst + lane * spp * 128, &k_map, 0, srow, bar);
           tma_load_2d(dst + kHalfBytes + lane * spp * 128, &k_map, 64, srow, bar);
@@ -218,9 +221,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     const uint32_t lane_addr = (uint32_t)(sub * 32) << 16;
     const int grp = row / R, r = row % R;
     const int i = i0 + grp / G, h = g * G + grp % G;
-    const bool row_ok = i < p.nqb;
+    const bool row_ok = i < nqb_b;
     const int r_glob = i * R + r;                        // index among the head's sampled rows
-    const int c_limit = p.causal ? r_glob : ns - 1;      // last sampled key this row may see
+    const int c_limit = p.causal ? r_glob : ns_b - 1;    // last sampled key this row may see
     constexpr int BPC = kPartCols / R;                   // key blocks per column part
     float top1 = -INFINITY, top2 = -INFINITY, top3 = -INFINITY;
     int jstar = 0, jstar2 = 0;
@@ -343,7 +346,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       const int oo = et % kOutsPerTile;
       const int blk = oo % BPT, og = oo / BPT;             // consecutive lanes: consecutive key blocks
       const int oi = i0 + og / G, oh = g * G + og % G;
-      const int J = p.causal ? oi + 1 : p.nqb;
+      const int J = p.causal ? oi + 1 : nqb_b;
       const float kLog2e = 1.4426950408889634f;
       const float scale2 = p.scale * kLog2e;
       // a thread reads its R maxima as R/4 vectors, starting at a vector that depends on the lane so that the
@@ -375,7 +378,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         for (int o = et; o < tiles_here * kOutsPerTile; o += kEpiThreads) {
           const int tl = o / kOutsPerTile;
           const int j = (c * kTilesPerChunk + tl) * BPT + blk;
-          if (oi < p.nqb && j < J) {
+          if (oi < nqb_b && j < J) {
             const float4* src = reinterpret_cast<const float4*>(stage + (size_t)tl * kTileFloats + ((size_t)og * BPT + blk) * R);
             float e0 = 0.f, e1 = 0.f;
             bool fl = false;

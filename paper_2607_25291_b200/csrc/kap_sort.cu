@@ -394,10 +394,18 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
   const int i_lo = big * T, i = i_lo + T - 1; // first and last row tile of the query block
   const int h = blockIdx.y, b = blockIdx.z;
   const int g = h / (p.hq / p.hkv);
-  const int J = p.causal ? i + 1 : p.nqb;     // candidates: key blocks some row of the block may see
+  const int nqb_b = item_blocks(p.pg, b, p.nqb);   // the item's own length in blocks
+  const int J = p.causal ? i + 1 : nqb_b;     // candidates: key blocks some row of the block may see
   const int tid = threadIdx.x;
   const size_t row_lo = (size_t)(b * p.hq + h) * p.nqb + i_lo;
   const size_t row = row_lo + (T - 1);
+  if (i >= nqb_b) {                           // padding past the item's length: empty lists
+    for (int tile = 0; tile < T; ++tile) {
+      for (int t = tid; t < p.order_stride; t += kThreads) p.order[(row_lo + tile) * p.order_stride + t] = -1;
+      if (tid == 0) p.count[row_lo + tile] = 0;
+    }
+    return;
+  }
   unsigned hard = 0u;                         // (tested only after the scores have been requested: one round trip, not two)
   unsigned long long amb = 0ULL;              // bit r: sampled row r of the block was too close to call
   for (int t = 0; t < T; ++t) {

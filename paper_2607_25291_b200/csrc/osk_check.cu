@@ -26,12 +26,14 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
   const int g = h / (p.hq / p.hkv);
   const int t = threadIdx.x;  // query row inside the tile
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  const int J = p.causal ? i + 1 : p.nqb;
+  const int nqb_b = item_blocks(p.pg, b, p.nqb);   // the item's own length in blocks; query blocks past it are padding
+  const int J = p.causal ? i + 1 : nqb_b;
   BlockWalk walk;
-  walk.init(p, row, J);
-  const int cnt = p.mask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride));
+  walk.init(p, row, max(J, 1));
+  const int cnt = i >= nqb_b ? 0 : (p.mask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride)));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
   const int dec_words = (p.order_stride + 31) / 32;
+  const float theta = p.use_threshold ? item_theta(p.pg, b, p.theta, p.skip_scale, nqb_b) : 0.f;
 
   // this thread's query row as packed bf16 pairs
   uint32_t qreg[kHeadDim / 2];
@@ -89,7 +91,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
     __syncthreads();
     if (t == 0) {
       float gm = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-      s_skip = (p.use_threshold && gm < p.theta) ? 1 : 0;
+      s_skip = (p.use_threshold && gm < theta) ? 1 : 0;
     }
     __syncthreads();
     const bool skip = s_skip != 0;

@@ -137,11 +137,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const int i = p.nqb - 1 - (wk % per_kv) / G;
   const int h = g * G + (wk % per_kv) % G;
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
-  const int J = p.causal ? i + 1 : p.nqb;
+  const int nqb_b = item_blocks(p.pg, b, p.nqb);   // the item's own length in blocks; query blocks past it are padding
+  const int J = p.causal ? i + 1 : max(nqb_b, 1);
   const int32_t* list = p.order + row * p.order_stride;   // unused when kMask
   BlockWalk walk;                         // (kMask only) every thread that needs block ids walks on its own
   if (kMask) walk.init(p, row, J);
-  const int cnt = kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride));
+  const int cnt = i >= nqb_b ? 0 : (kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride)));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
   const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N, d] view
 
@@ -184,7 +185,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
-    if (ctl->poisoned == 0) {
+    if (ctl->poisoned == 0 && cnt > 0) {   // (an empty list fetches nothing: no copy may be in flight when its CTA retires)
       // Q and the first K tiles are requested before the rest of the CTA has even finished setting up
       mbar_expect_tx(smem_u32(&ctl->q_stage), kTileBytes);
       tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_stage));
@@ -217,7 +218,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   volatile int* abort_flag = &ctl->abort_flag;
   const float kLog2e = 1.4426950408889634f;
   const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
-  const float theta2 = p.theta * kLog2e;
+  const float theta2 = (p.use_threshold ? item_theta(p.pg, b, p.theta, p.skip_scale, nqb_b) : 0.f) * kLog2e;
 
   // register budget: the control warps need few, the softmax threads hold a whole S row
   if (warp < 4) {

@@ -618,6 +618,71 @@ def test_batch_of_two_equals_single_items(impl):
         assert torch.equal(x, y)
 
 
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("causal", [True, False])
+@pytest.mark.parametrize("n,lens", [(1024, [1024, 640]), (4096, [1536, 4096])])
+def test_batch_with_different_lengths(impl, causal, n, lens):
+    """Prompts of 1024 and 640 tokens in one call, padded to 1024 (cosa_options.seq_lens): every item gives exactly
+    what a call on its unpadded tensors gives -- lists also checked against the oracle -- and the padding gets empty
+    lists, zero output, lse = -inf.  The same through page pools whose table rows point at a wrong (but valid) page
+    past the length: nothing there may be read.  (At 4096 tokens whole CTAs of the screen kernel lie in the padding.)"""
+    items = []
+    for seed in (51, 52):
+        w = tiny(seed=seed, hq=4, hkv=2, n=n, needles=2)
+        qb, kb, vb, _ = w.make()
+        items.append((qb, kb, vb))
+    stack = lambda idx: torch.cat([to_dev(it[idx]) for it in items], dim=0).contiguous()
+    q2, k2, v2 = stack(0), stack(1), stack(2)
+    seq_lens = torch.tensor(lens, dtype=torch.int32, device="cuda")
+
+    def run(q, k, v, batch, n_tok, **extra):
+        nqb = n_tok // 128
+        order = torch.full((batch, 4, nqb, nqb), -7, dtype=torch.int32, device="cuda")
+        count = torch.full((batch, 4, nqb), -7, dtype=torch.int32, device="cuda")
+        out = torch.full_like(q, 3.0)
+        lse = torch.full((batch, 4, n_tok), 3.0, dtype=torch.float32, device="cuda")
+        vis = torch.full((batch, 4, nqb), -7, dtype=torch.int32, device="cuda")
+        opt = cosa.default_options(impl=impl, skip_scale=200.0, **extra)
+        cosa.cosa_kap_select(q, k, 0.6, order, count, causal=causal, opt=opt)
+        cosa.cosa_osk_attention(q, k, v, order, count, 0.4, out, lse, vis, causal=causal, opt=opt)
+        assert cosa.cosa_device_status() == 0
+        return order, count, out, lse, vis
+
+    def check(both):
+        order, count, out, lse, vis = both
+        for b, ln in enumerate(lens):
+            nb = ln // 128
+            cut = lambda t: t[b:b + 1, :, :ln].contiguous()
+            o1, c1, out1, lse1, vis1 = run(cut(q2), cut(k2), cut(v2), 1, ln)
+            assert torch.equal(count[b:b + 1, :, :nb], c1) and torch.equal(vis[b:b + 1, :, :nb], vis1)
+            assert torch.equal(order[b:b + 1, :, :nb, :nb], o1) and bool((order[b, :, :nb, nb:] == -1).all())
+            assert torch.equal(out[b:b + 1, :, :ln], out1) and torch.equal(lse[b:b + 1, :, :ln], lse1)
+            assert bool((count[b, :, nb:] == 0).all()) and bool((order[b, :, nb:] == -1).all())
+            assert bool((vis[b, :, nb:] == 0).all()) and bool((out[b, :, ln:] == 0).all())
+            assert bool(torch.isinf(lse[b, :, ln:]).all()) and bool((lse[b, :, ln:] < 0).all())
+            qf, kf, _ = widen(items[b][0][:, :ln], items[b][1][:, :ln], items[b][2][:, :ln])
+            ref_order, ref_count = O.kap_select(qf, kf, s=8, budget=0.6, causal=causal, order_stride=nb)
+            assert np.array_equal(count.cpu().numpy()[b, :, :nb], ref_count)
+            assert np.array_equal(order.cpu().numpy()[b, :, :nb, :nb], ref_order)
+
+    check(run(q2, k2, v2, 2, n, seq_lens=seq_lens))
+    page_size = 64
+    pools, tables = [], []
+    for (_, kb, vb), ln in zip(items, lens):
+        kp, tab = scatter_to_pages(kb, page_size, seed=6)
+        vp, _ = scatter_to_pages(vb, page_size, seed=6)
+        tab = tab + sum(p_[0].shape[0] for p_ in pools)
+        tab[ln // page_size:] = 0                       # past the length: some other sequence's page
+        tables.append(tab)
+        pools.append((kp, vp))
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda().contiguous()
+    kpool = dev(np.concatenate([p_[0] for p_ in pools])); vpool = dev(np.concatenate([p_[1] for p_ in pools]))
+    table = torch.from_numpy(np.stack(tables).astype(np.int32)).cuda().contiguous()
+    paged = run(q2, kpool, vpool, 2, n, seq_lens=seq_lens, kv_page_table=table, kv_page_size=page_size,
+                kv_num_pages=kpool.shape[0])
+    check(paged)
+
+
 def test_osk_is_deterministic(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
