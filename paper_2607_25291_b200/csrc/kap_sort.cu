@@ -7,8 +7,11 @@
 //  1. Rows whose two largest block maxima the screen could not tell apart (ambmask) are settled
 //     first: both blocks are re-evaluated with double-precision FMAs on the exact bf16 inputs,
 //     which fixes the row's M* and which block(s) earn the HRM flag from that row (Eq. 12).
-//  2. The candidates are sorted by (HRM flag descending, float32 score descending, block id
-//     ascending).
+//  2. The candidates are ordered by (HRM flag descending, float32 score descending, block id
+//     ascending).  With a small budget only the head of that order is needed (the kept prefix
+//     plus a margin for step 3): it is selected by a threshold (pivots from a sample, or a radix
+//     selection) and rank-sorted; otherwise, and whenever the head proves too short, everything
+//     is sorted by a bitonic network.
 //  3. Two sorted neighbours with the same flag whose scores differ by less than tau_score
 //     (relative) are a "near tie"; a maximal chain of near ties that starts inside the kept
 //     prefix (or straddles its end) is recounted: M[r,j] of each of its blocks and M*[r] are
@@ -25,7 +28,7 @@ namespace cosa {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kMaxTied = 96;
+constexpr int kMaxTied = 96;      // chained entries one list may have before it is left to the double-precision kernel
 constexpr int kMaxRows = 64;   // sampled rows of one (possibly two-tile) query block
 constexpr int kHeadCap = 256;     // entries of the order's head that are selected and sorted on their own
 constexpr int kPad = kHeadDim + 1;
