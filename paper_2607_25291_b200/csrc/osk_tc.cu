@@ -268,6 +268,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           while (kk >= ctl->n_needed + kSpec) {
             if (ctl->end_kk >= 0) { ended = true; break; }
             if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+            __nanosleep(20);   // a bare spin here takes issue slots from the two softmax warps of this sub-partition (1 % of the kernel)
           }
           if (ended || !alive) break;
         }
