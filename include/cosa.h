@@ -270,6 +270,10 @@ int cosa_device_status(void* stream);
 const char* cosa_last_cuda_error(void);
 const char* cosa_status_string(int status);
 int cosa_version(void);
+/* sizeof(cosa_options) and sizeof(cosa_shape) as this library was built: a binding in another language checks its own
+ * declarations against them before it passes a structure in (cosa_default_options writes sizeof(cosa_options) bytes). */
+size_t cosa_options_bytes(void);
+size_t cosa_shape_bytes(void);
 
 #ifdef __cplusplus
 }

@@ -29,7 +29,7 @@ COSA_ERR_BAD_ORDER = -6
 EXPORTS = (
     "cosa_default_options", "cosa_workspace_bytes", "cosa_budget_count", "cosa_kap_select",
     "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_reorder_lists", "cosa_lists_to_mask", "cosa_validate_order",
-    "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status",
+    "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status", "cosa_options_bytes", "cosa_shape_bytes",
     "cosa_last_cuda_error", "cosa_status_string", "cosa_version",
 )
 
@@ -67,6 +67,11 @@ def _load():
         raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_25291_b200.build` "
                           "(there is no CPU or PyTorch fallback)")
     lib = ctypes.CDLL(LIB_PATH)
+    lib.cosa_options_bytes.restype = c_size_t
+    lib.cosa_shape_bytes.restype = c_size_t
+    if lib.cosa_options_bytes() != ctypes.sizeof(CosaOptions) or lib.cosa_shape_bytes() != ctypes.sizeof(CosaShape):
+        raise ImportError(f"{LIB_PATH} was built from another cosa.h than this binding declares "
+                          f"(options {lib.cosa_options_bytes()} vs {ctypes.sizeof(CosaOptions)} bytes): rebuild it")
     lib.cosa_default_options.argtypes = [POINTER(CosaOptions)]
     lib.cosa_default_options.restype = None
     lib.cosa_workspace_bytes.argtypes = [c_int, POINTER(CosaShape), POINTER(CosaOptions)]

@@ -472,5 +472,7 @@ const char* cosa_status_string(int status) {
 }
 
 int cosa_version(void) { return 100; }
+size_t cosa_options_bytes(void) { return sizeof(cosa_options); }
+size_t cosa_shape_bytes(void) { return sizeof(cosa_shape); }
 
 }  // extern "C"
