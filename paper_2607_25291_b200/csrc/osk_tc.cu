@@ -164,8 +164,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 
   static_assert(kVStages == 2 && kKStages == 4, "PV product n frees V stage n & 1 together with p_empty[n & 1]");
   if (threadIdx.x == 0) {
-    // once some CTA has reported a timeout the rest of the grid returns at once
-    ctl->poisoned = poisoned_early;
+    // barriers first, then the Q tile at once: its address needs nothing from global memory, while the list
+    // entries, the count and the status word requested above are still on their way (2 k cycles at the start of a CTA)
     mbar_init(smem_u32(&ctl->q_stage), 1); mbar_init(smem_u32(&ctl->q_full), kBlock);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
@@ -177,7 +177,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     mbar_init(smem_u32(&ctl->out_bar), kBlock);
     mbar_init(smem_u32(&ctl->p_full), kBlock);
     mbar_init(smem_u32(&ctl->fin_bar), kBlock);
-    ctl->n_needed = min(cnt, cap);
     ctl->n_dec = 0;
     ctl->end_kk = -1;
     ctl->k_loaded = -1;
@@ -185,11 +184,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
-    if (ctl->poisoned == 0 && cnt > 0) {   // (an empty list fetches nothing: no copy may be in flight when its CTA retires)
-      // Q and the first K tiles are requested before the rest of the CTA has even finished setting up
-      mbar_expect_tx(smem_u32(&ctl->q_stage), kTileBytes);
-      tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_stage));
-      tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, smem_u32(&ctl->q_stage));
+    mbar_expect_tx(smem_u32(&ctl->q_stage), kTileBytes);
+    tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_stage));
+    tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, smem_u32(&ctl->q_stage));
+    // once some CTA has reported a timeout the rest of the grid returns at once
+    ctl->poisoned = poisoned_early;
+    ctl->n_needed = min(cnt, cap);
+    if (poisoned_early == 0 && cnt > 0) {
+      // the first K tiles, before the rest of the CTA has even finished setting up
       const int n_first = min(min(cnt, cap), kKStages);
       for (int kk = 0; kk < n_first; ++kk) {
         const int j = min(max(first_ids[kk], 0), p.nqb - 1);
@@ -208,6 +210,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   tc_fence_after();
   if (ctl->poisoned != 0) {
     if (warp == 1) tmem_dealloc(ctl->tmem_base, kTmemCols);
+    if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&ctl->q_stage), 0, &ctl->abort_flag);   // no copy may be in flight when the CTA retires
     return;
   }
   const uint32_t tmem = ctl->tmem_base;
@@ -390,6 +393,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (threadIdx.x == 128) {
         if (p.visited) p.visited[row] = 0;
         if (p.scored) p.scored[row] = 0;
+        if (!mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag) && !*abort_flag) report_timeout(ctl, status);   // the Q tile was requested all the same
       }
     }
   } else {
