@@ -554,11 +554,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           const float inv = lt > 0.f ? 1.f / lt : 0.f;
           // stage the tile in (now idle) K stage memory, swizzled like two TMA boxes of 64 columns, and let
           // one thread store it with two bulk tensor copies
+          // (all four loads in flight at once, into the registers that held the logits)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) tmem_ld32(tmem_o + lane_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+          tmem_wait_ld();
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tmem_o + lane_addr + c * 32, o);
-            tmem_wait_ld();
+            const uint32_t* o = &s[c * 32];
             unsigned char* stage = smem + (c >> 1) * kHalfBytes;
 #pragma unroll
             for (int e = 0; e < 32; e += 8) {
