@@ -421,20 +421,42 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
   // no score for key blocks wholly after it
   int P2 = 2;
   while (P2 < J) P2 <<= 1;
-  for (int j = tid; j < P2; j += kThreads) {
-    unsigned long long key = 0ULL;
-    if (j < J) {
-      float sum = 0.f;
-      unsigned flag = 0u;
-      for (int t = 0; t < T; ++t) {
-        if (p.causal && j > i_lo + t) continue;
-        const float v = sp.scores[(row_lo + t) * p.nqb + j];
-        sum += fabsf(v);
-        flag |= (v < 0.f) ? 0x80000000u : 0u;
+  if (T == 1) {
+    // four scores per thread requested before any is used: the loads of a list are one round trip, not four
+    const float* srow = sp.scores + row_lo * p.nqb;
+    for (int j0 = 0; j0 < P2; j0 += 4 * kThreads) {
+      float v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u * kThreads + tid;
+        v[u] = j < J ? srow[j] : 0.f;
       }
-      key = ((unsigned long long)(__float_as_uint(sum) | flag) << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u * kThreads + tid;
+        if (j < P2) {
+          const unsigned flag = (v[u] < 0.f) ? 0x80000000u : 0u;
+          keys[j] = j < J ? ((unsigned long long)(__float_as_uint(fabsf(v[u])) | flag) << 32) | (unsigned long long)(0xffffffffu - (unsigned)j)
+                          : 0ULL;
+        }
+      }
     }
-    keys[j] = key;
+  } else {
+    for (int j = tid; j < P2; j += kThreads) {
+      unsigned long long key = 0ULL;
+      if (j < J) {
+        float sum = 0.f;
+        unsigned flag = 0u;
+        for (int t = 0; t < T; ++t) {
+          if (p.causal && j > i_lo + t) continue;
+          const float v = sp.scores[(row_lo + t) * p.nqb + j];
+          sum += fabsf(v);
+          flag |= (v < 0.f) ? 0x80000000u : 0u;
+        }
+        key = ((unsigned long long)(__float_as_uint(sum) | flag) << 32) | (unsigned long long)(0xffffffffu - (unsigned)j);
+      }
+      keys[j] = key;
+    }
   }
   if (hard) {  // left to the double-precision kernel
     if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
