@@ -114,12 +114,15 @@ __device__ void f64_block_maxima(const KapParams& p, const double* Qs, int b, in
 }
 
 // The same maxima when a set names ONE key block for all rows (block_of(set) >= 0): a thread takes one sampled key
-// of the block against eight consecutive rows, so that every key element is widened once for eight FMA chains --
-// widening bf16 to double is what this stage spends its time on.  rows is a multiple of 8.
+// of the block against four consecutive rows, so that every key element is widened once for four FMA chains
+// (widening float to double runs at a quarter of the FP64 FMA rate on this GPU).  Four, not eight: under this
+// kernel's register limit eight accumulators spilled, and every FMA then went through local memory (40 k cycles
+// for the stage instead of 5 k).  rows is a multiple of 4.
 template <typename BlockOf>
 __device__ void f64_block_maxima_shared_key(const KapParams& p, const double* Qs, int b, int g, int row0, int rows, int R,
                                             int n_sets, BlockOf block_of, double (*out)[kMaxRows], int tid) {
-  const int chunks = rows / 8;
+  constexpr int kRowsPer = 4;
+  const int chunks = rows / kRowsPer;
   const int per_set = chunks * R, items = n_sets * per_set;
   const int items_pad = (items + 31) & ~31;      // whole warps: the R lanes of a (set, rows) group shuffle
   for (int e = tid; e < items_pad; e += kThreads) {
@@ -127,10 +130,10 @@ __device__ void f64_block_maxima_shared_key(const KapParams& p, const double* Qs
     const int set = valid ? e / per_set : 0, ch = (e / R) % chunks, c = e % R;
     const int kc = block_of(set) * R + c;        // sampled key index
     const uint4* ks = reinterpret_cast<const uint4*>(p.k + (size_t)kv_row(p.pg, b, p.hkv, g, p.n, kc * p.stride) * kHeadDim);
-    const double* q0 = Qs + (size_t)(ch * 8) * kPad;
-    double acc[8];
+    const double* q0 = Qs + (size_t)(ch * kRowsPer) * kPad;
+    double acc[kRowsPer];
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) acc[rr] = 0.0;
+    for (int rr = 0; rr < kRowsPer; ++rr) acc[rr] = 0.0;
 #pragma unroll 2
     for (int c8 = 0; c8 < kHeadDim / 8; ++c8) {
       const uint4 w = ks[c8];
@@ -139,14 +142,14 @@ __device__ void f64_block_maxima_shared_key(const KapParams& p, const double* Qs
       for (int u = 0; u < 4; ++u) {
         const double klo = bf16_lo(kw[u]), khi = bf16_hi(kw[u]);
 #pragma unroll
-        for (int rr = 0; rr < 8; ++rr) acc[rr] = fma(q0[rr * kPad + c8 * 8 + 2 * u], klo, acc[rr]);
+        for (int rr = 0; rr < kRowsPer; ++rr) acc[rr] = fma(q0[rr * kPad + c8 * 8 + 2 * u], klo, acc[rr]);
 #pragma unroll
-        for (int rr = 0; rr < 8; ++rr) acc[rr] = fma(q0[rr * kPad + c8 * 8 + 2 * u + 1], khi, acc[rr]);
+        for (int rr = 0; rr < kRowsPer; ++rr) acc[rr] = fma(q0[rr * kPad + c8 * 8 + 2 * u + 1], khi, acc[rr]);
       }
     }
 #pragma unroll
-    for (int rr = 0; rr < 8; ++rr) {
-      const int r = ch * 8 + rr;
+    for (int rr = 0; rr < kRowsPer; ++rr) {
+      const int r = ch * kRowsPer + rr;
       double z = (valid && (!p.causal || kc <= row0 + r)) ? acc[rr] * p.scale : -INFINITY;
       for (int o = R >> 1; o > 0; o >>= 1) z = fmax(z, __shfl_xor_sync(0xffffffffu, z, o));
       if (valid && c == 0) out[set][r] = z;
