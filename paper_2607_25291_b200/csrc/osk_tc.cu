@@ -492,15 +492,23 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       // ---- P = exp(S - m), row sums (in registers)
       const float alpha = ex2_approx(m_in - m_new);   // O refers to m_in: skipped blocks never move the maximum
       const float neg_m = -m_new;
-      float rs[4] = {0.f, 0.f, 0.f, 0.f};
+      // (two elements per FMA and per add: the packed float32 forms; the phase is bound by instruction issue)
+      float rs[4];
+      {
+        const unsigned long long sc2 = pack_f32x2(scale2, scale2), nm2 = pack_f32x2(neg_m, neg_m);
+        unsigned long long acc01 = pack_f32x2(0.f, 0.f), acc23 = acc01;
 #pragma unroll
-      for (int c = 0; c < kBlock; c += 4) {
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const float e = ex2_approx(fmaf(__uint_as_float(s[c + u]), scale2, neg_m));
-          rs[u] += e;
-          s[c + u] = __float_as_uint(e);
+        for (int c = 0; c < kBlock; c += 4) {
+          float e0, e1, e2, e3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2), e0, e1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), sc2, nm2), e2, e3);
+          e0 = ex2_approx(e0); e1 = ex2_approx(e1); e2 = ex2_approx(e2); e3 = ex2_approx(e3);
+          acc01 = add_f32x2(acc01, pack_f32x2(e0, e1));
+          acc23 = add_f32x2(acc23, pack_f32x2(e2, e3));
+          s[c] = __float_as_uint(e0); s[c + 1] = __float_as_uint(e1); s[c + 2] = __float_as_uint(e2); s[c + 3] = __float_as_uint(e3);
         }
+        unpack_f32x2(acc01, rs[0], rs[1]);
+        unpack_f32x2(acc23, rs[2], rs[3]);
       }
 #pragma unroll
       for (int c = 0; c < 64; ++c) s[c] = pack_bf16(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1]));
