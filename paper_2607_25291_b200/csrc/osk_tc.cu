@@ -452,11 +452,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 #pragma unroll
         for (int c = 0; c < kBlock; ++c) if (c > r) s[c] = 0xff800000u;  // -inf
       }
+      // (three-input maxima: half the instructions of the two-input form; the walk is bound by instruction issue)
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < kBlock; c += 4) {
+      for (int c = 0; c < kBlock; c += 8) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) mx[u] = fmaxf(mx[u], __uint_as_float(s[c + u]));
+        for (int u = 0; u < 4; ++u) mx[u] = max3(mx[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
       }
       const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
       // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
