@@ -264,34 +264,49 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (!alive && !*abort_flag) report_timeout(ctl, status);
       const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
       int last_issued = -1;
+      int n_certain = 0;        // a copy of n_needed, which only grows: positions below it are certain to be scored
+      bool verified = false;    // tile and S buffer of the position at hand were found ready while the previous product was set up
       for (int kk = 0; kk < cnt && alive; ++kk) {
-        if (kk >= ctl->n_needed + kSpec) {       // at most kSpec products beyond the blocks that are certain to be scored
-          const long long t0 = clock64();
-          bool ended = false;
-          while (kk >= ctl->n_needed + kSpec) {
-            if (ctl->end_kk >= 0) { ended = true; break; }
-            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
-            __nanosleep(20);   // a bare spin here takes issue slots from the two softmax warps of this sub-partition (1 % of the kernel)
-          }
-          if (ended || !alive) break;
-        }
-        if (ctl->end_kk >= 0 && kk > ctl->end_kk) break;
         const int st = kk % kKStages, sb = kk & 1;
-        {   // the tile, unless the loader stopped short of it (a position beyond the walk's end)
-          const uint32_t bar = smem_u32(&ctl->k_full[st]), par = (kk / kKStages) & 1;
-          bool none = false;
-          if (!mbar_try_wait(bar, par)) {
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar, par)) {
-              const int kl = ctl->k_loaded;
-              if (kl >= 0 && kk >= kl) { none = true; break; }
-              if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+        if (!verified) {
+          if (kk >= n_certain) {
+            n_certain = ctl->n_needed;
+            if (kk >= n_certain + kSpec) {         // at most kSpec products beyond the blocks that are certain to be scored
+              const long long t0 = clock64();
+              bool ended = false;
+              while (kk >= (n_certain = ctl->n_needed) + kSpec) {
+                if (ctl->end_kk >= 0) { ended = true; break; }
+                if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+                __nanosleep(20);   // a bare spin here takes issue slots from the two softmax warps of this sub-partition (1 % of the kernel)
+              }
+              if (ended || !alive) break;
             }
+            if (kk >= n_certain) { const int e = ctl->end_kk; if (e >= 0 && kk > e) break; }
           }
-          if (none || !alive) break;
+          {   // the tile, unless the loader stopped short of it (a position beyond the walk's end)
+            const uint32_t bar = smem_u32(&ctl->k_full[st]), par = (kk / kKStages) & 1;
+            bool none = false;
+            if (!mbar_try_wait(bar, par)) {
+              const long long t0 = clock64();
+              while (!mbar_try_wait(bar, par)) {
+                const int kl = ctl->k_loaded;
+                if (kl >= 0 && kk >= kl) { none = true; break; }
+                if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+              }
+            }
+            if (none || !alive) break;
+          }
+          alive = mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
+          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         }
-        alive = mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
-        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        // Issuing a product keeps this thread busy for about as long as the product runs, so whatever is checked
+        // between two products leaves the tensor pipe idle: look at the next position now, without waiting.
+        verified = false;
+        if (kk + 1 < n_certain) {
+          const int k1 = kk + 1;
+          verified = mbar_test_wait(smem_u32(&ctl->k_full[k1 % kKStages]), (k1 / kKStages) & 1) &&
+                     mbar_test_wait(smem_u32(&ctl->s_empty[k1 & 1]), ((k1 >> 1) & 1) ^ 1);
+        }
         tc_fence_after();
         // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
         mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
@@ -422,10 +437,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       tc_fence_before();
       mbar_arrive(smem_u32(&ctl->q_full));
     }
+    // only "is this the diagonal block" matters to a group; an ascending mask walk meets it last, if at all.  The list
+    // entry of a position is requested one turn ahead: its latency (some 400 cycles) would otherwise sit between a
+    // decision and the group's next S tile
+    const bool mask_diag = kMask && ((walk.mask[i >> 5] >> (i & 31)) & 1u);
+    int j_ahead = (!kMask && grp < cnt) ? list[grp] : 0;
     for (int kk = grp; kk < cnt && alive; kk += 2) {
-      // only "is this the diagonal block" matters here; an ascending mask walk meets it last, if at all
-      const int j = kMask ? ((kk == cnt - 1 && ((walk.mask[i >> 5] >> (i & 31)) & 1u)) ? i : -1)
-                           : min(max(list[kk], 0), p.nqb - 1);
+      const int j = kMask ? ((kk == cnt - 1 && mask_diag) ? i : -1) : j_ahead;
+      if (!kMask && kk + 2 < cnt) j_ahead = list[kk + 2];
       // wait for S(kk), or learn that the walk ended before this position
       {
         const uint32_t bar = smem_u32(&ctl->k_empty[kk % kKStages]), par = (kk / kKStages) & 1;   // QK^T(kk) finished
