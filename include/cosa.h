@@ -104,8 +104,12 @@ typedef struct {
                               logical page (Sec. C.1: a logical block of 128 tokens is resolved through
                               one or more physical pages when the page size differs).  NULL: k and v are
                               the dense [B, Hkv, N, d] tensors (page = block, identity table)        */
-  int32_t kv_page_size;    /* tokens per physical page: a power of two in [8, N] that divides N and, for
-                              KAP, is a multiple of the stride                                       */
+  int32_t kv_page_size;    /* tokens per physical page: a power of two in [8, N] that divides N.  Pools whose
+                              pages are smaller than a key block (for KAP: that hold fewer than 32 sampled
+                              rows) are first copied, sequence by sequence, into dense staging tensors in
+                              the scratch (impl = 0; the check kernels of impl = 1 read the pages row by
+                              row): cosa_workspace_bytes() then includes B*Hkv*N*d*2 bytes for K, and
+                              the same again for V in cosa_osk_attention                             */
   int32_t kv_num_pages;    /* pages in the pools                                                     */
   const int32_t* seq_lens; /* Non-NULL: device array [B]; batch item b holds seq_lens[b] tokens, a multiple
                               of 128 in [128, N] (a batch of prompts of different lengths, padded to N;
@@ -124,7 +128,8 @@ void cosa_default_options(cosa_options* opt);
 /* Scratch bytes a call with explicit workspace needs.  op: 0 = KAP, 1 = OSK, 2 = both.  The KAP figure covers the
  * screened scores ([B,Hq,nQB,nQB] floats) and one area of parked block maxima per CTA of the screen kernel that can be
  * resident at once, so it depends on the SM count of the current device (160 is assumed when there is none): ask
- * with the device current on which the call will run. */
+ * with the device current on which the call will run.  With small pages (see kv_page_size) both figures include
+ * the dense staging tensors; otherwise OSK needs none. */
 size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt);
 
 /* Number of blocks kept out of `candidates` under a budget fraction: ceil(budget*candidates)

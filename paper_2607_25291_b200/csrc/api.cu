@@ -78,7 +78,6 @@ int resolve_paging(const cosa_shape* s, const cosa_options& o, int stride, KvPag
   if (!o.kv_page_table) return COSA_OK;
   const int ps = o.kv_page_size;
   if (ps < 8 || (ps & (ps - 1)) != 0 || ps > s->n || s->n % ps != 0 || o.kv_num_pages < s->n / ps) return COSA_ERR_INVALID_ARG;
-  if (stride > 0 && ps % stride != 0) return COSA_ERR_UNSUPPORTED;
   if ((long long)o.kv_num_pages * s->hkv * ps > 0x7fffffffLL) return COSA_ERR_UNSUPPORTED;   // tensor-map row coordinates
   pg->table = o.kv_page_table;
   pg->page_size = ps;
@@ -102,14 +101,20 @@ cosa_options resolve_options(const cosa_options* opt) {
 }  // namespace
 
 // scratch the kernels of one call need (beyond inputs and outputs)
-struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, slot_taken, maxima, total; int slots; };
+struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, slot_taken, maxima, kstage, total; int slots; bool gather; };
 static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
   KapScratch L{};
   const int stride = o.stride > 0 ? o.stride : 8;
   KvPaging pg{};
   if (resolve_paging(s, o, stride, &pg) != COSA_OK) return L;
   const size_t nqb = s->n / kBlock, heads = (size_t)s->batch * s->hq;
-  if (o.impl == 1 || stride < 1 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv, stride, pg)) return L;  // exact kernel: none
+  if (o.impl == 1 || stride < 1) return L;   // exact kernel: none
+  // pages too small for the screen's strided boxes, or so small that a key tile takes many of them (below 32 sampled
+  // rows per page the copy is cheaper than the extra boxes: 1.8 against 2.0-2.4 ms at 128K): the keys are first
+  // copied into a dense staging tensor
+  const bool gather = pg.table && (pg.page_size / stride < 32 || !kap_screen_supported(kBlock / stride, s->hq / s->hkv, stride, pg));
+  if (gather) pg.table = nullptr;
+  if (!kap_screen_supported(kBlock / stride, s->hq / s->hkv, stride, pg)) return L;
   size_t off = 0;
   L.scores = off; off += align_up(heads * nqb * nqb * 4, 256);
   L.jstar = off; off += align_up(heads * (s->n / stride) * 8, 256);
@@ -122,11 +127,18 @@ static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o)
   L.slots = std::min(L.slots, kap_screen_grid(s->batch, s->hq, s->hkv, (int)nqb, stride));
   L.slot_taken = off; off += align_up((size_t)L.slots * 4, 256);
   L.maxima = off; off += align_up((size_t)L.slots * kap_screen_slot_bytes(s->n, stride), 256);
+  L.gather = gather;
+  if (gather) { L.kstage = off; off += align_up((size_t)s->batch * s->hkv * s->n * s->d * 2, 256); }
   L.total = off;
   return L;
 }
 static size_t kap_scratch_bytes(const cosa_shape* s, const cosa_options& o) { return kap_scratch_layout(s, o).total; }
-static size_t osk_scratch_bytes(const cosa_shape*, const cosa_options&) { return 0; }
+// OSK fetches a key block as one pair of TMA boxes per page: pools whose pages are smaller than a block are copied
+// into dense staging tensors (K, then V) first
+static bool osk_gathers(const cosa_options& o) { return o.kv_page_table && o.impl != 1 && o.kv_page_size < kBlock; }
+static size_t osk_scratch_bytes(const cosa_shape* s, const cosa_options& o) {
+  return osk_gathers(o) ? 2 * align_up((size_t)s->batch * s->hkv * s->n * s->d * 2, 256) : 0;
+}
 
 }  // namespace cosa
 
@@ -223,6 +235,15 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.causal = p.causal; sp.stride = s;
   sp.scale = (float)p.scale;
   sp.tau_row = 1e-4f;
+  if (L.gather) {
+    __nv_bfloat16* staged = reinterpret_cast<__nv_bfloat16*>(ws + L.kstage);
+    cudaError_t ge = launch_gather_pages(p.k, staged, p.pg, p.batch, p.hkv, p.n, st);
+    if (ge != cudaSuccess) return cuda_fail(ge, "page gather launch");
+    p.k = staged; sp.k = staged;
+    const int32_t* lens = p.pg.seq_lens;
+    p.pg = KvPaging{};
+    p.pg.seq_lens = lens;
+  }
   sp.pg = p.pg;
   cudaError_t e = launch_kap_screen(sp, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");
@@ -271,6 +292,27 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   p.skip_scale = o.skip_scale;
   p.scale = o.softmax_scale > 0.f ? o.softmax_scale : (float)(1.0 / sqrt((double)shape->d));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (osk_gathers(o)) {
+    const size_t need = osk_scratch_bytes(shape, o), one = need / 2;
+    char* ws = static_cast<char*>(o.workspace);
+    if (ws) {
+      if (o.workspace_bytes < need || !aligned16(ws)) return COSA_ERR_WORKSPACE;
+    } else {
+      void* own = nullptr;
+      rc = own_scratch(need, &own);
+      if (rc != COSA_OK) return rc;
+      ws = static_cast<char*>(own);
+    }
+    __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(ws);
+    __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(ws + one);
+    cudaError_t ge = launch_gather_pages(p.k, ks, p.pg, p.batch, p.hkv, p.n, st);
+    if (ge == cudaSuccess) ge = launch_gather_pages(p.v, vs, p.pg, p.batch, p.hkv, p.n, st);
+    if (ge != cudaSuccess) return cuda_fail(ge, "page gather launch");
+    p.k = ks; p.v = vs;
+    const int32_t* lens = p.pg.seq_lens;
+    p.pg = KvPaging{};
+    p.pg.seq_lens = lens;
+  }
   cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : launch_osk_tc(p, st);
   if (e != cudaSuccess) return cuda_fail(e, "osk launch");
   return COSA_OK;

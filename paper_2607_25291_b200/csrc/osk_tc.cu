@@ -93,18 +93,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 // physical pages): one pair of boxes of b_p rows per page, looked up in the page table.
 __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensorMap* map, uint32_t dst, int b, int g, int j,
                                               uint32_t bar) {
-  if (!p.pg.table || p.pg.page_size >= kBlock) {
-    const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock);
-    tma_load_2d(dst, map, 0, row, bar);
-    tma_load_2d(dst + kHalfBytes, map, 64, row, bar);
-  } else {
-    const int ps = p.pg.page_size;
-    for (int part = 0; part < kBlock / ps; ++part) {
-      const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock + part * ps);
-      tma_load_2d(dst + part * ps * 128, map, 0, row, bar);
-      tma_load_2d(dst + kHalfBytes + part * ps * 128, map, 64, row, bar);
-    }
-  }
+  // a page holds whole key blocks (pools with smaller pages reach this kernel as dense staging tensors)
+  const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock);
+  tma_load_2d(dst, map, 0, row, bar);
+  tma_load_2d(dst + kHalfBytes, map, 64, row, bar);
 }
 
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
@@ -657,9 +649,10 @@ bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows, int box_r
 
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
   CUtensorMap qm, km, vm, om;
-  // K and V: the dense tensors, or the page pools (boxes of one page when a page is smaller than a block)
+  // K and V: the dense tensors, or page pools whose pages hold whole key blocks
   const uint64_t kv_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * p.pg.page_size : (uint64_t)p.batch * p.hkv * p.n;
-  const int kv_box = (p.pg.table && p.pg.page_size < kBlock) ? p.pg.page_size : kBlock;
+  if (p.pg.table && p.pg.page_size < kBlock) return cudaErrorInvalidValue;   // staged as dense tensors by the caller of this launcher
+  const int kv_box = kBlock;
   if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, kv_rows, kv_box) ||
       !make_tile_map(&vm, p.v, kv_rows, kv_box) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
     return cudaErrorInvalidValue;

@@ -150,7 +150,7 @@ def test_qwen3_32k_and_128k_topp_sampled():
 
 
 def test_qwen3_32k_paged_equals_dense():
-    """Page pools of 64- and 256-token pages (Sec. C.1) against the dense tensors they hold, whole workload."""
+    """Page pools of 16-, 64- and 256-token pages (Sec. C.1) against the dense tensors they hold, whole workload."""
     w = WORKLOADS["qwen3_32k"]
     qb, kb, vb, _ = w.make()
     q, k, v = (to_dev(x) for x in (qb, kb, vb))
@@ -169,7 +169,7 @@ def test_qwen3_32k_paged_equals_dense():
         return order, count, out, vis
 
     dense = run(k, v)
-    for page_size in (64, 256):
+    for page_size in (16, 64, 256):
         kpool, table = scatter_to_pages(kb, page_size, seed=12)
         vpool, _ = scatter_to_pages(vb, page_size, seed=12)
         dev = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).cuda().contiguous()

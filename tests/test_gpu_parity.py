@@ -517,7 +517,7 @@ def _pools(w, page_size):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("page_size", [16, 64, 128, 256])
+@pytest.mark.parametrize("page_size", [8, 16, 32, 64, 128, 256])
 def test_paged_kv_small(small, impl, page_size):
     """Pools + page table give the lists and outputs of the dense tensors behind them (Sec. C.1)."""
     q, k, v = small["dev"]
@@ -546,7 +546,7 @@ def test_paged_kv_small(small, impl, page_size):
 def test_paged_kv_4k(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
-    for page_size in (64, 512):
+    for page_size in (16, 64, 512):
         kpool, vpool, table, n_pages = _pools(w, page_size)
         paging = dict(kv_page_table=table, kv_page_size=page_size, kv_num_pages=n_pages)
         order, count = alloc_lists(w.hq, w.n_blocks)
@@ -570,6 +570,39 @@ def test_paged_kv_rejects_bad_arguments(small):
         args.update(bad)
         with pytest.raises(cosa.CosaError):
             cosa.cosa_kap_select(q, kpool, 0.5, order, count, opt=cosa.default_options(**args))
+
+
+
+def test_paged_kv_small_pages_with_caller_workspace(small):
+    """Pages smaller than a key block are staged as dense tensors in the scratch: a caller-owned workspace of the size
+    the library asks for gives the dense results, a smaller one is refused."""
+    q, k, v = small["dev"]
+    nqb = q.shape[2] // 128
+    kpool, vpool, table, n_pages = _pools(small["w"], 16)
+    paging = dict(kv_page_table=table, kv_page_size=16, kv_num_pages=n_pages)
+    shape = cosa.make_shape(q, k)
+    kv_bytes = k.numel() * 2
+    need = cosa.cosa_workspace_bytes(2, shape, cosa.default_options(**paging))
+    assert need >= 2 * kv_bytes
+    assert cosa.cosa_workspace_bytes(1, shape, cosa.default_options(**paging)) >= 2 * kv_bytes
+    assert cosa.cosa_workspace_bytes(1, shape, cosa.default_options()) == 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    order, count = alloc_lists(q.shape[1], nqb)
+    opt = cosa.default_options(workspace=ws, workspace_bytes=need, **paging)
+    cosa.cosa_kap_select(q, kpool, 0.6, order, count, opt=opt)
+    d_order, d_count = run_kap(q, k, 0.6)
+    assert torch.equal(order, d_order) and torch.equal(count, d_count)
+    bufs = alloc_outputs(q, nqb)
+    cosa.cosa_osk_attention(q, kpool, vpool, order, count, 0.4, bufs["out"], bufs["lse"], bufs["visited"],
+                            opt=cosa.default_options(skip_scale=150.0, workspace=ws, workspace_bytes=need, **paging))
+    assert cosa.cosa_device_status() == 0
+    dense = run_osk(q, k, v, order, count, 0.4, 150.0)
+    assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
+    small_opt = cosa.default_options(workspace=ws, workspace_bytes=kv_bytes, **paging)
+    with pytest.raises(cosa.CosaError):
+        cosa.cosa_kap_select(q, kpool, 0.6, order, count, opt=small_opt)
+    with pytest.raises(cosa.CosaError):
+        cosa.cosa_osk_attention(q, kpool, vpool, order, count, 0.4, bufs["out"], bufs["lse"], bufs["visited"], opt=small_opt)
 
 
 # ---------------------------------------------------------------------------------- batch > 1
