@@ -120,7 +120,7 @@ typedef struct {
                               counts (budget counts, the Stage-2 cap) and the N of the skip rule
                               (Eq. 5; skip_scale must stay below the shortest length) follow the
                               item's own length: every item comes out as in a call of its own.
-                              Not with block_q = 256, not in cosa_prefill_host                      */
+                              Not with block_q = 256                                               */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);
@@ -257,7 +257,8 @@ int cosa_validate_order(const int32_t* order, const int32_t* count, const cosa_s
  * synchronised.  out_lse_host and out_visited_host may be NULL.
  * The call works through the (batch item, KV head) slices one after the other; the copies to and from the
  * device run on two internal streams (created once per device) so that they overlap the kernels of the other
- * slices; `stream` is ordered after all of them.  opt->kv_page_table and opt->logical_mask are ignored.
+ * slices; `stream` is ordered after all of them.  opt->kv_page_table and opt->logical_mask are ignored;
+ * opt->seq_lens (a DEVICE array, as everywhere) is honoured, padding rows are copied like the rest.
  */
 size_t cosa_host_call_workspace_bytes(const cosa_shape* shape, const cosa_options* opt);
 int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host,

@@ -419,7 +419,6 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
   if (rc != COSA_OK) return rc;
   if (!q_host || !k_host || !v_host || !out_host || !device_workspace) return COSA_ERR_INVALID_ARG;
   cosa_options o = resolve_options(opt);
-  if (o.seq_lens) return COSA_ERR_UNSUPPORTED;   // the slices of this call are whole sequences
   HostCallLayout L = host_layout(shape, o);
   if (device_workspace_bytes < L.total || !aligned16(device_workspace)) return COSA_ERR_WORKSPACE;
   char* ws = static_cast<char*>(device_workspace);
@@ -468,9 +467,11 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
     int32_t* count_d = reinterpret_cast<int32_t*>(ws + L.count + c * cnt_chunk);
     int32_t* visited_d = reinterpret_cast<int32_t*>(ws + L.visited + c * cnt_chunk);
     float* lse_d = reinterpret_cast<float*>(ws + L.lse + c * lse_chunk);
-    rc = cosa_kap_select_ex(qd, kd, &sub, budget, order_d, count_d, stream, &o);
+    cosa_options oc = o;
+    if (o.seq_lens) oc.seq_lens = o.seq_lens + c / shape->hkv;   // the slice's batch item (lengths live on the device: padding is copied too)
+    rc = cosa_kap_select_ex(qd, kd, &sub, budget, order_d, count_d, stream, &oc);
     if (rc != COSA_OK) return rc;
-    rc = cosa_osk_attention_ex(qd, kd, vd, &sub, order_d, count_d, tightened_budget, od, lse_d, visited_d, stream, &o);
+    rc = cosa_osk_attention_ex(qd, kd, vd, &sub, order_d, count_d, tightened_budget, od, lse_d, visited_d, stream, &oc);
     if (rc != COSA_OK) return rc;
     if (!order_after(down, st)) return cuda_fail(e, "stream order");
     if ((e = cudaMemcpyAsync(static_cast<char*>(out_host) + c * q_chunk, od, q_chunk, cudaMemcpyDeviceToHost, down)) != cudaSuccess)

@@ -763,3 +763,34 @@ def test_host_call_equals_device_calls(small):
     with pytest.raises(cosa.CosaError) as e:
         cosa.cosa_prefill_host(qh, kh, vh, shape, 0.5, 0.3, out_h, lse_h, vis_h, small_ws, opt=opt)
     assert e.value.status == -3
+
+
+def test_host_call_with_different_lengths():
+    """cosa_prefill_host on a padded batch with per-item lengths gives the device calls' results."""
+    n, lens, hq, hkv = 1024, [640, 1024], 4, 2
+    items = [tiny(seed=71 + b, hq=hq, hkv=hkv, n=n, needles=2).make() for b in range(2)]
+    q = torch.stack([to_dev(it[0])[0] for it in items]).contiguous()
+    k = torch.stack([to_dev(it[1])[0] for it in items]).contiguous()
+    v = torch.stack([to_dev(it[2])[0] for it in items]).contiguous()
+    nqb = n // 128
+    seq_lens = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    order = torch.empty(2, hq, nqb, nqb, dtype=torch.int32, device="cuda")
+    count = torch.empty(2, hq, nqb, dtype=torch.int32, device="cuda")
+    out = torch.empty_like(q)
+    lse = torch.empty(2, hq, n, dtype=torch.float32, device="cuda")
+    vis = torch.empty(2, hq, nqb, dtype=torch.int32, device="cuda")
+    opt = cosa.default_options(skip_scale=100.0, seq_lens=seq_lens)
+    cosa.cosa_kap_select(q, k, 0.5, order, count, opt=opt)
+    cosa.cosa_osk_attention(q, k, v, order, count, 0.3, out, lse, vis, opt=opt)
+    assert cosa.cosa_device_status() == 0
+    shape = cosa.make_shape(q, k, True)
+    ws = torch.empty(cosa.cosa_host_call_workspace_bytes(shape, opt), dtype=torch.uint8, device="cuda")
+    qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
+    out_h = torch.empty(q.shape, dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.empty(lse.shape, dtype=torch.float32).pin_memory()
+    vis_h = torch.empty(vis.shape, dtype=torch.int32).pin_memory()
+    cosa.cosa_prefill_host(qh, kh, vh, shape, 0.5, 0.3, out_h, lse_h, vis_h, ws, opt=opt)
+    assert cosa.cosa_device_status() == 0
+    assert torch.equal(vis_h, vis.cpu()) and torch.equal(out_h, out.cpu())
+    assert torch.equal(lse_h[0, :, :lens[0]], lse.cpu()[0, :, :lens[0]]) and torch.equal(lse_h[1], lse.cpu()[1])
+    assert bool((out_h[0, :, lens[0]:] == 0).all()) and bool((vis_h[0, :, lens[0] // 128:] == 0).all())
