@@ -80,7 +80,9 @@ typedef struct {
   float*  kap_scores;      /* optional [B,Hq,nQB,nQB]: KAP block scores s_ij (Eq. 11), j <= i    */
   uint8_t* kap_flags;      /* optional [B,Hq,nQB,nQB]: HRM flags h_ij (Eq. 12)                   */
   void*   workspace;       /* device scratch; NULL -> the library's own per-device scratch,
-                              which is allocated (cudaMalloc) on first use or growth             */
+                              which is allocated (cudaMalloc) on first use or growth and shared
+                              by every such call on the device: calls that may overlap on
+                              different streams must each bring a workspace of their own          */
   size_t  workspace_bytes;
   int32_t impl;            /* 0 = fastest available; 1 = plain CUDA-core check kernels; 2 and 3 = as 0,
                               but the sort stage of cosa_kap_select takes the route it otherwise
