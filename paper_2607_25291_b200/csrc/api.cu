@@ -237,7 +237,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.tau_row = 1e-4f;
   if (L.gather) {
     __nv_bfloat16* staged = reinterpret_cast<__nv_bfloat16*>(ws + L.kstage);
-    cudaError_t ge = launch_gather_pages(p.k, staged, p.pg, p.batch, p.hkv, p.n, st);
+    cudaError_t ge = launch_gather_pages(p.k, staged, p.pg, p.batch, p.hkv, p.n, s, st);   // the sampled rows are all KAP reads
     if (ge != cudaSuccess) return cuda_fail(ge, "page gather launch");
     p.k = staged; sp.k = staged;
     const int32_t* lens = p.pg.seq_lens;
@@ -305,8 +305,8 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
     }
     __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(ws);
     __nv_bfloat16* vs = reinterpret_cast<__nv_bfloat16*>(ws + one);
-    cudaError_t ge = launch_gather_pages(p.k, ks, p.pg, p.batch, p.hkv, p.n, st);
-    if (ge == cudaSuccess) ge = launch_gather_pages(p.v, vs, p.pg, p.batch, p.hkv, p.n, st);
+    cudaError_t ge = launch_gather_pages(p.k, ks, p.pg, p.batch, p.hkv, p.n, 1, st);
+    if (ge == cudaSuccess) ge = launch_gather_pages(p.v, vs, p.pg, p.batch, p.hkv, p.n, 1, st);
     if (ge != cudaSuccess) return cuda_fail(ge, "page gather launch");
     p.k = ks; p.v = vs;
     const int32_t* lens = p.pg.seq_lens;

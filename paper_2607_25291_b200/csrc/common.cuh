@@ -171,9 +171,10 @@ size_t kap_screen_slot_bytes(int n, int stride);
 // sorts the screened scores, recomputes near-ties in double precision, writes the lists
 cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float tau_score, cudaStream_t st);
 size_t kap_exact_smem_bytes(int rows, int nqb, int qtiles);
-// copies the pages of the call's sequences into a dense [B, Hkv, N, d] tensor (pools with pages smaller than a key block)
+// copies the pages of the call's sequences into a dense [B, Hkv, N, d] tensor (pools with pages smaller than a key block);
+// every > 1: only the rows whose token index is a multiple of it
 cudaError_t launch_gather_pages(const __nv_bfloat16* pool, __nv_bfloat16* dense, const KvPaging& pg, int batch, int hkv, int n,
-                                cudaStream_t st);
+                                int every, cudaStream_t st);
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
 cudaError_t launch_reorder_lists(int32_t* order, const int32_t* count, int total_qb, int order_stride, int descending,

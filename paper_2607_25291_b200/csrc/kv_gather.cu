@@ -9,32 +9,35 @@
 namespace cosa {
 namespace {
 
-// one 16-byte chunk per thread and step; a row of d = 128 bf16 has 16 chunks
+// one 16-byte chunk per thread and turn; a row of d = 128 bf16 has 16 chunks.  every: copy only the rows whose token
+// index is a multiple of it (KAP reads nothing but its sampled rows; the other rows of the staging tensor stay unwritten)
 __global__ void __launch_bounds__(256) gather_pages_kernel(const uint4* __restrict__ pool, uint4* __restrict__ dense, KvPaging pg,
-                                                           int batch, int hkv, int n) {
+                                                           int batch, int hkv, int n, int every) {
   constexpr int kChunks = kHeadDim * 2 / 16;
-  const long long total = (long long)batch * hkv * n * kChunks;
+  const int rows = n / every;
+  const long long total = (long long)batch * hkv * rows * kChunks;
   for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (long long)gridDim.x * blockDim.x) {
     const int c = (int)(idx % kChunks);
-    const long long row = idx / kChunks;            // ((b * hkv) + g) * n + token
-    const int token = (int)(row % n);
-    const int bg = (int)(row / n);
+    const long long row = idx / kChunks;            // ((b * hkv) + g) * rows + token / every
+    const int token = (int)(row % rows) * every;
+    const int bg = (int)(row / rows);
     const int b = bg / hkv, g = bg % hkv;
     if (pg.seq_lens && token >= pg.seq_lens[b]) continue;   // padding: never read as keys
     const long long src = kv_row(pg, b, hkv, g, n, token);
-    dense[idx] = pool[src * kChunks + c];
+    dense[((long long)bg * n + token) * kChunks + c] = pool[src * kChunks + c];
   }
 }
 
 }  // namespace
 
 cudaError_t launch_gather_pages(const __nv_bfloat16* pool, __nv_bfloat16* dense, const KvPaging& pg, int batch, int hkv, int n,
-                                cudaStream_t st) {
-  const long long total = (long long)batch * hkv * n * (kHeadDim * 2 / 16);
+                                int every, cudaStream_t st) {
+  if (every < 1 || n % every != 0) return cudaErrorInvalidValue;
+  const long long total = (long long)batch * hkv * (n / every) * (kHeadDim * 2 / 16);
   long long blocks = (total + 255) / 256;
   if (blocks > 148LL * 32) blocks = 148LL * 32;
   gather_pages_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const uint4*>(pool), reinterpret_cast<uint4*>(dense), pg,
-                                                       batch, hkv, n);
+                                                       batch, hkv, n, every);
   return cudaGetLastError();
 }
 
