@@ -70,8 +70,10 @@ typedef struct {
 typedef struct {
   int32_t stride;          /* KAP sampling stride s: sampled row r is token r*s; power of two,
                               1 <= s <= 128; default 8                                           */
-  float   skip_scale;      /* Delta of Eq. (5); <= 0 disables the threshold test (the paper's
-                              Delta = -1); must be < N otherwise; default 2000                   */
+  float   skip_scale;      /* Delta of Eq. (5).  < 0 disables the threshold test (the paper's
+                              Delta = -1); 0 stands for the default, 2000; a positive value must be
+                              < N (with seq_lens: a batch item no longer than Delta runs with the
+                              test off, since ln(Delta/N) >= 0 would skip its first block)      */
   float   softmax_scale;   /* 0 -> 1/sqrt(d)                                                     */
   int32_t order_stride;    /* row pitch of the order tensor in elements; 0 -> nQB                */
   int32_t* out_scored;     /* optional [B,Hq,nQB]: blocks whose logits OSK formed                */
@@ -123,6 +125,11 @@ typedef struct {
                               (Eq. 5; skip_scale must stay below the shortest length) follow the
                               item's own length: every item comes out as in a call of its own.
                               Not with block_q = 256                                               */
+  int64_t wait_cycles;     /* Clock cycles a wait inside a kernel may take before the kernel gives up, sets the
+                              device status word (see cosa_device_status) and returns without writing further
+                              results.  0: the default, 2^31 (about a second).  A few cycles make every
+                              wait that is not already satisfied run out: that is how the tests reach this path
+                              without ever leaving a kernel waiting                                       */
 } cosa_options;
 
 void cosa_default_options(cosa_options* opt);
@@ -186,8 +193,14 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape,
  *   - Arguments and results are those of cosa_kap_select_ex; opt->workspace is ignored.  Inputs and
  *     outputs are still the caller's buffers.
  *   - Returns COSA_ERR_WORKSPACE, and enqueues nothing, when cosa_workspace_bytes(0, shape, opt)
- *     exceeds the array: roughly B*Hq*(N/128)^2*4 bytes, e.g. 8 heads at N = 16384 fit, 32 heads at
- *     N = 32768 do not.
+ *     exceeds the array.  Two terms make up that figure: the screened scores, B*Hq*(N/128)^2*4 bytes,
+ *     and the screen kernel's parked block maxima, one area of ceil(N/s/128)*256*(128/R)*4 bytes
+ *     (R = 128/s sampled rows per block) for every CTA of that kernel that can be resident, i.e.
+ *     min(SM count, CTAs of the call); the second term dominates.  With stride 8 on a 148-SM part:
+ *     32 query / 8 KV heads at N = 4096 need 2.3 MiB and fit; the same heads at N = 8192 need 10 MiB
+ *     and 8 query / 2 KV heads at N = 16384 need 8.6 MiB: both are refused.  To know beforehand, ask
+ *     cosa_workspace_bytes(0, shape, opt) <= cosa_kap_select_static_max_bytes() with the device
+ *     current on which the call will run.
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call before starting any stream capture.
  *   - All calls on one device share the array, which keeps whatever the last call left in it; the

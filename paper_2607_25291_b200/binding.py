@@ -9,7 +9,6 @@ raised.
 from __future__ import annotations
 
 import ctypes
-import math
 import os
 from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int, c_int32, c_size_t, c_uint8, c_uint32, c_void_p
 
@@ -44,7 +43,7 @@ class CosaOptions(Structure):
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p), ("kv_page_table", c_void_p),
-                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p)]
+                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p), ("wait_cycles", ctypes.c_int64)]
 
 
 class CosaError(RuntimeError):

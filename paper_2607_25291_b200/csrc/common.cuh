@@ -106,6 +106,7 @@ struct OskParams {
   float theta;           // ln(Delta / N)
   float skip_scale;      // Delta (for items whose own length replaces N, see item_theta)
   float scale;           // softmax scale
+  long long wait_budget; // clock cycles a device-side wait may take before the kernel gives up
   KvPaging pg;
 };
 

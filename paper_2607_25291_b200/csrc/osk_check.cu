@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
     __syncthreads();
     if (t == 0) {
       float gm = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
-      s_skip = (p.use_threshold && gm < theta) ? 1 : 0;
+      s_skip = (p.use_threshold && theta < 0.f && gm < theta) ? 1 : 0;   // theta >= 0 (an item no longer than Delta): test off
     }
     __syncthreads();
     const bool skip = s_skip != 0;

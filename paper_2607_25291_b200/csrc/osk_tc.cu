@@ -8,8 +8,9 @@
 //   warp 1       QK issuer: S = Q K_j^T into one of two TMEM buffers
 //   warp 3       PV issuer: O += P V_j.  Two issuing threads, because a single thread's
 //                instruction stream (descriptors, barrier tests, commits) is what limits how fast
-//                MMAs reach the tensor pipe.  Both products take their A operand (Q, resp. P) from
-//                tensor memory: with both operands in shared memory the QK^T product ran slower.
+//                MMAs reach the tensor pipe.  Q K^T takes both operands from shared memory, P V its A
+//                operand from tensor memory, where P has two buffers: the probabilities of the next
+//                computed block are stored while the product of the previous one still runs.
 //   warp 2       controller (see below)
 //   warps 4..7   softmax group A: list positions 0, 2, 4, ...   (one thread per query row)
 //   warps 8..11  softmax group B: list positions 1, 3, 5, ...
@@ -23,14 +24,15 @@
 //                the cap on computed blocks, the V tile load of computed blocks, and the
 //                decisions the other warps follow
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
-// expect; the Q tile is fetched by TMA as well and copied from shared memory into TMEM by the first group.
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P [384,448) Q [448,512).
+// expect; the Q tile is fetched by TMA as well and stays in shared memory.
+// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
 // down without writing results.
 #include <math.h>
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "tile_maps.cuh"
 
 namespace cosa {
 namespace {
@@ -48,12 +50,12 @@ constexpr int kSpec = 2;   // K tiles fetched and products issued ahead of the b
                            // binds, certainty grows one block per decision and each block would otherwise wait out a full
                            // tile fetch + product (at most 2: the S buffer of position kk is freed by position kk-2)
 constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks before this position
-constexpr long long kWaitBudget = 1LL << 31;       // clock cycles (about a second)
 
 struct __align__(8) Control {
-  unsigned long long q_stage, q_full, k_full[kKStages], v_full[kVStages];   // Q tile landed / Q copied into TMEM
+  unsigned long long q_stage, k_full[kKStages], v_full[kVStages];   // q_stage: the Q tile has landed
   unsigned long long k_empty[kKStages];  // QK^T of that stage finished: the stage is free AND its S tile is ready
-  unsigned long long s_empty[2], p_full;
+  unsigned long long s_empty[2];
+  unsigned long long p_full[2];   // P of computed block n is in buffer n & 1
   unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1] (P free, O updated, V stage n & 1 free); two
                                   // barriers because a waiter may run two products ahead of the tensor pipe, which one
                                   // barrier's single parity bit cannot tell apart
@@ -158,16 +160,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   if (threadIdx.x == 0) {
     // barriers first, then the Q tile at once: its address needs nothing from global memory, while the list
     // entries, the count and the status word requested above are still on their way (2 k cycles at the start of a CTA)
-    mbar_init(smem_u32(&ctl->q_stage), 1); mbar_init(smem_u32(&ctl->q_full), kBlock);
+    mbar_init(smem_u32(&ctl->q_stage), 1);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&ctl->v_full[s]), 1);
       mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
       mbar_init(smem_u32(&ctl->m_ready[s]), kBlock); mbar_init(smem_u32(&ctl->dec_bar[s]), 1);
       mbar_init(smem_u32(&ctl->p_empty[s]), 1);
+      mbar_init(smem_u32(&ctl->p_full[s]), kBlock);
     }
     mbar_init(smem_u32(&ctl->out_bar), kBlock);
-    mbar_init(smem_u32(&ctl->p_full), kBlock);
     mbar_init(smem_u32(&ctl->fin_bar), kBlock);
     ctl->n_dec = 0;
     ctl->end_kk = -1;
@@ -202,18 +204,20 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   tc_fence_after();
   if (ctl->poisoned != 0) {
     if (warp == 1) tmem_dealloc(ctl->tmem_base, kTmemCols);
-    if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&ctl->q_stage), 0, &ctl->abort_flag);   // no copy may be in flight when the CTA retires
+    if (threadIdx.x == 0) (void)mbar_wait_noabort(smem_u32(&ctl->q_stage), 0);   // no copy may be in flight when the CTA retires
     return;
   }
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
-  const uint32_t tmem_p = tmem + 384u;
-  const uint32_t tmem_q = tmem + 448u;
+  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 448u};
   volatile int* abort_flag = &ctl->abort_flag;
+  const long long budget = p.wait_budget;
   const float kLog2e = 1.4426950408889634f;
   const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
   const float theta2 = (p.use_threshold ? item_theta(p.pg, b, p.theta, p.skip_scale, nqb_b) : 0.f) * kLog2e;
+  // a batch item no longer than Delta would have ln(Delta/N) >= 0 and lose even its first block: the test is off for it
+  const bool thr_on = p.use_threshold && theta2 < 0.f;
 
   // register budget: the control warps need few, the softmax threads hold a whole S row
   if (warp < 4) {
@@ -228,12 +232,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         bool ok = true;
         while (kk >= ctl->n_needed + kSpec) {  // at most kSpec tiles beyond the blocks that are certain to be scored
           if (ctl->end_kk >= 0) { ok = false; break; }
-          if (*abort_flag || clock64() - t0 > kWaitBudget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+          if (*abort_flag || clock64() - t0 > budget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           __nanosleep(32);
         }
         if (!ok || ctl->end_kk >= 0) break;
         const int st = kk % kKStages;
-        if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag)) {
+        if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag, budget)) {
           if (!*abort_flag) report_timeout(ctl, status);
           break;
         }
@@ -246,14 +250,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       ctl->k_loaded = last_issued + 1;       // the QK issuer must not wait for a tile beyond these
       // tiles fetched ahead may never be multiplied: their copies must have landed before the CTA retires
       for (int kk = max(0, last_issued - (kKStages - 1)); kk <= last_issued; ++kk)
-        if (!mbar_wait(smem_u32(&ctl->k_full[kk % kKStages]), (kk / kKStages) & 1, abort_flag) && !*abort_flag) report_timeout(ctl, status);
+        if (!mbar_wait_noabort(smem_u32(&ctl->k_full[kk % kKStages]), (kk / kKStages) & 1) && !*abort_flag) report_timeout(ctl, status);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ QK issuer
     if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] from TMEM, K_j [N x K] K-major
-      bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag);
+      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] and K_j [N x K], both K-major in shared memory
+      bool alive = mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag, budget);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
+      const uint64_t qdesc = smem_desc_sw128(q_sm, 16, 1024);
       const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
       int last_issued = -1;
       int n_certain = 0;        // a copy of n_needed, which only grows: positions below it are certain to be scored
@@ -268,7 +273,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
               bool ended = false;
               while (kk >= (n_certain = ctl->n_needed) + kSpec) {
                 if (ctl->end_kk >= 0) { ended = true; break; }
-                if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+                if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
                 __nanosleep(20);   // a bare spin here takes issue slots from the two softmax warps of this sub-partition (1 % of the kernel)
               }
               if (ended || !alive) break;
@@ -283,12 +288,12 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
               while (!mbar_try_wait(bar, par)) {
                 const int kl = ctl->k_loaded;
                 if (kl >= 0 && kk >= kl) { none = true; break; }
-                if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+                if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
               }
             }
             if (none || !alive) break;
           }
-          alive = mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag);
+          alive = mbar_wait(smem_u32(&ctl->s_empty[sb]), ((kk >> 1) & 1) ^ 1, abort_flag, budget);
           if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         }
         // Issuing a product keeps this thread busy for about as long as the product runs, so whatever is checked
@@ -301,14 +306,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         }
         tc_fence_after();
         // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
-        mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
-            tmem_s[sb], tmem_q, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk, false);
+        mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+            tmem_s[sb], qdesc, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk);
         mma_commit(smem_u32(&ctl->k_empty[st]));
         last_issued = kk;
       }
       // a product issued ahead of the walk's end may still be running: it must finish before TMEM is released
       if (alive && last_issued >= 0 &&
-          !mbar_wait(smem_u32(&ctl->k_empty[last_issued % kKStages]), (last_issued / kKStages) & 1, abort_flag) && !*abort_flag)
+          !mbar_wait(smem_u32(&ctl->k_empty[last_issued % kKStages]), (last_issued / kKStages) & 1, abort_flag, budget) && !*abort_flag)
         report_timeout(ctl, status);
     }
   } else if (warp == 3) {
@@ -319,22 +324,22 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       bool alive = true;
       for (int n = 0; alive; ++n) {
         // the next computed block's P, or the end of the walk
-        const uint32_t bar = smem_u32(&ctl->p_full), par = n & 1;
+        const uint32_t bar = smem_u32(&ctl->p_full[n & 1]), par = (n >> 1) & 1;
         bool done = false;
         if (!mbar_try_wait(bar, par)) {
           const long long t0 = clock64();
           while (!mbar_try_wait(bar, par)) {
             if (ctl->end_kk >= 0 && n >= ctl->final_computed) { done = true; break; }
-            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+            if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
         if (done || !alive) break;
         const int vs = n % kVStages;
-        alive = mbar_wait(smem_u32(&ctl->v_full[vs]), (n / kVStages) & 1, abort_flag);
+        alive = mbar_wait(smem_u32(&ctl->v_full[vs]), (n / kVStages) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
         // 16 keys per MMA: 8 TMEM columns of P, 2 KiB (two 8-key groups) of the V tile
-        mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p, vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
+        mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p[n & 1], vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
         mma_commit(smem_u32(&ctl->p_empty[n & 1]));
       }
     }
@@ -347,13 +352,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int par = kk & 1;
       const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
-      alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag);
+      alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
       // The statistic is <= 0, so among bit patterns the smallest unsigned word is the largest value.
       const volatile unsigned* gw = ctl->gapw[par];
       const float gm = __uint_as_float(min(min(gw[0], gw[1]), min(gw[2], gw[3])));
-      const bool compute = !(p.use_threshold && gm < theta2);
+      const bool compute = !(thr_on && gm < theta2);
       ++scored;
       const int n_before = computed;
       if (compute) ++computed; else n_needed = min(cnt, n_needed + 1);
@@ -368,7 +373,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         if (last) ctl->end_kk = kk;
         if (compute) {                            // fetch V_j now that the block is known to be computed
           const int vs = n_before % kVStages;
-          if (!mbar_wait(smem_u32(&ctl->p_empty[vs]), ((n_before >> 1) & 1) ^ 1, abort_flag)) {   // PV n-2 read this stage
+          if (!mbar_wait(smem_u32(&ctl->p_empty[vs]), ((n_before >> 1) & 1) ^ 1, abort_flag, budget)) {   // PV n-2 read this stage
             if (!*abort_flag) report_timeout(ctl, status);
           } else {
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
@@ -400,7 +405,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (threadIdx.x == 128) {
         if (p.visited) p.visited[row] = 0;
         if (p.scored) p.scored[row] = 0;
-        if (!mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag) && !*abort_flag) report_timeout(ctl, status);   // the Q tile was requested all the same
+        if (!mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag, budget) && !*abort_flag) report_timeout(ctl, status);   // the Q tile was requested all the same
       }
     }
   } else {
@@ -412,23 +417,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     float m_ref = -INFINITY, l = 0.f;         // this group's partial row sum and the maximum it refers to
     bool alive = true;
     uint32_t s[kBlock];                       // this row's raw logits, then probabilities
-    if (grp == 0) {
-      // Q row: shared memory (TMA box layout, 16-byte chunks swizzled by row) -> TMEM as the A operand of
-      // QK^T: lane = row, two consecutive d per 32-bit column
-      alive = mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag);
-      if (!alive && !*abort_flag) report_timeout(ctl, status);
-      const unsigned char* qs = smem + (size_t)kTileBytes * (kKStages + kVStages);
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const uint4 wv = *reinterpret_cast<const uint4*>(qs + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
-        s[4 * c] = wv.x; s[4 * c + 1] = wv.y; s[4 * c + 2] = wv.z; s[4 * c + 3] = wv.w;
-      }
-      tmem_st32(tmem_q + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_st32(tmem_q + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->q_full));
-    }
     // only "is this the diagonal block" matters to a group; an ascending mask walk meets it last, if at all.  The list
     // entry of a position is requested one turn ahead: its latency (some 400 cycles) would otherwise sit between a
     // decision and the group's next S tile
@@ -446,7 +434,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           while (!mbar_try_wait(bar, par)) {
             const int e = ctl->end_kk;
             if (e >= 0 && kk > e) { ended = true; break; }
-            if (*abort_flag || clock64() - t0 > kWaitBudget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
+            if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
         if (ended || !alive) break;
@@ -474,14 +462,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
       //      walk gets here at all (n_needed only grows: an old value merely costs this wait)
       if (kk >= ctl->n_needed) {
-        alive = mbar_wait(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag);
+        alive = mbar_wait(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         if (ctl->dec[(kk - 1) % kDecRing] & kDecEnd) break;
       }
       // ---- running maximum before this position comes from the other group
       float m_in = -INFINITY;
       if (kk > 0) {
-        alive = mbar_wait(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag);
+        alive = mbar_wait(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         m_in = ctl->mrow[grp ^ 1][r];
       }
@@ -492,7 +480,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       ctl->mrow[grp][r] = m_new;
       mbar_arrive(smem_u32(&ctl->m_ready[grp]));
       // ---- the controller's decision
-      alive = mbar_wait(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag);
+      alive = mbar_wait(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget);
       if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
       const uint32_t d = ctl->dec[kk % kDecRing];
       const bool last = (d & kDecEnd) != 0;
@@ -524,28 +512,32 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       }
 #pragma unroll
       for (int c = 0; c < 64; ++c) s[c] = pack_bf16(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1]));
-      // ---- the previous PV product must have finished: P is free and O may be rescaled
-      if (n_before > 0) {
-        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag);
+      // ---- P has two buffers: the product before last must have finished with this one; O is rescaled only if a row
+      //      maximum moved, and only then must the previous product have finished as well
+      if (n_before > 1) {
+        alive = mbar_wait(smem_u32(&ctl->p_empty[n_before & 1]), ((n_before - 2) >> 1) & 1, abort_flag, budget);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+      }
+      if (n_before > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O
+        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O, only if a row maximum moved
-          uint32_t o[32];
+        uint32_t o[32];
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_o + lane_addr + c * 32, o);
-            tmem_wait_ld();
+        for (int c = 0; c < 4; ++c) {
+          tmem_ld32(tmem_o + lane_addr + c * 32, o);
+          tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-            tmem_st32(tmem_o + lane_addr + c * 32, o);
-          }
+          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+          tmem_st32(tmem_o + lane_addr + c * 32, o);
         }
       }
-      tmem_st32(tmem_p + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_st32(tmem_p + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tc_fence_after();
+      tmem_st32(tmem_p[n_before & 1] + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_st32(tmem_p[n_before & 1] + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->p_full));
+      mbar_arrive(smem_u32(&ctl->p_full[n_before & 1]));
       l = l * ex2_approx(m_ref - m_new) + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
       m_ref = m_new;
       if (last) break;
@@ -557,7 +549,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       mbar_arrive(smem_u32(&ctl->fin_bar));
     } else {
       if (alive) {
-        alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag);
+        alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag, budget);
         if (!alive && !*abort_flag) report_timeout(ctl, status);
       }
       if (alive && !*abort_flag) {
@@ -566,7 +558,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const float lt = l * ex2_approx(m_ref - mf) + ctl->fin_l[r] * ex2_approx(mb - mf);
         const int n_comp = ctl->final_computed;
         if (n_comp > 0) {
-          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag);
+          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag, budget);
           if (!alive && !*abort_flag) report_timeout(ctl, status);
         }
         if (alive) {
@@ -597,7 +589,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           mbar_arrive(smem_u32(&ctl->out_bar));
           if (p.lse) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
           if (r == 0) {
-            if (mbar_wait(smem_u32(&ctl->out_bar), 0, abort_flag)) {
+            if (mbar_wait(smem_u32(&ctl->out_bar), 0, abort_flag, budget)) {
               tma_store_2d(&o_map, 0, q_row0, k_sm);
               tma_store_2d(&o_map, 64, q_row0, k_sm + kHalfBytes);
               tma_store_commit_and_wait_read();
@@ -613,36 +605,6 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-// [rows, 128] bf16 row-major viewed as boxes of 128 rows x 64 columns with the 128-byte swizzle
-bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows, int box_rows = kBlock) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(basep), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS;
 }
 
 }  // namespace
