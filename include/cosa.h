@@ -287,6 +287,11 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
  * no further results), then clears it. */
 int cosa_device_status(void* stream);
 
+/* For tests of the error path: writes `status` into the device status word of the current device (synchronously),
+ * as a kernel whose wait ran out would.  Kernels that start while the word is non-zero return at once and leave
+ * their outputs untouched; cosa_device_status() reports the value and clears it. */
+int cosa_debug_set_device_status(int status);
+
 /* Text of the last failing CUDA runtime call on this thread ("" if none). */
 const char* cosa_last_cuda_error(void);
 const char* cosa_status_string(int status);

@@ -28,7 +28,7 @@ COSA_ERR_BAD_ORDER = -6
 EXPORTS = (
     "cosa_default_options", "cosa_workspace_bytes", "cosa_budget_count", "cosa_kap_select",
     "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_reorder_lists", "cosa_lists_to_mask", "cosa_validate_order",
-    "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status", "cosa_options_bytes", "cosa_shape_bytes",
+    "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status", "cosa_debug_set_device_status", "cosa_options_bytes", "cosa_shape_bytes",
     "cosa_last_cuda_error", "cosa_status_string", "cosa_version",
 )
 
@@ -94,6 +94,8 @@ def _load():
     lib.cosa_prefill_host.argtypes = [c_void_p, c_void_p, c_void_p, POINTER(CosaShape), c_float, c_float, c_void_p,
                                       c_void_p, c_void_p, c_void_p, c_size_t, c_void_p, POINTER(CosaOptions)]
     lib.cosa_device_status.argtypes = [c_void_p]
+    lib.cosa_debug_set_device_status.argtypes = [c_int]
+    lib.cosa_debug_set_device_status.restype = c_int
     lib.cosa_last_cuda_error.restype = c_char_p
     lib.cosa_status_string.argtypes = [c_int]
     lib.cosa_status_string.restype = c_char_p
@@ -254,6 +256,12 @@ def cosa_prefill_host(q_host, k_host, v_host, shape: CosaShape, budget: float, t
 
 def cosa_device_status(stream=None) -> int:
     return int(_load().cosa_device_status(_stream_ptr(stream)))
+
+
+def cosa_debug_set_device_status(status: int) -> None:
+    rc = _load().cosa_debug_set_device_status(int(status))
+    if rc != 0:
+        raise CosaError(rc, "cosa_debug_set_device_status")
 
 
 def cosa_version() -> int:

@@ -235,6 +235,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.causal = p.causal; sp.stride = s;
   sp.scale = (float)p.scale;
   sp.tau_row = 1e-4f;
+  sp.wait_budget = o.wait_cycles > 0 ? (long long)o.wait_cycles : (1LL << 31);
   if (L.gather) {
     __nv_bfloat16* staged = reinterpret_cast<__nv_bfloat16*>(ws + L.kstage);
     cudaError_t ge = launch_gather_pages(p.k, staged, p.pg, p.batch, p.hkv, p.n, s, st);   // the sampled rows are all KAP reads
@@ -498,6 +499,13 @@ int cosa_device_status(void* stream) {
     if (e != cudaSuccess) return cuda_fail(e, "clear status");
   }
   return word;
+}
+
+int cosa_debug_set_device_status(int status) {
+  int32_t word = status;
+  cudaError_t e = cudaMemcpyToSymbol(g_status_word, &word, sizeof(word));
+  if (e != cudaSuccess) return cuda_fail(e, "set status");
+  return COSA_OK;
 }
 
 const char* cosa_last_cuda_error(void) { return tl_cuda_error; }

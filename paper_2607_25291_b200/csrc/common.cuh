@@ -82,6 +82,7 @@ struct KapScreenParams {
   int stride;
   float scale;
   float tau_row;         // two block maxima of a row closer than this (scaled logits) are "too close to call"
+  long long wait_budget; // clock cycles a device-side wait may take before the kernel gives up
   KvPaging pg;
 };
 

@@ -28,7 +28,8 @@ __global__ void __launch_bounds__(kThreads) kap_exact_kernel(KapParams p, int kb
 
 // 1-d grid: the CTAs share out the entries of a redo list (usually empty)
 __global__ void __launch_bounds__(kThreads) kap_exact_list_kernel(KapParams p, const int32_t* redo_list, int kb_per_iter,
-                                                                 int sort_cap) {
+                                                                 int sort_cap, const int32_t* status) {
+  if (*reinterpret_cast<const volatile int32_t*>(status) != 0) return;   // an earlier kernel of the call gave up: the list is not to be trusted
   const int n = redo_list[0];
   for (int e = blockIdx.x; e < n; e += gridDim.x) {
     const int flat = redo_list[1 + e];
@@ -234,7 +235,9 @@ cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaS
   if (redo_list) {
     cudaError_t e = cudaFuncSetAttribute(kap_exact_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kap_exact_list_kernel<<<148, kThreads, smem, st>>>(p, redo_list, kb_per_iter_for(p.rows), next_pow2(p.nqb));
+    const int32_t* status = device_status_word();
+    if (!status) return cudaErrorInvalidSymbol;
+    kap_exact_list_kernel<<<148, kThreads, smem, st>>>(p, redo_list, kb_per_iter_for(p.rows), next_pow2(p.nqb), status);
     return cudaGetLastError();
   }
   cudaError_t e = cudaFuncSetAttribute(kap_exact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -53,6 +53,7 @@ struct __align__(8) ScreenCtl {
   unsigned long long m_full[kStages], m_empty[kStages];   // parked maxima fetched back into a key stage / read by all
   uint32_t tmem_base;
   volatile int abort_flag;
+  volatile int t_issued, t_done, c_fetched, c_done;   // key tiles requested / multiplied, chunks of parked maxima requested / read
   int slot;                             // scratch area held by this CTA, -1 = none
   int poisoned;
   float xt[kParts][3][kRows];           // exchange between the column parts: top-3 block maxima
@@ -128,6 +129,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     mbar_init(smem_u32(&ctl->x_bar), kEpiThreads);
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&ctl->m_full[s]), 1); mbar_init(smem_u32(&ctl->m_empty[s]), kEpiThreads); }
     ctl->abort_flag = 0;
+    ctl->t_issued = 0; ctl->t_done = 0; ctl->c_fetched = 0; ctl->c_done = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
     prefetch_tensormap(&q_map); prefetch_tensormap(&k_map);
@@ -138,8 +140,10 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort_flag;
+  const long long budget = p.wait_budget;
 
   if (warp == 0) {
+    int t_issued = 0;   // (lane 0) key tiles requested so far
     if (lane == 0) {
       // A tiles: one strided box of R sampled rows per (query block, query head of the group)
       mbar_expect_tx(smem_u32(&ctl->a_full), kRowTiles * kTileBytes);
@@ -154,7 +158,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const int krow0 = (b * p.hkv + g) * ns;
         for (int t = 0; t < n_tiles; ++t) {
           const int st = t % kStages;
-          if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag)) {
+          if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag, budget)) {
             if (!*abort_flag) screen_timeout(ctl, status);
             break;
           }
@@ -162,6 +166,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           mbar_expect_tx(bar, kTileBytes);
           tma_load_2d(dst, &k_map, 0, krow0 + t * 128, bar);
           tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + t * 128, bar);
+          t_issued = t + 1;
         }
       }
     }
@@ -176,7 +181,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
         int ok = 1;
         if (lane == 0) {
-          ok = mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag) ? 1 : 0;
+          ok = mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag, budget) ? 1 : 0;
           if (!ok && !*abort_flag) screen_timeout(ctl, status);
           if (ok) mbar_expect_tx(bar, kTileBytes);
         }
@@ -190,17 +195,20 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           tma_load_2d(dst + kHalfBytes + lane * spp * 128, &k_map, 64, srow, bar);
         }
         __syncwarp();
+        t_issued = t + 1;
       }
     }
+    if (lane == 0) ctl->t_issued = t_issued;
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16(128, 128, 0, 0);
-      bool alive = mbar_wait(smem_u32(&ctl->a_full), 0, abort_flag);
+      bool alive = mbar_wait(smem_u32(&ctl->a_full), 0, abort_flag, budget);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
+      int t_done = 0;
       for (int t = 0; t < n_tiles && alive; ++t) {
         const int st = t % kStages, sb = t % kSteps;
-        alive = mbar_wait(smem_u32(&ctl->k_full[st]), (t / kStages) & 1, abort_flag) &&
-                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t / kSteps) & 1) ^ 1, abort_flag);
+        alive = mbar_wait(smem_u32(&ctl->k_full[st]), (t / kStages) & 1, abort_flag, budget) &&
+                mbar_wait(smem_u32(&ctl->s_empty[sb]), ((t / kSteps) & 1) ^ 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         tc_fence_after();
         const uint64_t kdesc = smem_desc_sw128(k_sm + st * kTileBytes, 16, 1024);
@@ -209,7 +217,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
               tmem + (sb * kRowTiles + rt) * 128, smem_desc_sw128(a_sm + rt * kTileBytes, 16, 1024), kdesc, idesc);
         mma_commit(smem_u32(&ctl->k_empty[st]));
+        t_done = t + 1;
       }
+      ctl->t_done = t_done;
     }
   } else {
     // ---------------------------------------------------------------- kParts threads per sampled query row
@@ -236,7 +246,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     bool alive = true;
     for (int t = 0; t < n_tiles && alive; ++t) {
       const int sb = t % kSteps, st = t % kStages;
-      alive = mbar_wait(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag);   // this tile's MMAs finished
+      alive = mbar_wait_warp(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag, budget);   // this tile's MMAs finished
       if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
       tc_fence_after();
       uint32_t v[kPartCols / 32][32];
@@ -282,7 +292,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       ctl->xt[part][0][row] = top1; ctl->xt[part][1][row] = top2; ctl->xt[part][2][row] = top3;
       ctl->xj[part][0][row] = jstar; ctl->xj[part][1][row] = jstar2;
       mbar_arrive(smem_u32(&ctl->x_bar));
-      alive = mbar_wait(smem_u32(&ctl->x_bar), 0, abort_flag);
+      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 0, abort_flag, budget);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
     }
     if (alive) {
@@ -318,7 +328,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       // every row's M* in shared memory and every parked maximum visible to the whole CTA
       __threadfence_block();
       mbar_arrive(smem_u32(&ctl->x_bar));
-      alive = mbar_wait(smem_u32(&ctl->x_bar), 1, abort_flag);
+      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 1, abort_flag, budget);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
     }
     if (alive) {
@@ -332,7 +342,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       static_assert(kTilesPerChunk >= 1 && kTileBytes % kTileBytesM == 0, "a stage holds whole tiles of maxima");
       const int et = threadIdx.x - 64;
       const int n_chunks = (n_tiles + kTilesPerChunk - 1) / kTilesPerChunk;
+      int c_fetched = 0;          // (thread et == 0) chunks requested so far
       auto fetch = [&](int c) {   // thread et == 0 only
+        c_fetched = c + 1;
         const int tiles_here = min(kTilesPerChunk, n_tiles - c * kTilesPerChunk);
         const uint32_t bar = smem_u32(&ctl->m_full[c % kStages]);
         mbar_expect_tx(bar, tiles_here * kTileBytesM);
@@ -361,17 +373,18 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         for (int q = 0; q < 4; ++q) ms[v4 * 4 + q] = ctl->mstar[og * R + src + q];
       }
       float* srow = p.scores + ((size_t)(b * p.hq + oh) * p.nqb + min(oi, p.nqb - 1)) * p.nqb;
+      int c_done = 0;
       for (int c = 0; c < n_chunks && alive; ++c) {
         const int st = c % kStages;
         if (et == 0 && c + kStages - 1 < n_chunks) {
           // the stage of chunk c - 1 takes chunk c + kStages - 1 once every thread has read it
-          if (c > 0 && !mbar_wait(smem_u32(&ctl->m_empty[(c - 1) % kStages]), ((c - 1) / kStages) & 1, abort_flag)) {
+          if (c > 0 && !mbar_wait(smem_u32(&ctl->m_empty[(c - 1) % kStages]), ((c - 1) / kStages) & 1, abort_flag, budget)) {
             if (!*abort_flag) screen_timeout(ctl, status);
           } else {
             fetch(c + kStages - 1);
           }
         }
-        alive = mbar_wait(smem_u32(&ctl->m_full[st]), (c / kStages) & 1, abort_flag);
+        alive = mbar_wait_warp(smem_u32(&ctl->m_full[st]), (c / kStages) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         const int tiles_here = min(kTilesPerChunk, n_tiles - c * kTilesPerChunk);
         const float* stage = reinterpret_cast<const float*>(smem + (size_t)kTileBytes * (kRowTiles + st));
@@ -396,11 +409,24 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           }
         }
         mbar_arrive(smem_u32(&ctl->m_empty[st]));
+        c_done = c + 1;
       }
+      if (et == 0) { ctl->c_fetched = c_fetched; ctl->c_done = c_done; }
     }
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    // the kernel gave up somewhere: copies and products still in flight finish on their own and must have done so
+    // before the CTA's shared and tensor memory go to the next one
+    (void)mbar_wait_noabort(smem_u32(&ctl->a_full), 0);
+    const int ti = ctl->t_issued, td = ctl->t_done;
+    for (int tt = max(0, ti - kStages); tt < ti; ++tt) (void)mbar_wait_noabort(smem_u32(&ctl->k_full[tt % kStages]), (tt / kStages) & 1);
+    if (td > 0) (void)mbar_wait_noabort(smem_u32(&ctl->k_empty[(td - 1) % kStages]), ((td - 1) / kStages) & 1);
+    const int cf = ctl->c_fetched;
+    for (int cc = max(ctl->c_done, cf - kStages); cc < cf; ++cc) (void)mbar_wait_noabort(smem_u32(&ctl->m_full[cc % kStages]), (cc / kStages) & 1);
+  }
+  __syncwarp();
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
   {
     // the parked maxima are dead: let L2 drop the lines instead of writing them back

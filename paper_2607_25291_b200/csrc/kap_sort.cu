@@ -382,7 +382,7 @@ __device__ void select_largest(const unsigned long long* a, int n, int want, uns
 }
 
 __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap,
-                                                            int tie_bytes) {
+                                                            int tie_bytes, const int32_t* status) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
   unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);        // [tie_bytes]
@@ -412,6 +412,8 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
     }
     return;
   }
+  // a screen kernel that gave up has left the scratch half written: nothing of it may be used for addressing
+  const int poisoned = *reinterpret_cast<const volatile int32_t*>(status);   // (tested together with `hard` below)
   unsigned hard = 0u;                         // (tested only after the scores have been requested: one round trip, not two)
   unsigned long long amb = 0ULL;              // bit r: sampled row r of the block was too close to call
   for (int t = 0; t < T; ++t) {
@@ -461,6 +463,7 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
       keys[j] = key;
     }
   }
+  if (poisoned != 0) return;
   if (hard) {  // left to the double-precision kernel
     if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
     return;
@@ -720,7 +723,9 @@ cudaError_t launch_kap_sort(const KapParams& p, const KapScreenParams& sp, float
   cudaError_t e = cudaFuncSetAttribute(kap_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid(p.nqb / p.qtiles, p.hq, p.batch);
-  kap_sort_kernel<<<grid, kThreads, smem, st>>>(p, sp, tau_score, cap, tie_bytes);
+  const int32_t* status = device_status_word();
+  if (!status) return cudaErrorInvalidSymbol;
+  kap_sort_kernel<<<grid, kThreads, smem, st>>>(p, sp, tau_score, cap, tie_bytes, status);
   return cudaGetLastError();
 }
 

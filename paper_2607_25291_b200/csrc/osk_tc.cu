@@ -69,6 +69,7 @@ struct __align__(8) Control {
   volatile int end_kk;            // last scored position, -1 until known
   volatile int k_loaded;          // K tiles the loader requested; -1 until it has stopped requesting
   volatile int final_computed;
+  volatile int v_req, v_taken;    // V tiles requested by the controller / whose arrival the PV issuer has waited for
   volatile int abort_flag;
   int poisoned;
   volatile uint32_t dec[kDecRing];
@@ -175,6 +176,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->end_kk = -1;
     ctl->k_loaded = -1;
     ctl->final_computed = 0;
+    ctl->v_req = 0; ctl->v_taken = 0;
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -312,8 +314,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         last_issued = kk;
       }
       // a product issued ahead of the walk's end may still be running: it must finish before TMEM is released
-      if (alive && last_issued >= 0 &&
-          !mbar_wait(smem_u32(&ctl->k_empty[last_issued % kKStages]), (last_issued / kKStages) & 1, abort_flag, budget) && !*abort_flag)
+      if (last_issued >= 0 &&
+          !mbar_wait_noabort(smem_u32(&ctl->k_empty[last_issued % kKStages]), (last_issued / kKStages) & 1) && !*abort_flag)
         report_timeout(ctl, status);
     }
   } else if (warp == 3) {
@@ -322,6 +324,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
       const uint64_t vdesc0 = smem_desc_sw128(v_sm, kHalfBytes, 1024);
       bool alive = true;
+      int n_issued = 0;
       for (int n = 0; alive; ++n) {
         // the next computed block's P, or the end of the walk
         const uint32_t bar = smem_u32(&ctl->p_full[n & 1]), par = (n >> 1) & 1;
@@ -337,11 +340,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const int vs = n % kVStages;
         alive = mbar_wait(smem_u32(&ctl->v_full[vs]), (n / kVStages) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        ctl->v_taken = n + 1;
         tc_fence_after();
         // 16 keys per MMA: 8 TMEM columns of P, 2 KiB (two 8-key groups) of the V tile
         mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p[n & 1], vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
         mma_commit(smem_u32(&ctl->p_empty[n & 1]));
+        n_issued = n + 1;
       }
+      // a product still running when the walk was given up must finish before tensor memory is released
+      if (!alive && n_issued > 0) (void)mbar_wait_noabort(smem_u32(&ctl->p_empty[(n_issued - 1) & 1]), ((n_issued - 1) >> 1) & 1);
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ controller
@@ -352,7 +359,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int par = kk & 1;
       const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
-      alive = mbar_wait(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
       // The statistic is <= 0, so among bit patterns the smallest unsigned word is the largest value.
@@ -379,6 +386,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
             mbar_expect_tx(bar, kTileBytes);
             load_kv_block(p, &v_map, dst, b, g, j, bar);
+            ctl->v_req = n_before + 1;
           }
           dec_word |= 1u << (kk & 31);
         }
@@ -437,6 +445,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
             if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
+        // one answer per warp: the loads below are executed by all of its lanes or by none
+        ended = __any_sync(0xffffffffu, ended) != 0;
+        alive = __all_sync(0xffffffffu, alive) != 0;
         if (ended || !alive) break;
       }
       tc_fence_after();
@@ -461,15 +472,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
       // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
       //      walk gets here at all (n_needed only grows: an old value merely costs this wait)
-      if (kk >= ctl->n_needed) {
-        alive = mbar_wait(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
+      if (kk >= __shfl_sync(0xffffffffu, ctl->n_needed, 0)) {   // (one reading per warp: the counter grows while it is read)
+        alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         if (ctl->dec[(kk - 1) % kDecRing] & kDecEnd) break;
       }
       // ---- running maximum before this position comes from the other group
       float m_in = -INFINITY;
       if (kk > 0) {
-        alive = mbar_wait(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         m_in = ctl->mrow[grp ^ 1][r];
       }
@@ -480,7 +491,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       ctl->mrow[grp][r] = m_new;
       mbar_arrive(smem_u32(&ctl->m_ready[grp]));
       // ---- the controller's decision
-      alive = mbar_wait(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget);
       if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
       const uint32_t d = ctl->dec[kk % kDecRing];
       const bool last = (d & kDecEnd) != 0;
@@ -515,11 +526,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       // ---- P has two buffers: the product before last must have finished with this one; O is rescaled only if a row
       //      maximum moved, and only then must the previous product have finished as well
       if (n_before > 1) {
-        alive = mbar_wait(smem_u32(&ctl->p_empty[n_before & 1]), ((n_before - 2) >> 1) & 1, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->p_empty[n_before & 1]), ((n_before - 2) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
       }
       if (n_before > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O
-        alive = mbar_wait(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
         uint32_t o[32];
@@ -549,16 +560,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       mbar_arrive(smem_u32(&ctl->fin_bar));
     } else {
       if (alive) {
-        alive = mbar_wait(smem_u32(&ctl->fin_bar), 0, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->fin_bar), 0, abort_flag, budget);
         if (!alive && !*abort_flag) report_timeout(ctl, status);
       }
-      if (alive && !*abort_flag) {
+      if (__all_sync(0xffffffffu, alive && !*abort_flag)) {
         const float mb = ctl->fin_m[r];
         const float mf = fmaxf(m_ref, mb);         // the running maximum is monotone: this is its final value
         const float lt = l * ex2_approx(m_ref - mf) + ctl->fin_l[r] * ex2_approx(mb - mf);
         const int n_comp = ctl->final_computed;
         if (n_comp > 0) {
-          alive = mbar_wait(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag, budget);
+          alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag, budget);
           if (!alive && !*abort_flag) report_timeout(ctl, status);
         }
         if (alive) {
@@ -604,6 +615,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) {
+    // copies that nobody has waited for when the walk was given up: the Q tile, a V tile the PV issuer never took
+    (void)mbar_wait_noabort(smem_u32(&ctl->q_stage), 0);
+    for (int n = ctl->v_taken; n < ctl->v_req; ++n) (void)mbar_wait_noabort(smem_u32(&ctl->v_full[n % kVStages]), (n / kVStages) & 1);
+  }
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
 

@@ -74,6 +74,12 @@ __device__ __forceinline__ bool mbar_wait_noabort(uint32_t bar, uint32_t parity,
     if (clock64() - t0 > budget) return false;
   }
 }
+// For code all 32 lanes of a warp run together: the same bounded wait, with one answer for the whole warp (lanes that
+// poll on their own can see the budget run out at different moments, and what follows -- tcgen05.ld/st, __syncwarp --
+// must be executed by all lanes or by none)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, budget)) != 0;
+}
 // named barrier among `nthreads` threads of the CTA (ids 1..15; 0 is __syncthreads)
 __device__ __forceinline__ void bar_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
