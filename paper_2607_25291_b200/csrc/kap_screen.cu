@@ -309,8 +309,10 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         }
       }
       // the row's best block, and whether the runner-up is too close to call
-      const bool amb = row_ok && (top1 - top2) * p.scale <= p.tau_row;
-      const bool amb3 = row_ok && (top1 - top3) * p.scale <= p.tau_row;
+      // (the threshold grows with the magnitude of the call's inputs, which is what the rounding error of a logit follows)
+      const float tau_row = fmaxf(p.tau_row, 2.f * screen_error_bound(p.mag[0], p.mag[1], p.scale));
+      const bool amb = row_ok && (top1 - top2) * p.scale <= tau_row;
+      const bool amb3 = row_ok && (top1 - top3) * p.scale <= tau_row;
       const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);
       const int shift = (lane / R) * R;
       const unsigned grp_mask = (R == 32) ? 0xffffffffu : (((1u << R) - 1u) << shift);

@@ -383,6 +383,8 @@ __device__ void select_largest(const unsigned long long* a, int n, int want, uns
 
 __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap,
                                                             int tie_bytes, const int32_t* status) {
+  // near ties: never closer than twice what the screen may be off by on inputs of this call's magnitude
+  tau_score = fmaxf(tau_score, 2.f * screen_error_bound(sp.mag[0], sp.mag[1], sp.scale));
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
   unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);        // [tie_bytes]

@@ -1,0 +1,121 @@
+"""Every Stage-1 list of the full-size workloads against the fp64 oracle, and the error of the float32 screen where the
+bit-exactness argument uses it.
+
+The CUDA path writes all lists of a workload in one call; the oracle re-derives every one of them (Algorithm A steps
+2-5), one query head per task in a pool of host processes.  On chosen heads the float32 scores the fast path sorted
+(exported through cosa_options.kap_scores) are compared with the oracle's double-precision scores: the sort stage
+treats two neighbours as ordered only when they differ by more than tau_score relative, which is sound as long as the
+screen's error stays well below tau_score / 2 -- asserted here at < tau_score / 4, on the measured workloads rather
+than assumed.  The oracle's own margins are audited too: no decision on these inputs hangs on less than 1e-9
+relative (two double-precision evaluations with different summation orders could otherwise disagree).
+"""
+import multiprocessing as mp
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_25291_b200 as cosa
+from oracle import cosa_oracle as O
+from synth.configs import WORKLOADS
+from synth.generator import bf16_bits_to_f64
+from tests.helpers import to_dev
+
+pytestmark = pytest.mark.gpu
+
+TAU_SCORE = 2.0 ** -15          # the sort stage's near-tie threshold (relative), as set in the library
+_G = {}                         # inputs of the running comparison, inherited by the forked workers
+
+
+def _one_head(h):
+    """Oracle lists of query head h (all query blocks); optionally the screen's score error on that head."""
+    try:
+        from threadpoolctl import threadpool_limits
+        limiter = threadpool_limits(1)
+    except Exception:
+        limiter = None
+    g = _G
+    G = g["qb"].shape[0] // g["kb"].shape[0]
+    qf = bf16_bits_to_f64(g["qb"][h])[None]
+    kf = bf16_bits_to_f64(g["kb"][h // G])[None]
+    order, count, audit = O.kap_select(qf, kf, s=g["stride"], budget=g["budget"], order_stride=g["pitch"], audit=True)
+    ok = np.array_equal(order[0], g["order"][h]) and np.array_equal(count[0], g["count"][h])
+    bad = []
+    if not ok:
+        bad = [int(i) for i in range(order.shape[1])
+               if count[0, i] != g["count"][h, i] or not np.array_equal(order[0, i], g["order"][h, i])][:8]
+    err = None
+    if g["scores"] is not None and h in g["score_heads"]:
+        err, flag_diff = 0.0, 0
+        for i in range(order.shape[1]):
+            s64, f64, _ = O.kap_scores(qf, kf, 0, i, g["stride"])
+            s32 = g["scores"][h, i, :i + 1].astype(np.float64)
+            err = max(err, float(np.max(np.abs(s32 - s64) / s64)))
+            flag_diff += int(np.sum(g["flags"][h, i, :i + 1].astype(bool) != f64))
+        err = (err, flag_diff)
+    del limiter
+    return h, ok, bad, audit["min_rel_score_gap"], audit["min_row_top2_gap"], err
+
+
+def compare_every_list(w, qb, kb, budget, score_heads=()):
+    q, k = to_dev(qb), to_dev(kb)
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(budget, nqb) + 7) // 8 * 8
+    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+    kw = {}
+    if len(score_heads):
+        kw["kap_scores"] = torch.zeros(1, w.hq, nqb, nqb, dtype=torch.float32, device="cuda")
+        kw["kap_flags"] = torch.zeros(1, w.hq, nqb, nqb, dtype=torch.uint8, device="cuda")
+    cosa.cosa_kap_select(q, k, budget, order, count, opt=cosa.default_options(stride=w.stride, order_stride=pitch, **kw))
+    assert cosa.cosa_device_status() == 0
+    _G.clear()
+    _G.update(qb=qb, kb=kb, stride=w.stride, budget=budget, pitch=pitch, order=order[0].cpu().numpy(),
+              count=count[0].cpu().numpy(), score_heads=set(score_heads),
+              scores=kw["kap_scores"][0].cpu().numpy() if kw else None,
+              flags=kw["kap_flags"][0].cpu().numpy() if kw else None)
+    del q, k, order, count, kw
+    procs = max(1, min(w.hq, (os.cpu_count() or 2)))
+    # the workers only run numpy on arrays they inherit; the heads with the (slower) score comparison go first
+    heads = sorted(range(w.hq), key=lambda h: h not in _G["score_heads"])
+    with mp.get_context("fork").Pool(procs) as pool:
+        results = pool.map(_one_head, heads, chunksize=1)
+    _G.clear()
+    worst_err, min_gap, min_top2 = 0.0, np.inf, np.inf
+    for h, ok, bad, gap, top2, err in results:
+        assert ok, f"head {h}: lists of query blocks {bad} differ from the oracle"
+        min_gap, min_top2 = min(min_gap, gap), min(min_top2, top2)
+        if err is not None:
+            assert err[1] == 0, f"head {h}: {err[1]} exported HRM flags differ from the oracle"
+            worst_err = max(worst_err, err[0])
+    # no decision of the oracle itself hangs on a margin that double-precision rounding could move
+    assert min_gap > 1e-9 and min_top2 > 1e-9, (min_gap, min_top2)
+    if len(score_heads):
+        assert worst_err < TAU_SCORE / 4, worst_err
+    return dict(lists=w.hq * nqb, screen_rel_err=worst_err, min_rel_score_gap=min_gap, min_row_top2_gap=min_top2)
+
+
+def test_qwen3_128k_every_list_and_screen_error():
+    w = WORKLOADS["qwen3_128k"]
+    qb, kb, _, _ = w.make()
+    print("128k", compare_every_list(w, qb, kb, w.kap_budget, score_heads=(0, 9, 18, 27)))
+
+
+def test_qwen3_32k_screen_error_on_every_head():
+    w = WORKLOADS["qwen3_32k"]
+    qb, kb, _, _ = w.make()
+    print("32k", compare_every_list(w, qb, kb, w.kap_budget, score_heads=range(w.hq)))
+
+
+def test_llama31_64k_every_list_at_25_percent():
+    w = WORKLOADS["llama31_64k_sweep"]
+    qb, kb, _, _ = w.make()
+    print("64k", compare_every_list(w, qb, kb, 0.25, score_heads=(5, 22)))
+
+
+def test_qwen3_128k_stack_two_whole_layers():
+    w = WORKLOADS["qwen3_128k_x36"]
+    for layer in (0, 4):                                       # 8 and 128 needle blocks per head
+        qb, kb, _, _ = w.make(layer=layer)
+        print("128k stack layer", layer, compare_every_list(w, qb, kb, w.kap_budget))

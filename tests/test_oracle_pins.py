@@ -280,6 +280,37 @@ def test_score_and_flag_invariants(small):
                 assert fl[np.argmax(M, axis=1)].all()
 
 
+def test_block_scores_from_explicit_index_sets():
+    """Eqs. (9)-(12) written out token by token: sampled query rows Q_i = {r : r div R = i}, sampled keys of a key
+    block K_j = {c : c div R = j}, sampled row r is token r*s (likewise for keys), causal mask c <= r.  Scalar
+    loops over plain Python floats that share nothing with the oracle's vectorised gather, reshape and max: a
+    wrong axis or a wrong grouping of the sampled keys into blocks in `kap_scores` fails here."""
+    q, k, _, _ = _inputs(seed=11, hq=2, hkv=1, n=512, needles=1)
+    n, d = q.shape[1], q.shape[2]
+    for s in (8, 32):
+        R = 128 // s
+        for h, i in ((0, 0), (0, 2), (1, 3)):
+            rows = [r for r in range(n // s) if r // R == i]                      # Q_i
+            J = i + 1
+            P = {}                                                                # (r, j) -> max_c softmax(z)[r, c]
+            for r in rows:
+                cs = [c for c in range(n // s) if c <= r]                         # causal: sampled key not after the row
+                z = {c: math.fsum(q[h, r * s, e] * k[0, c * s, e] for e in range(d)) / math.sqrt(d) for c in cs}
+                zmax = max(z.values())
+                den = math.fsum(math.exp(z[c] - zmax) for c in cs)                # Eq. 8: softmax over the sampled keys
+                for j in range(J):
+                    Kj = [c for c in cs if c // R == j]                           # K_j
+                    P[r, j] = max(math.exp(z[c] - zmax) / den for c in Kj) if Kj else 0.0     # Eq. 9: MaxPool
+            want_s, want_h = [], []
+            for j in range(J):
+                pbar = [P[r, j] / max(P[r, jj] for jj in range(J)) for r in rows]            # Eq. 10: MaxNorm
+                want_s.append(math.fsum(pbar))                                               # Eq. 11
+                want_h.append(any(x == 1.0 for x in pbar))                                   # Eq. 12
+            got_s, got_h, _ = O.kap_scores(q, k, h, i, s)
+            assert np.allclose(got_s, want_s, rtol=1e-12, atol=0)
+            assert list(got_h) == want_h
+
+
 def test_single_sample_per_block_reduces_to_argsort(small):
     """s = b: one sampled row and key per block, so exactly one HRM block and the list is
     that block followed by the others in descending order of the sampled logit."""
