@@ -14,7 +14,7 @@ import torch
 import paper_2607_25291_b200 as cosa
 from oracle import cosa_oracle as O
 from synth.configs import WORKLOADS, tiny
-from synth.generator import scatter_to_pages
+from synth.generator import bf16_bits_to_f64, scatter_to_pages
 from tests.helpers import alloc_lists, alloc_outputs, to_dev, widen
 
 pytestmark = pytest.mark.gpu
@@ -294,6 +294,35 @@ def test_kap_16k_tie_chain_longer_than_the_margin(mid):
         for i in blocks:
             assert np.array_equal(_np(count)[:, i], ref_count[:, i]), (budget, i)
             assert np.array_equal(_np(order)[:, i], ref_order[:, i]), (budget, i)
+
+
+def _scaled_bits(bits, factor, outliers=(), outlier_factor=1.0):
+    """bf16 bit patterns times a power of two, a few channels times another one: exact in bf16."""
+    x = bf16_bits_to_f64(bits) * factor
+    for c in outliers:
+        x[..., c] *= outlier_factor
+    u = x.astype(np.float32).view(np.uint32)
+    assert ((u & 0xffff) == 0).all()                      # still exactly representable
+    return (u >> 16).astype(np.uint16)
+
+
+@pytest.mark.parametrize("factor,outlier_factor", [(4.0, 1.0), (4.0, 8.0), (16.0, 4.0)])
+def test_kap_inputs_of_large_magnitude(factor, outlier_factor):
+    """Activations far larger than the benchmark's, with a few outlier channels (Sec. 4.2 is silent on magnitudes): the
+    rounding error of the float32 screen grows with |q| |k|, and the thresholds below which its verdicts are
+    re-examined in double precision grow with it, so the lists stay those of exact arithmetic."""
+    w = tiny(seed=77, hq=4, hkv=2, n=2048, needles=3)
+    qb, kb, _, _ = w.make()
+    qs = _scaled_bits(qb, factor, outliers=(3, 64, 101), outlier_factor=outlier_factor)
+    ks = _scaled_bits(kb, factor, outliers=(3, 64, 101), outlier_factor=outlier_factor)
+    q, k = to_dev(qs), to_dev(ks)
+    qf, kf = widen(qs, ks)
+    nqb = w.n // 128
+    ref_order, ref_count = O.kap_select(qf, kf, s=8, budget=0.4, order_stride=nqb)
+    for impl in (0, 1):
+        order, count = run_kap(q, k, 0.4, impl=impl)
+        assert np.array_equal(_np(count), ref_count), impl
+        assert np.array_equal(_np(order), ref_order), impl
 
 
 @pytest.mark.parametrize("stride", [4, 8, 16])
