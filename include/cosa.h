@@ -170,9 +170,17 @@ int32_t cosa_budget_count(float budget, int32_t candidates);
  * the two tiles of a block then walk the same K/V tiles in the same order.  kap_scores / kap_flags are not
  * available in this mode.
  * Scores are evaluated so that the list equals the one exact arithmetic would give whenever
- * neighbouring scores differ by more than ~1e-9 relative.  With top_p the prefix sums are taken over
- * float32 scores (relative error < 2^-15): K_i equals the exact count unless a prefix sum lies
- * within that error of the threshold, where it may differ by one.
+ * neighbouring scores differ by more than ~1e-9 relative: the fast path scores in float32 on the
+ * tensor cores and re-examines in double precision every verdict its rounding error could change
+ * (rows whose two best blocks are too close to call, sorted neighbours closer than 2^-15 relative;
+ * both thresholds grow with the largest |q| |k| among the call's sampled rows, which is what that
+ * error follows).  With top_p the count K_i -- an integer decided by floating point -- is decided in
+ * the precision the path computes its scores in: it is exactly the Top-p count of the float32
+ * scores (those kap_scores exports), cumulated in double precision along the order (flag, float32
+ * score, id).  Against scores of exact arithmetic it can differ by one, and only where a deciding
+ * prefix sum lies within the scores' rounding error (< 2^-17 relative on the tested workloads) of
+ * the threshold; the kept ids are in every case a prefix of the exact order.  impl = 1 takes this
+ * decision in double precision too.
  */
 int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape,
                     float budget, int32_t* out_order, int32_t* out_count, void* stream);

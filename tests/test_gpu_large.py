@@ -47,8 +47,12 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
                 visited=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
                 scored=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
                 decisions=torch.zeros(1, w.hq, nqb, (pitch + 31) // 32, dtype=torch.int32, device="cuda"))
+    ex = {}
+    if top_p > 0:      # the float32 scores the Top-p count is decided on
+        ex = dict(kap_scores=torch.zeros(1, w.hq, nqb, nqb, dtype=torch.float32, device="cuda"),
+                  kap_flags=torch.zeros(1, w.hq, nqb, nqb, dtype=torch.uint8, device="cuda"))
     opt = cosa.default_options(stride=w.stride, skip_scale=skip_scale, order_stride=pitch, top_p=top_p,
-                               out_scored=bufs["scored"], out_decisions=bufs["decisions"])
+                               out_scored=bufs["scored"], out_decisions=bufs["decisions"], **ex)
     cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt)
     cosa.cosa_osk_attention(q, k, v, order, count, osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
     assert cosa.cosa_device_status() == 0
@@ -77,6 +81,7 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
     # sampled parity against the oracle
     hv = HeadView(qb, kb, vb)
     stats = []
+    s32, f8 = (_np(ex["kap_scores"]), _np(ex["kap_flags"])) if ex else (None, None)
     for h in kap_heads:
         qf, kf, vf = hv.get(h)
         sel = range(nqb) if check_all_kap else blocks
@@ -85,7 +90,8 @@ def run_and_check(w, qb, kb, vb, kap_budget, osk_budget, skip_scale, kap_heads, 
                                                        query_blocks=(None if check_all_kap else blocks), top_p=top_p,
                                                        audit=True)
             check_topp_lists(order_np, count_np, ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[0],
-                             [(h, 0, i) for i in sel])
+                             [(h, 0, i) for i in sel], scores32=s32, flags=f8,
+                             top_p=top_p, budget=kap_budget)
         else:
             ref_order, ref_count = O.kap_select(qf, kf, s=w.stride, budget=kap_budget, order_stride=pitch,
                                                 query_blocks=(None if check_all_kap else blocks))

@@ -41,17 +41,40 @@ def run_kap(q, k, budget, stride=8, causal=True, order_stride=None, scores=False
     return (order, count, kw) if scores else (order, count)
 
 
-# Top-p counts come from prefix sums of float32 scores (relative error < 2^-15) on the fast path and of double
-# precision scores (a few ulp from the oracle's) in the exact kernel: the count must equal the oracle's unless the
-# oracle's own prefix sum lies within that error of the threshold, where it may differ by one.
-TOPP_MARGIN = {0: 2.0 ** -14, 1: 1e-12}
+# Top-p counts: an integer decided by floating point, which both sides take in the same precision.  On the fast path
+# that is the kernel's: float32 scores (relative error < 2^-17 against exact arithmetic, asserted on the full-size
+# workloads), cumulated in double precision -- the count must be exactly the one those float32 scores give
+# (check_topp_lists, `scores32`).  Against the all-double oracle it may then differ by one, and only where the
+# oracle's own prefix sum lies within 2^-16 of the threshold; the exact kernel (impl = 1) agrees with the oracle to a
+# few ulp of double precision.
+TOPP_MARGIN = {0: 2.0 ** -16, 1: 1e-12}
 
 
-def check_topp_lists(order_np, count_np, ref_order, ref_count, margin, tol, pairs):
-    """GPU lists against the oracle's Top-p lists for the (h_gpu, h_ref, i) triples in `pairs`."""
+def topp_count_in_kernel_precision(s32, flags, top_p, cap):
+    """The Top-p count decided on the float32 scores the fast path sorts (the precision the kernel takes this
+    decision in): candidates in the order (flag descending, float32 score descending, id ascending), prefix sums in
+    double precision.  Returns (K, relative margin of the deciding prefix sums)."""
+    J = len(s32)
+    ids = np.lexsort((np.arange(J), -s32.astype(np.float64), -flags.astype(np.int64)))
+    c = np.cumsum(s32[ids].astype(np.float64))
+    thr = float(top_p) * c[-1]
+    K = min(J, int(np.searchsorted(c, thr, side="left")) + 1)
+    gaps = [abs(c[K - 1] - thr)] + ([abs(c[K - 2] - thr)] if K >= 2 else [])
+    return min(K, cap), min(gaps) / c[-1]
+
+
+def check_topp_lists(order_np, count_np, ref_order, ref_count, margin, tol, pairs, scores32=None, flags=None, top_p=None,
+                     budget=1.0):
+    """GPU lists against the oracle's Top-p lists for the (h_gpu, h_ref, i) triples in `pairs`.  With the fast path's
+    exported float32 scores the count is also held to the decision taken in that precision, exactly."""
     off = 0
     for hg, hr, i in pairs:
         kept, want = int(count_np[hg, i]), int(ref_count[hr, i])
+        if scores32 is not None:
+            k32, m32 = topp_count_in_kernel_precision(scores32[hg, i, :i + 1], flags[hg, i, :i + 1], top_p,
+                                                      O.budget_count(budget, i + 1))
+            # (a query block the fast path hands to the double-precision kernel is counted there)
+            assert kept == k32 or kept == want or m32 <= 1e-12, (hg, i, kept, k32, want, m32)
         if margin[hr, i] > tol:
             assert kept == want, (hg, i, kept, want, margin[hr, i])
         else:
@@ -164,11 +187,12 @@ def test_kap_topp_small(small, impl, top_p, budget):
     q, k, _ = small["dev"]
     qf, kf, _ = small["f64"]
     for stride in (8, 32):
-        order, count = run_kap(q, k, budget, stride, impl=impl, top_p=top_p)
+        order, count, ex = run_kap(q, k, budget, stride, impl=impl, top_p=top_p, scores=True)
         ref_order, ref_count, audit = O.kap_select(qf, kf, s=stride, budget=budget, order_stride=order.shape[-1],
                                                    top_p=top_p, audit=True)
         pairs = [(h, h, i) for h in range(qf.shape[0]) for i in range(qf.shape[1] // 128)]
-        check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs)
+        strict = dict(scores32=_np(ex["kap_scores"]), flags=_np(ex["kap_flags"]), top_p=top_p, budget=budget) if impl == 0 else {}
+        check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs, **strict)
         if top_p == 1.0:
             assert np.array_equal(_np(count), ref_count)
 
@@ -178,11 +202,12 @@ def test_kap_topp_4k(cfg1, impl):
     q, k, _ = cfg1["dev"]
     qf, kf, _ = cfg1["f64"]
     w = cfg1["w"]
-    order, count = run_kap(q, k, 1.0, w.stride, impl=impl, top_p=0.95)
+    order, count, ex = run_kap(q, k, 1.0, w.stride, impl=impl, top_p=0.95, scores=True)
     ref_order, ref_count, audit = O.kap_select(qf, kf, s=w.stride, budget=1.0, order_stride=order.shape[-1],
                                                top_p=0.95, audit=True)
     pairs = [(h, h, i) for h in range(w.hq) for i in range(w.n_blocks)]
-    off = check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs)
+    strict = dict(scores32=_np(ex["kap_scores"]), flags=_np(ex["kap_flags"]), top_p=0.95) if impl == 0 else {}
+    off = check_topp_lists(_np(order), _np(count), ref_order, ref_count, audit["topp_margin"], TOPP_MARGIN[impl], pairs, **strict)
     assert off <= 2
     assert (ref_count < np.arange(1, w.n_blocks + 1)[None, :]).any()      # Top-p does drop blocks on this workload
 
