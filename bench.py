@@ -7,7 +7,9 @@ at 128K tokens (32 query / 8 KV heads, d = 128, causal, block 128, KAP budget 10
 OSK budget 4 %).  `value` is the visited-block TFLOP/s of the whole job: 2*128*128*128
 FLOPs per block whose logits OSK formed plus the same per block it computed, summed over
 all ranks, divided by the (max over ranks) time of KAP + OSK.  With N > 1 every rank
-processes its own layer (independent seeds): weak scaling, no data-path collective.
+processes its own layer (independent seeds): weak scaling, no data-path collective.  With --shard kv_head
+the ranks split one layer by KV-head group instead (strong scaling; still no data-path collective: the
+work items of different KV heads share nothing, and the outputs stay head-sharded).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 """
@@ -46,6 +48,9 @@ def parse():
                     help="K and V as page pools of this many tokens per page behind a shuffled page table (Sec. C.1); not the headline config")
     ap.add_argument("--block-q", type=int, default=128, choices=[128, 256],
                     help="256: one Stage-1 ranking per 256-row query block shared by its two row tiles; not the headline config")
+    ap.add_argument("--shard", default="layer", choices=["layer", "kv_head"],
+                    help="with --gpus N: 'layer' gives every rank a layer of its own (weak scaling, the default); 'kv_head' splits "
+                         "ONE layer by KV-head group, rank r running KAP + OSK on its heads only (strong scaling; N <= KV heads)")
     ap.add_argument("--top-p", type=float, default=0.0,
                     help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
     return ap.parse_args()
@@ -210,19 +215,29 @@ def main():
     # ---- synthetic inputs (rank r = its own layer of the same shape: independent problems)
     t_gen = time.perf_counter()
     import dataclasses
-    qb, kb, vb, _ = w.make(layer=rank) if w.layers > 1 else dataclasses.replace(w, seed=w.seed + rank).make()
+    hq_l, hkv_l = w.hq, w.hkv                               # heads this rank works on
+    if args.shard == "kv_head":
+        from paper_2607_25291_b200.shard import kv_head_shard
+        if world > w.hkv:
+            raise SystemExit(f"--shard kv_head: {world} ranks but only {w.hkv} KV heads")
+        qb, kb, vb, _ = w.make(layer=0) if w.layers > 1 else w.make()       # the same layer on every rank ...
+        kv_lo, kv_hi, q_lo, q_hi = kv_head_shard(w.hq, w.hkv, world, rank)
+        qb, kb, vb = qb[q_lo:q_hi], kb[kv_lo:kv_hi], vb[kv_lo:kv_hi]          # ... of which it keeps its heads
+        hq_l, hkv_l = q_hi - q_lo, kv_hi - kv_lo
+    else:
+        qb, kb, vb, _ = w.make(layer=rank) if w.layers > 1 else dataclasses.replace(w, seed=w.seed + rank).make()
     t_gen = time.perf_counter() - t_gen
     pin = lambda bits: torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)[None].contiguous().pin_memory()
     qh, kh, vh = pin(qb), pin(kb), pin(vb)
     q, k, v = (t.to(dev, non_blocking=True) for t in (qh, kh, vh))
     kap_budget = 1.0 if args.top_p > 0 else w.kap_budget
     pitch = order_pitch(cosa, kap_budget, nqb)
-    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device=dev)
-    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
+    order = torch.empty(1, hq_l, nqb, pitch, dtype=torch.int32, device=dev)
+    count = torch.empty(1, hq_l, nqb, dtype=torch.int32, device=dev)
     out = torch.empty_like(q)
-    lse = torch.empty(1, w.hq, w.n, dtype=torch.float32, device=dev)
-    visited = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
-    scored = torch.empty(1, w.hq, nqb, dtype=torch.int32, device=dev)
+    lse = torch.empty(1, hq_l, w.n, dtype=torch.float32, device=dev)
+    visited = torch.empty(1, hq_l, nqb, dtype=torch.int32, device=dev)
+    scored = torch.empty(1, hq_l, nqb, dtype=torch.int32, device=dev)
     opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=scored,
                                top_p=args.top_p)
     stream = torch.cuda.current_stream()
@@ -321,11 +336,11 @@ def main():
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
     pipe_peak = sms * 8192 * clocks["sm_mhz"] * 1e6 / 1e12 if clocks.get("sm_mhz") else None
     osk_tflops = flops_step / (osk_ms * 1e-3) / 1e12
-    pairs = w.hq * (nqb * (nqb + 1) // 2)
+    pairs = hq_l * (nqb * (nqb + 1) // 2)
     R = 128 // w.stride
     kap_flops = 2.0 * R * R * 128 * pairs
     kap_tflops = kap_flops / (kap_ms * 1e-3) / 1e12
-    kap_bytes = (w.hq + w.hkv) * (w.n // w.stride) * 128 * 2 + order.numel() * 4 + count.numel() * 4
+    kap_bytes = (hq_l + hkv_l) * (w.n // w.stride) * 128 * 2 + order.numel() * 4 + count.numel() * 4
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
     if os.path.exists(tpath):
@@ -384,11 +399,14 @@ def main():
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong" if args.shard == "kv_head" else "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
                            "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "kap_block_q": args.block_q, "osk_budget": w.osk_budget, "stride": w.stride,
-                           "skip_scale": w.skip_scale, "parallelism": f"layer-per-rank x{world}",
+                           "skip_scale": w.skip_scale,
+                           "parallelism": (f"one layer, KV heads split over {world} ranks" if args.shard == "kv_head"
+                                           else f"layer-per-rank x{world}"),
                            "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
                            "blocks_scored": n_scored, "blocks_computed": n_computed,
                            "causal_block_pairs": pairs, "input_generation_s": round(t_gen, 1)},

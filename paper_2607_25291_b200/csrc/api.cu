@@ -101,7 +101,7 @@ cosa_options resolve_options(const cosa_options* opt) {
 }  // namespace
 
 // scratch the kernels of one call need (beyond inputs and outputs)
-struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, mag, slot_taken, maxima, kstage, total; int slots; bool gather; };
+struct KapScratch { size_t scores, jstar, ambmask, hard, redo_list, k2max, q2max, slot_taken, maxima, kstage, total; int slots; bool gather; };
 static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o) {
   KapScratch L{};
   const int stride = o.stride > 0 ? o.stride : 8;
@@ -121,7 +121,8 @@ static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o)
   L.ambmask = off; off += align_up(heads * nqb * 4, 256);
   L.hard = off; off += align_up(heads * nqb, 256);
   L.redo_list = off; off += align_up((1 + heads * nqb) * 4, 256);
-  L.mag = off; off += 256;
+  L.k2max = off; off += 256;
+  L.q2max = off; off += align_up(heads * nqb * 4, 256);
   // the screen's parked block maxima: one area per CTA that can be resident on the current device
   L.slots = kap_screen_slots();
   if (L.slots <= 0) L.slots = 160;   // no usable device (a size query only): the count of the largest sm_100a part, rounded up
@@ -230,7 +231,8 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   sp.hard = reinterpret_cast<uint8_t*>(ws + L.hard);
   sp.redo_list = reinterpret_cast<int32_t*>(ws + L.redo_list);
   sp.slot_taken = reinterpret_cast<int32_t*>(ws + L.slot_taken);
-  sp.mag = reinterpret_cast<const float*>(ws + L.mag);
+  sp.k2max = reinterpret_cast<const float*>(ws + L.k2max);
+  sp.q2max = reinterpret_cast<float*>(ws + L.q2max);
   sp.maxima = reinterpret_cast<float*>(ws + L.maxima);
   sp.slots = L.slots;
   sp.batch = p.batch; sp.hq = p.hq; sp.hkv = p.hkv; sp.n = p.n; sp.nqb = nqb;
@@ -248,7 +250,7 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
     p.pg.seq_lens = lens;
   }
   sp.pg = p.pg;
-  cudaError_t e = launch_kap_norms(sp.q, sp.k, sp.pg, p.batch, p.hq, p.hkv, p.n, s, reinterpret_cast<float*>(ws + L.mag), st);
+  cudaError_t e = launch_kap_norms(sp.k, sp.pg, p.batch, p.hkv, p.n, s, reinterpret_cast<float*>(ws + L.k2max), st);
   if (e != cudaSuccess) return cuda_fail(e, "kap norms launch");
   e = launch_kap_screen(sp, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");

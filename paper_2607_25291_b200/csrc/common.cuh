@@ -76,7 +76,8 @@ struct KapScreenParams {
   int32_t* redo_list;    // [1 + B*Hq*nQB]  [0] = number of entries, then flat (b*Hq+h)*nQB+i of query blocks to redo
   float* maxima;         // [slots][key tiles][128 rows x 128/R blocks]  per-row block maxima of the CTA that holds the slot
   int32_t* slot_taken;   // [slots]  0 = free; zeroed before every launch
-  const float* mag;      // [2]  largest squared norm of a sampled query row / key row of the call (kap_norms_kernel)
+  const float* k2max;    // [1]  largest squared norm of a sampled key row of the call (kap_norms_kernel)
+  float* q2max;          // [B,Hq,nQB]  largest squared norm of the sampled query rows of every (head, query block)
   int slots;             // CTAs that can be resident at once
   int batch, hq, hkv, n, nqb;
   int causal;
@@ -161,7 +162,7 @@ inline long long budget_to_fx(float budget) {
 
 // What the float32 screen may be off by: bound used for the error of a difference of two scaled logits of one sampled
 // row -- and so, relatively, of a block score, a sum of exponentials of such differences -- given the largest squared
-// norms of the call's sampled rows.  Products of two bf16 numbers are exact in float32; what is lost is lost in adding
+// norms of the sampled rows involved.  Products of two bf16 numbers are exact in float32; what is lost is lost in adding
 // 128 of them, in proportion to their size, which |q| |k| bounds.  The factor (8 x 2^-24) is calibrated: the largest
 // error seen on the measured workloads, all lists of all heads, is 3.4 times smaller (asserted by the tests at the
 // sizes the benchmark runs).
@@ -176,8 +177,8 @@ int32_t* device_status_word();
 cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st);
 bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
-cudaError_t launch_kap_norms(const __nv_bfloat16* q, const __nv_bfloat16* k, const KvPaging& pg, int batch, int hq, int hkv, int n,
-                             int stride, float* mag, cudaStream_t st);
+cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, int batch, int hkv, int n, int stride, float* k2max,
+                             cudaStream_t st);
 // CTAs of the screen kernel that can be resident at once on the current device (0 on failure), and the bytes of
 // block-maxima scratch each of them needs
 int kap_screen_slots();

@@ -1,5 +1,5 @@
-// KAP fast path, stage 0: the largest squared norms among the sampled query rows and among the sampled key rows of a
-// call (Algorithm A step 2 samples every s-th row of Q and K).
+// KAP fast path, stage 0: the largest squared norm among the sampled key rows of a call (Algorithm A step 2 samples
+// every s-th row of Q and K; the screen kernel takes the norms of the sampled query rows itself, from shared memory).
 //
 // The float32 screen forms its logits on the tensor cores; the rounding error of a logit grows with the size of the
 // products it adds up, which |q| |k| bounds (Cauchy-Schwarz).  The thresholds below which the later stages distrust the
@@ -12,35 +12,31 @@ namespace {
 
 constexpr int kThreads = 256;
 
-// one warp per row and turn, four rows in flight per warp; mag[0] = max |q_row|^2, mag[1] = max |k_row|^2 (bit patterns
-// of non-negative floats order like unsigned integers, so atomicMax on the bits is a float maximum)
-__global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
-                                                             KvPaging pg, int batch, int hq, int hkv, int n, int stride,
-                                                             float* mag) {
+// one warp per row and turn, four rows in flight per warp; *k2max = max |k_row|^2 over the sampled key rows (bit
+// patterns of non-negative floats order like unsigned integers, so atomicMax on the bits is a float maximum)
+__global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16* __restrict__ k, KvPaging pg, int batch, int hkv,
+                                                             int n, int stride, float* k2max) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const long long n_warps = ((long long)gridDim.x * kThreads) >> 5;
   const int ns = n / stride;
-  const long long rows_q = (long long)batch * hq * ns, rows = rows_q + (long long)batch * hkv * ns;
-  float best[2] = {0.f, 0.f};
+  const long long rows = (long long)batch * hkv * ns;
+  float best = 0.f;
   for (long long r0 = warp * 4; r0 < rows; r0 += n_warps * 4) {
     uint2 w[4];
-    int which[4];
+    bool live[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const long long r = r0 + u;
-      which[u] = -1;
+      live[u] = false;
       w[u] = make_uint2(0u, 0u);
       if (r >= rows) continue;
-      const bool is_q = r < rows_q;
-      const long long rr = is_q ? r : r - rows_q;
-      const int token = (int)(rr % ns) * stride;
-      const int bh = (int)(rr / ns);
-      const int b = bh / (is_q ? hq : hkv);
+      const int token = (int)(r % ns) * stride;
+      const int bg = (int)(r / ns);
+      const int b = bg / hkv;
       if (pg.seq_lens && token >= pg.seq_lens[b]) continue;      // padding past the item's length
-      const long long row = is_q ? (long long)bh * n + token : kv_row(pg, b, hkv, bh % hkv, n, token);
-      w[u] = reinterpret_cast<const uint2*>((is_q ? q : k) + row * kHeadDim)[lane];
-      which[u] = is_q ? 0 : 1;
+      w[u] = reinterpret_cast<const uint2*>(k + kv_row(pg, b, hkv, bg % hkv, n, token) * kHeadDim)[lane];
+      live[u] = true;
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
@@ -49,26 +45,23 @@ __global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16
       float s = a * a + b2 * b2 + c * c + d * d;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      if (which[u] >= 0 && s == s) best[which[u]] = fmaxf(best[which[u]], s);     // (a NaN row is left to the later stages)
+      if (live[u] && s == s) best = fmaxf(best, s);     // (a NaN row is left to the later stages)
     }
   }
-  if (lane == 0) {
-    if (best[0] > 0.f) atomicMax(reinterpret_cast<unsigned*>(mag), __float_as_uint(best[0]));
-    if (best[1] > 0.f) atomicMax(reinterpret_cast<unsigned*>(mag) + 1, __float_as_uint(best[1]));
-  }
+  if (lane == 0 && best > 0.f) atomicMax(reinterpret_cast<unsigned*>(k2max), __float_as_uint(best));
 }
 
 }  // namespace
 
-cudaError_t launch_kap_norms(const __nv_bfloat16* q, const __nv_bfloat16* k, const KvPaging& pg, int batch, int hq, int hkv, int n,
-                             int stride, float* mag, cudaStream_t st) {
-  cudaError_t e = cudaMemsetAsync(mag, 0, 2 * sizeof(float), st);
+cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, int batch, int hkv, int n, int stride, float* k2max,
+                             cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(k2max, 0, sizeof(float), st);
   if (e != cudaSuccess) return e;
-  const long long rows = (long long)batch * (hq + hkv) * (n / stride);
+  const long long rows = (long long)batch * hkv * (n / stride);
   long long blocks = (rows + 4 * (kThreads / 32) - 1) / (4 * (kThreads / 32));
   if (blocks > 148LL * 8) blocks = 148LL * 8;
   if (blocks < 1) blocks = 1;
-  kap_norms_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(q, k, pg, batch, hq, hkv, n, stride, mag);
+  kap_norms_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(k, pg, batch, hkv, n, stride, k2max);
   return cudaGetLastError();
 }
 

@@ -243,7 +243,29 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     float* parked = p.maxima + (size_t)ctl->slot * ((size_t)((ns + 127) / 128) * kTileFloats);
     float* mine = parked + ((size_t)grp * BPT + part * BPC) * R + r;
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
-    bool alive = true;
+    // squared norm of this thread's sampled query row, from the A tile in shared memory (a row is 2 x 128 bytes, one in
+    // each half tile; the swizzle permutes 16-byte chunks inside a row, which a sum of squares does not notice; the
+    // chunk order is rotated by the lane so that the rows of a warp hit different banks)
+    float q2 = 0.f;
+    bool alive = mbar_wait_warp(smem_u32(&ctl->a_full), 0, abort_flag, budget);
+    if (!alive && !*abort_flag) screen_timeout(ctl, status);
+    if (alive) {
+      const unsigned char* arow = smem + (size_t)rt * kTileBytes + (size_t)(row % 128) * 128;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 wv = *reinterpret_cast<const uint4*>(arow + (c >> 3) * kHalfBytes + (((c + lane) & 7) << 4));
+        const unsigned ws4[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const float lo = __uint_as_float(ws4[u] << 16), hi = __uint_as_float(ws4[u] & 0xffff0000u);
+          q2 = fmaf(lo, lo, fmaf(hi, hi, q2));
+        }
+      }
+      float g2 = q2;                                     // the group's rows are R consecutive lanes
+#pragma unroll
+      for (int o = 1; o < R; o <<= 1) g2 = fmaxf(g2, __shfl_xor_sync(0xffffffffu, g2, o));
+      if (part == 0 && r == 0 && row_ok) p.q2max[(size_t)(b * p.hq + h) * p.nqb + i] = g2;
+    }
     for (int t = 0; t < n_tiles && alive; ++t) {
       const int sb = t % kSteps, st = t % kStages;
       alive = mbar_wait_warp(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag, budget);   // this tile's MMAs finished
@@ -309,8 +331,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         }
       }
       // the row's best block, and whether the runner-up is too close to call
-      // (the threshold grows with the magnitude of the call's inputs, which is what the rounding error of a logit follows)
-      const float tau_row = fmaxf(p.tau_row, 2.f * screen_error_bound(p.mag[0], p.mag[1], p.scale));
+      // (the threshold grows with the magnitude of the row and of the call's keys, which is what the rounding error of a
+      // logit follows)
+      const float tau_row = fmaxf(p.tau_row, 2.f * screen_error_bound(q2, *p.k2max, p.scale));
       const bool amb = row_ok && (top1 - top2) * p.scale <= tau_row;
       const bool amb3 = row_ok && (top1 - top3) * p.scale <= tau_row;
       const unsigned any_amb = __ballot_sync(0xffffffffu, amb), any_amb3 = __ballot_sync(0xffffffffu, amb3);

@@ -383,8 +383,6 @@ __device__ void select_largest(const unsigned long long* a, int n, int want, uns
 
 __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapScreenParams sp, float tau_score, int sort_cap,
                                                             int tie_bytes, const int32_t* status) {
-  // near ties: never closer than twice what the screen may be off by on inputs of this call's magnitude
-  tau_score = fmaxf(tau_score, 2.f * screen_error_bound(sp.mag[0], sp.mag[1], sp.scale));
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);  // [sort_cap]
   unsigned char* tie = reinterpret_cast<unsigned char*>(keys + sort_cap);        // [tie_bytes]
@@ -416,10 +414,13 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
   }
   // a screen kernel that gave up has left the scratch half written: nothing of it may be used for addressing
   const int poisoned = *reinterpret_cast<const volatile int32_t*>(status);   // (tested together with `hard` below)
+  const float k2 = *sp.k2max;
   unsigned hard = 0u;                         // (tested only after the scores have been requested: one round trip, not two)
+  float q2 = 0.f;                             // largest squared norm among the block's sampled query rows
   unsigned long long amb = 0ULL;              // bit r: sampled row r of the block was too close to call
   for (int t = 0; t < T; ++t) {
     hard |= sp.hard[row_lo + t];
+    q2 = fmaxf(q2, sp.q2max[row_lo + t]);
     amb |= (unsigned long long)sp.ambmask[row_lo + t] << (t * R);
   }
   const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
@@ -466,6 +467,8 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
     }
   }
   if (poisoned != 0) return;
+  // near ties: never closer than twice what the screen may be off by on rows of this magnitude
+  tau_score = fmaxf(tau_score, 2.f * screen_error_bound(q2, k2, sp.scale));
   if (hard) {  // left to the double-precision kernel
     if (tid == 0) sp.redo_list[1 + atomicAdd(sp.redo_list, 1)] = (int)row_lo;
     return;

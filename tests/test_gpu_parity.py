@@ -770,6 +770,27 @@ def test_batch_with_different_lengths(impl, causal, n, lens):
     check(paged)
 
 
+def test_kv_head_shards_concatenate_to_the_unsharded_result(small):
+    """One layer split by KV-head group (what bench.py --shard kv_head gives each rank): every shard runs KAP + OSK on
+    its heads alone, here one after the other on one GPU, and the concatenated lists and outputs are those of the
+    unsharded call, bit for bit (work items of different KV heads share nothing)."""
+    from paper_2607_25291_b200.shard import shard_tensors
+    w = small["w"]
+    q, k, v = small["dev"]
+    whole_order, whole_count = run_kap(q, k, 0.5)
+    whole = run_osk(q, k, v, whole_order, whole_count, 0.3, 200.0)
+    for world in (2,):
+        parts = []
+        for rank in range(world):
+            qs, ks, vs = (t.contiguous() for t in shard_tensors(q, k, v, world, rank))
+            order, count = run_kap(qs, ks, 0.5)
+            parts.append((order, count, run_osk(qs, ks, vs, order, count, 0.3, 200.0)))
+        assert torch.equal(torch.cat([p[0] for p in parts], 1), whole_order)
+        assert torch.equal(torch.cat([p[1] for p in parts], 1), whole_count)
+        for key in ("out", "lse", "visited", "scored"):
+            assert torch.equal(torch.cat([p[2][key] for p in parts], 1), whole[key]), key
+
+
 def test_osk_is_deterministic(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
