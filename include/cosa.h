@@ -90,7 +90,11 @@ typedef struct {
                               but the sort stage of cosa_kap_select takes the route it otherwise
                               keeps for the lists its fastest route cannot settle: 2 = the head of
                               the order selected by radix, 3 = the whole order sorted (same lists,
-                              slower; for tests and comparisons)                                  */
+                              slower; for tests and comparisons); 4 = as 0, but cosa_osk_attention
+                              runs the kernel that walks two work items per CTA, each with a softmax
+                              group, an S and an O accumulator of its own (the arrangement a 256-row
+                              query block with one vote per 128-row tile takes; measured slower than
+                              one work item per CTA, kept for comparison)                          */
   float   top_p;           /* KAP only.  > 0: Top-p retention (Sec. 4.2, text after Eq. 13; p = 0.95
                               in Sec. C.1): K_i = length of the shortest prefix of the order whose
                               scores sum to >= top_p * (sum over all candidates), never more than

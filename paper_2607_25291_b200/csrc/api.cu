@@ -323,7 +323,7 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
     p.pg.seq_lens = lens;
   }
   p.wait_budget = o.wait_cycles > 0 ? (long long)o.wait_cycles : (1LL << 31);
-  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : launch_osk_tc(p, st);
+  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : (o.impl == 4 ? launch_osk_duo(p, st) : launch_osk_tc(p, st));
   if (e != cudaSuccess) return cuda_fail(e, "osk launch");
   return COSA_OK;
 }

@@ -21,6 +21,7 @@ pytestmark = pytest.mark.gpu
 
 OUT_MAX, OUT_MEAN, LSE_TOL, MARGIN = 2e-2, 2e-3, 1e-3, 1e-4
 IMPLS = (0, 1)
+OSK_IMPLS = (0, 1, 4)     # tensor-core kernel, CUDA-core check kernel, tensor-core kernel with two work items per CTA
 
 
 def _np(t):
@@ -366,7 +367,7 @@ def test_kap_query_group_sizes(hq, hkv, stride):
 
 
 # ---------------------------------------------------------------------------------- OSK
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 def test_osk_dense_path_matches_dense_attention(small, impl):
     """Full lists, Stage 2 off: the library's dense path (Property 2, Eq. 4)."""
     q, k, v = small["dev"]
@@ -389,7 +390,7 @@ def test_osk_dense_path_matches_dense_attention(small, impl):
         assert np.array_equal(_np(bufs["visited"]), count_np) and np.array_equal(_np(bufs["scored"]), count_np)
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 @pytest.mark.parametrize("tb,skip_scale", [(0.3, 200.0), (0.999, 100.0), (0.2, -1.0), (1.0, 200.0), (0.05, 500.0)])
 def test_osk_skip_rule_and_cap_small(small, impl, tb, skip_scale):
     q, k, v = small["dev"]
@@ -401,7 +402,7 @@ def test_osk_skip_rule_and_cap_small(small, impl, tb, skip_scale):
     check_osk_against_oracle(qf, kf, vf, order_np, count_np, bufs, tb, skip_scale, range(4), range(8))
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 def test_osk_4k_workload(cfg1, impl):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
@@ -414,7 +415,7 @@ def test_osk_4k_workload(cfg1, impl):
     print("4k", stats)
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 def test_osk_noncausal(small, impl):
     q, k, v = small["dev"]
     qf, kf, vf = small["f64"]
@@ -448,7 +449,7 @@ def test_list_tools_bit_exact(small, cfg1):
     assert _np(o3).tolist() == [[[5, -1, -1, -1], [0, 1, 2, 3]]]
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 @pytest.mark.parametrize("tb,skip_scale", [(1.0, 200.0), (0.4, 150.0)])
 def test_osk_logical_mask_walk(small, cfg1, impl, tb, skip_scale):
     """Walking the binary mask visits the kept blocks in ascending order: same decisions and outputs as the
@@ -570,7 +571,7 @@ def _pools(w, page_size):
     return dev(kpool), dev(vpool), torch.from_numpy(table).cuda()[None].contiguous(), kpool.shape[0]
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 @pytest.mark.parametrize("page_size", [8, 16, 32, 64, 128, 256])
 def test_paged_kv_small(small, impl, page_size):
     """Pools + page table give the lists and outputs of the dense tensors behind them (Sec. C.1)."""
@@ -660,7 +661,7 @@ def test_paged_kv_small_pages_with_caller_workspace(small):
 
 
 # ---------------------------------------------------------------------------------- batch > 1
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 def test_batch_of_two_equals_single_items(impl):
     """Two different sequences in one call give exactly the results of two calls (dense and paged)."""
     items = []
@@ -705,7 +706,7 @@ def test_batch_of_two_equals_single_items(impl):
         assert torch.equal(x, y)
 
 
-@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("impl", OSK_IMPLS)
 @pytest.mark.parametrize("causal", [True, False])
 @pytest.mark.parametrize("n,lens", [(1024, [1024, 640]), (4096, [1536, 4096])])
 def test_batch_with_different_lengths(impl, causal, n, lens):

@@ -43,26 +43,27 @@ def test_kap_wait_budget_of_one_cycle_reports_a_timeout_and_the_next_call_is_cle
     assert torch.equal(order, ref_order) and torch.equal(count, ref_count)
 
 
-def test_osk_wait_budget_of_one_cycle_reports_a_timeout_and_the_next_call_is_clean(cfg1):
+@pytest.mark.parametrize("impl", [0, 4])        # one work item per CTA, two work items per CTA
+def test_osk_wait_budget_of_one_cycle_reports_a_timeout_and_the_next_call_is_clean(cfg1, impl):
     w, (q, k, v) = cfg1["w"], cfg1["dev"]
     nqb = w.n // 128
     order, count = alloc_lists(w.hq, nqb)
     cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride))
     ref = alloc_outputs(q, nqb)
     cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, ref["out"], ref["lse"], ref["visited"],
-                            opt=cosa.default_options(skip_scale=w.skip_scale))
+                            opt=cosa.default_options(skip_scale=w.skip_scale, impl=impl))
     assert cosa.cosa_device_status() == 0
     for _ in range(2):                                  # twice: a timed-out call leaves nothing behind that trips the next
         bufs = alloc_outputs(q, nqb)
         bufs["visited"].fill_(-7)
         cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, bufs["out"], bufs["lse"], bufs["visited"],
-                                opt=cosa.default_options(skip_scale=w.skip_scale, wait_cycles=1))
+                                opt=cosa.default_options(skip_scale=w.skip_scale, wait_cycles=1, impl=impl))
         assert cosa.cosa_device_status() == TIMEOUT
         assert cosa.cosa_device_status() == 0
         assert int((bufs["visited"] == -7).sum()) > 0   # the CTAs that started after the first timeout returned at once
     bufs = alloc_outputs(q, nqb)
     cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, bufs["out"], bufs["lse"], bufs["visited"],
-                            opt=cosa.default_options(skip_scale=w.skip_scale))
+                            opt=cosa.default_options(skip_scale=w.skip_scale, impl=impl))
     assert cosa.cosa_device_status() == 0
     assert torch.equal(bufs["out"], ref["out"]) and torch.equal(bufs["visited"], ref["visited"])
     assert torch.equal(bufs["lse"], ref["lse"])
