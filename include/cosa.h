@@ -12,8 +12,9 @@
  *        maximum lies more than ln(N/Delta) below the running row maximum.
  *
  * Conventions
- *   - All tensors are dense, row-major, innermost dimension contiguous, base pointers
- *     16-byte aligned.  Layouts:
+ *   - All tensors are row-major with the innermost dimension contiguous, base pointers
+ *     16-byte aligned; q, k, v and out may carry their own strides (cosa_options.q_strides ...).
+ *     Default layouts:
  *         q, out              [B, Hq,  N, d]   bf16
  *         k, v                [B, Hkv, N, d]   bf16      (query head h reads KV head h / (Hq/Hkv));
  *                                                       or page pools, see cosa_options.kv_page_table
@@ -129,6 +130,15 @@ typedef struct {
                               (Eq. 5; skip_scale must stay below the shortest length) follow the
                               item's own length: every item comes out as in a call of its own.
                               Not with block_q = 256                                               */
+  /* Element strides (batch, head, token) of q, of k and v (one layout for both), and of out, for tensors that are
+     not the dense [B, H, N, d] default: e.g. the token-major [B, N, H, d] a fused QKV projection writes has strides
+     (N*H*d, d, H*d), and q, k, v may then be three base pointers into one buffer.  The d elements of a row stay
+     contiguous; every stride is a multiple of 8 elements (16 bytes) and the token stride at least d.  All three
+     zero: the dense layout.  kv_strides are not accepted together with kv_page_table (pools are contiguous by
+     definition); lse, lists and counters keep their dense layouts.  Results do not depend on the layout. */
+  int64_t q_strides[3];
+  int64_t kv_strides[3];
+  int64_t out_strides[3];
   int64_t wait_cycles;     /* Clock cycles a wait inside a kernel may take before the kernel gives up, sets the
                               device status word (see cosa_device_status) and returns without writing further
                               results.  0: the default, 2^31 (about a second).  A few cycles make every

@@ -43,7 +43,8 @@ class CosaOptions(Structure):
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p), ("kv_page_table", c_void_p),
-                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p), ("wait_cycles", ctypes.c_int64)]
+                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p), ("q_strides", ctypes.c_int64 * 3), ("kv_strides", ctypes.c_int64 * 3),
+                ("out_strides", ctypes.c_int64 * 3), ("wait_cycles", ctypes.c_int64)]
 
 
 class CosaError(RuntimeError):
@@ -139,12 +140,42 @@ def default_options(**kw) -> CosaOptions:
     return opt
 
 
+def _is_pool(opt) -> bool:
+    """k and v are page pools [P,Hkv,b_p,d] (contiguous by definition) rather than [B,Hkv,N,d] tensors."""
+    return opt is not None and bool(opt.kv_page_table)
+
+
 def _dev_ptr(t: torch.Tensor, dtype, name: str) -> int:
     if t is None:
         return 0
     if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
         raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
     return t.data_ptr()
+
+
+def _strided_ptr(t: torch.Tensor, name: str):
+    """Pointer and (batch, head, token) element strides of a [B,H,N,d] bf16 CUDA tensor or view whose rows are contiguous;
+    strides (0, 0, 0) stand for the dense layout."""
+    if t.dim() == 3:
+        t = t[None]                                         # [H,N,d]: one batch item
+    if not t.is_cuda or t.dtype != torch.bfloat16 or t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError(f"{name}: expected a [B,H,N,d] CUDA bfloat16 tensor with contiguous rows")
+    return t.data_ptr(), ((0, 0, 0) if t.is_contiguous() else tuple(int(x) for x in t.stride()[:3]))
+
+
+def _set_strides(opt, q=None, k=None, v=None, out=None):
+    """Writes the layouts of the call's tensors into the options (creating them when a tensor needs strides)."""
+    given = {"q_strides": q, "kv_strides": k, "out_strides": out}
+    if v is not None and k is not None and v != k:
+        raise ValueError("k and v must share one layout")
+    if opt is None:
+        if all(s is None or s == (0, 0, 0) for s in given.values()):
+            return None
+        opt = default_options()
+    for field, strides in given.items():
+        if strides is not None:
+            setattr(opt, field, (ctypes.c_int64 * 3)(*strides))
+    return opt
 
 
 def cosa_budget_count(budget: float, candidates: int) -> int:
@@ -162,7 +193,12 @@ def cosa_kap_select(q, k, budget: float, out_order, out_count, causal=True, stre
     lib = _load()
     shape = make_shape(q, k, causal)
     shape.block_q = block_q
-    args = (_dev_ptr(q, torch.bfloat16, "q"), _dev_ptr(k, torch.bfloat16, "k"), byref(shape), c_float(budget),
+    (qp, qstr), (kp, kstr) = _strided_ptr(q, "q"), _strided_ptr(k, "k") if k.dim() == 4 and not _is_pool(opt) else (_dev_ptr(k, torch.bfloat16, "k"), None)
+    had_opt = opt is not None
+    opt = _set_strides(opt, q=qstr, k=kstr)
+    if opt is not None and not had_opt:
+        opt.order_stride = out_order.shape[-1]
+    args = (qp, kp, byref(shape), c_float(budget),
             _dev_ptr(out_order, torch.int32, "out_order"), _dev_ptr(out_count, torch.int32, "out_count"),
             _stream_ptr(stream))
     if opt is None:
@@ -199,9 +235,18 @@ def cosa_osk_attention(q, k, v, order, count, tightened_budget: float, out, out_
     """Stage 2: fills out [B,Hq,N,d] bf16, out_lse [B,Hq,N] f32, out_visited [B,Hq,nQB] int32."""
     lib = _load()
     shape = make_shape(q, k, causal)
-    args = (_dev_ptr(q, torch.bfloat16, "q"), _dev_ptr(k, torch.bfloat16, "k"), _dev_ptr(v, torch.bfloat16, "v"),
+    (qp, qstr), (op, ostr) = _strided_ptr(q, "q"), _strided_ptr(out, "out")
+    if _is_pool(opt):
+        (kp, kstr), (vp, vstr) = (_dev_ptr(k, torch.bfloat16, "k"), None), (_dev_ptr(v, torch.bfloat16, "v"), None)
+    else:
+        (kp, kstr), (vp, vstr) = _strided_ptr(k, "k"), _strided_ptr(v, "v")
+    had_opt = opt is not None
+    opt = _set_strides(opt, q=qstr, k=kstr, v=vstr, out=ostr)
+    if opt is not None and not had_opt and order is not None:
+        opt.order_stride = order.shape[-1]
+    args = (qp, kp, vp,
             byref(shape), _dev_ptr(order, torch.int32, "order"), _dev_ptr(count, torch.int32, "count"),
-            c_float(tightened_budget), _dev_ptr(out, torch.bfloat16, "out"),
+            c_float(tightened_budget), op,
             _dev_ptr(out_lse, torch.float32, "out_lse"), _dev_ptr(out_visited, torch.int32, "out_visited"),
             _stream_ptr(stream))
     if opt is None:

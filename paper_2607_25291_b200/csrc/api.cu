@@ -88,6 +88,18 @@ int resolve_paging(const cosa_shape* s, const cosa_options& o, int stride, KvPag
   return COSA_OK;
 }
 
+// Strides of a q / k / v / out tensor from the three option words; all zero = the dense [B, H, N, d] layout.
+int resolve_strides(const int64_t* given, int batch, int heads, int n, Strides* out) {
+  *out = dense_strides(heads, n);
+  if (given[0] == 0 && given[1] == 0 && given[2] == 0) return COSA_OK;
+  const long long sb = given[0], sh = given[1], st = given[2];
+  if (st < kHeadDim || st % 8 != 0) return COSA_ERR_INVALID_ARG;
+  if ((heads > 1 && (sh <= 0 || sh % 8 != 0)) || (batch > 1 && (sb <= 0 || sb % 8 != 0))) return COSA_ERR_INVALID_ARG;
+  *out = Strides{batch > 1 ? sb : out->b, heads > 1 ? sh : out->h, st};
+  return COSA_OK;
+}
+bool strides_given(const int64_t* s) { return s[0] != 0 || s[1] != 0 || s[2] != 0; }
+
 cosa_options resolve_options(const cosa_options* opt) {
   cosa_options o;
   cosa_default_options(&o);
@@ -202,6 +214,10 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   if (p.qtiles == 2 && p.rows * 2 > 64) return COSA_ERR_UNSUPPORTED;                  // stride 2 and below
   rc = resolve_paging(shape, o, s, &p.pg);
   if (rc != COSA_OK) return rc;
+  if (p.pg.table && strides_given(o.kv_strides)) return COSA_ERR_INVALID_ARG;
+  rc = resolve_strides(o.q_strides, p.batch, p.hq, p.n, &p.qs);
+  if (rc == COSA_OK) rc = resolve_strides(o.kv_strides, p.batch, p.hkv, p.n, &p.ks);
+  if (rc != COSA_OK) return rc;
   // the list of the longest row must fit the pitch
   if (budget_count_fx(p.budget_fx, nqb) > order_stride) return COSA_ERR_INVALID_ARG;
   if (kap_exact_smem_bytes(p.rows, nqb, p.qtiles) > 227 * 1024) return COSA_ERR_UNSUPPORTED;
@@ -250,7 +266,8 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
     p.pg.seq_lens = lens;
   }
   sp.pg = p.pg;
-  cudaError_t e = launch_kap_norms(sp.k, sp.pg, p.batch, p.hkv, p.n, s, reinterpret_cast<float*>(ws + L.k2max), st);
+  sp.qs = p.qs; sp.ks = p.ks;
+  cudaError_t e = launch_kap_norms(sp.k, sp.pg, sp.ks, p.batch, p.hkv, p.n, s, reinterpret_cast<float*>(ws + L.k2max), st);
   if (e != cudaSuccess) return cuda_fail(e, "kap norms launch");
   e = launch_kap_screen(sp, st);
   if (e != cudaSuccess) return cuda_fail(e, "kap screen launch");
@@ -287,6 +304,11 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   p.mask = o.logical_mask;
   rc = resolve_paging(shape, o, 0, &p.pg);
   if (rc != COSA_OK) return rc;
+  if (p.pg.table && strides_given(o.kv_strides)) return COSA_ERR_INVALID_ARG;
+  rc = resolve_strides(o.q_strides, shape->batch, shape->hq, shape->n, &p.qs);
+  if (rc == COSA_OK) rc = resolve_strides(o.kv_strides, shape->batch, shape->hkv, shape->n, &p.ks);
+  if (rc == COSA_OK) rc = resolve_strides(o.out_strides, shape->batch, shape->hq, shape->n, &p.os);
+  if (rc != COSA_OK) return rc;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = out_lse; p.visited = out_visited;
   p.scored = o.out_scored; p.decisions = o.out_decisions;
@@ -322,6 +344,7 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
     p.pg = KvPaging{};
     p.pg.seq_lens = lens;
   }
+  if (!p.pg.table && !strides_given(o.kv_strides)) p.ks = dense_strides(p.hkv, p.n);
   p.wait_budget = o.wait_cycles > 0 ? (long long)o.wait_cycles : (1LL << 31);
   cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : (o.impl == 4 ? launch_osk_duo(p, st) : launch_osk_tc(p, st));
   if (e != cudaSuccess) return cuda_fail(e, "osk launch");
@@ -439,6 +462,7 @@ int cosa_prefill_host(const void* q_host, const void* k_host, const void* v_host
   o.workspace_bytes = L.total - L.scratch;
   o.kap_scores = nullptr; o.kap_flags = nullptr; o.out_scored = nullptr; o.out_decisions = nullptr;
   o.kv_page_table = nullptr;   // the host buffers are dense tensors
+  memset(o.q_strides, 0, sizeof(o.q_strides)); memset(o.kv_strides, 0, sizeof(o.kv_strides)); memset(o.out_strides, 0, sizeof(o.out_strides));
   o.logical_mask = nullptr;
 
   // One chunk per (batch item, KV head): its query heads, lists and outputs are contiguous slices of every tensor,

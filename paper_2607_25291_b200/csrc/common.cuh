@@ -37,11 +37,38 @@ __device__ __forceinline__ float item_theta(const KvPaging& pg, int b, float the
   return (float)log((double)skip_scale / (double)(blocks_b * kBlock));
 }
 
-// Row of the [rows, d] view of k / v that holds `token` of KV head g of batch item b.
-__host__ __device__ inline long long kv_row(const KvPaging& pg, int b, int hkv, int g, int n, int token) {
-  if (!pg.table) return ((long long)b * hkv + g) * n + token;
+// Element strides (batch, head, token) of a q / k / v / out tensor; the d elements of a row are contiguous.  The
+// default is the dense [B, H, N, d] layout; a token-major [B, N, H, d] tensor (what a fused QKV projection writes) has
+// t = H * d and h = d.
+struct Strides {
+  long long b, h, t;
+};
+inline Strides dense_strides(int heads, int n) { return Strides{(long long)heads * n * kHeadDim, (long long)n * kHeadDim, kHeadDim}; }
+__host__ __device__ inline long long elem_off(const Strides& s, int b, int h, long long token) {
+  return (long long)b * s.b + (long long)h * s.h + token * s.t;
+}
+
+// Element offset, in k / v, of the row of `token` of KV head g of batch item b: through the page table for pools
+// (which are contiguous [P, Hkv, b_p, d]), by the tensor's strides otherwise.
+__host__ __device__ inline long long kv_off(const KvPaging& pg, const Strides& s, int b, int hkv, int g, int token) {
+  if (!pg.table) return elem_off(s, b, g, token);
   const int page = pg.table[(long long)b * pg.pages_per_seq + (token >> pg.page_shift)];
-  return ((long long)page * hkv + g) * pg.page_size + (token & (pg.page_size - 1));
+  return (((long long)page * hkv + g) * pg.page_size + (token & (pg.page_size - 1))) * kHeadDim;
+}
+// Which coordinate of a 4-d tensor map (after the column) the row, the head and the outer index (batch item or page)
+// of a tile go to: the map lists its dimensions by ascending stride, whatever the tensor's layout is.
+struct TileOrder {
+  int row, head, outer;   // each 0, 1 or 2
+};
+// The same row as coordinates of the 4-d tensor maps over k / v: (row, head, batch item) for dense tensors,
+// (row inside the page, head, page) for pools.
+struct KvCoord {
+  int row, head, outer;
+};
+__device__ __forceinline__ KvCoord kv_coord(const KvPaging& pg, int b, int g, int token) {
+  if (!pg.table) return KvCoord{token, g, b};
+  const int page = pg.table[(long long)b * pg.pages_per_seq + (token >> pg.page_shift)];
+  return KvCoord{token & (pg.page_size - 1), g, page};
 }
 
 // Resolved call parameters handed to the kernels.
@@ -60,6 +87,7 @@ struct KapParams {
   long long budget_fx;   // floor(budget_f32 * 2^20)
   double scale;          // softmax scale applied to the sampled logits
   double top_p;          // > 0: Top-p retention, capped by the budget count; 0: budget count alone
+  Strides qs, ks;        // strides of q and of k (dense k; pools are contiguous)
   int qtiles;            // 1, or 2: one ranking per query block of 2 x 128 rows, shared by its two row tiles
   int sort_mode;         // sort stage of the fast path: 0 = as fast as it can, 1 = head selected by radix, 2 = everything sorted
   KvPaging pg;
@@ -84,6 +112,8 @@ struct KapScreenParams {
   int stride;
   float scale;
   float tau_row;         // two block maxima of a row closer than this (scaled logits) are "too close to call"
+  Strides qs, ks;        // strides of q and of k (dense k; pools are contiguous)
+  TileOrder qo, ko;      // coordinate order of the tensor maps over the sampled rows of q and of k (set by the launcher)
   long long wait_budget; // clock cycles a device-side wait may take before the kernel gives up
   KvPaging pg;
 };
@@ -110,6 +140,8 @@ struct OskParams {
   float skip_scale;      // Delta (for items whose own length replaces N, see item_theta)
   float scale;           // softmax scale
   long long wait_budget; // clock cycles a device-side wait may take before the kernel gives up
+  Strides qs, ks, os;    // strides of q, of k and v (dense; pools are contiguous), of out
+  TileOrder qo, ko, oo;  // coordinate order of the tensor maps over q, over k and v, over out (set by the launcher)
   KvPaging pg;
 };
 
@@ -177,8 +209,8 @@ int32_t* device_status_word();
 cudaError_t launch_kap_exact(const KapParams& p, const int32_t* redo_list, cudaStream_t st);
 bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg);
 cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st);
-cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, int batch, int hkv, int n, int stride, float* k2max,
-                             cudaStream_t st);
+cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, const Strides& ks, int batch, int hkv, int n, int stride,
+                             float* k2max, cudaStream_t st);
 // CTAs of the screen kernel that can be resident at once on the current device (0 on failure), and the bytes of
 // block-maxima scratch each of them needs
 int kap_screen_slots();
@@ -190,7 +222,7 @@ size_t kap_exact_smem_bytes(int rows, int nqb, int qtiles);
 // copies the pages of the call's sequences into a dense [B, Hkv, N, d] tensor (pools with pages smaller than a key block);
 // every > 1: only the rows whose token index is a multiple of it
 cudaError_t launch_gather_pages(const __nv_bfloat16* pool, __nv_bfloat16* dense, const KvPaging& pg, int batch, int hkv, int n,
-                                int every, cudaStream_t st);
+                                int every, cudaStream_t st);   // (pools are contiguous; the staging tensor is dense)
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_duo(const OskParams& p, cudaStream_t st);

@@ -68,7 +68,7 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
   unsigned* ids = reinterpret_cast<unsigned*>(keys + sort_cap);
   unsigned char* flag = reinterpret_cast<unsigned char*>(ids + sort_cap);   // [Jpad]
 
-  const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+  const __nv_bfloat16* qh = p.q + elem_off(p.qs, b, h, 0);
   for (int j = tid; j < J; j += kThreads) { score[j] = 0.0; flag[j] = 0; }
 
   // one row tile after the other: its block maxima M[r,j], its row maxima M*[r], its share of the sums of Eq. (11)
@@ -78,7 +78,7 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
     for (int e = tid; e < R * kHeadDim; e += kThreads) {
       int r = e / kHeadDim, d = e % kHeadDim;
       size_t tok = (size_t)(row0 + r) * p.stride;
-      Qs[r * kPad + d] = (double)__bfloat162float(qh[tok * kHeadDim + d]);
+      Qs[r * kPad + d] = (double)__bfloat162float(qh[tok * p.qs.t + d]);
     }
     for (int j0 = 0; j0 < J; j0 += kb_per_iter) {
       const int nb = min(kb_per_iter, J - j0);
@@ -86,7 +86,7 @@ __device__ void kap_exact_item(const KapParams& p, const int b, const int h, con
       for (int e = tid; e < nb * R * kHeadDim; e += kThreads) {
         int c = e / kHeadDim, d = e % kHeadDim;  // c: sampled key within this group of blocks
         const int tok = (j0 * R + c) * p.stride;
-        Ks[c * kPad + d] = (double)__bfloat162float(p.k[(size_t)kv_row(p.pg, b, p.hkv, g, p.n, tok) * kHeadDim + d]);
+        Ks[c * kPad + d] = (double)__bfloat162float(p.k[kv_off(p.pg, p.ks, b, p.hkv, g, tok) + d]);
       }
       __syncthreads();
       for (int e = tid; e < nb * R * R; e += kThreads) {

@@ -14,8 +14,8 @@ constexpr int kThreads = 256;
 
 // one warp per row and turn, four rows in flight per warp; *k2max = max |k_row|^2 over the sampled key rows (bit
 // patterns of non-negative floats order like unsigned integers, so atomicMax on the bits is a float maximum)
-__global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16* __restrict__ k, KvPaging pg, int batch, int hkv,
-                                                             int n, int stride, float* k2max) {
+__global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16* __restrict__ k, KvPaging pg, Strides ks, int batch,
+                                                             int hkv, int n, int stride, float* k2max) {
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * kThreads + threadIdx.x) >> 5;
   const long long n_warps = ((long long)gridDim.x * kThreads) >> 5;
@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16
       const int bg = (int)(r / ns);
       const int b = bg / hkv;
       if (pg.seq_lens && token >= pg.seq_lens[b]) continue;      // padding past the item's length
-      w[u] = reinterpret_cast<const uint2*>(k + kv_row(pg, b, hkv, bg % hkv, n, token) * kHeadDim)[lane];
+      w[u] = reinterpret_cast<const uint2*>(k + kv_off(pg, ks, b, hkv, bg % hkv, token))[lane];
       live[u] = true;
     }
 #pragma unroll
@@ -53,15 +53,15 @@ __global__ void __launch_bounds__(kThreads) kap_norms_kernel(const __nv_bfloat16
 
 }  // namespace
 
-cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, int batch, int hkv, int n, int stride, float* k2max,
-                             cudaStream_t st) {
+cudaError_t launch_kap_norms(const __nv_bfloat16* k, const KvPaging& pg, const Strides& ks, int batch, int hkv, int n, int stride,
+                             float* k2max, cudaStream_t st) {
   cudaError_t e = cudaMemsetAsync(k2max, 0, sizeof(float), st);
   if (e != cudaSuccess) return e;
   const long long rows = (long long)batch * hkv * (n / stride);
   long long blocks = (rows + 4 * (kThreads / 32) - 1) / (4 * (kThreads / 32));
   if (blocks > 148LL * 8) blocks = 148LL * 8;
   if (blocks < 1) blocks = 1;
-  kap_norms_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(k, pg, batch, hkv, n, stride, k2max);
+  kap_norms_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(k, pg, ks, batch, hkv, n, stride, k2max);
   return cudaGetLastError();
 }
 

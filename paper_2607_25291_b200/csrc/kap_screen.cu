@@ -26,6 +26,7 @@
 
 #include "common.cuh"
 #include "ptx_sm100.cuh"
+#include "tile_maps.cuh"
 
 namespace cosa {
 namespace {
@@ -149,13 +150,11 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       mbar_expect_tx(smem_u32(&ctl->a_full), kRowTiles * kTileBytes);
       for (int grp = 0; grp < kGroups; ++grp) {
         const int i = i0 + grp / G, h = g * G + grp % G;
-        const int row = (b * p.hq + h) * ns + i * R;   // rows past the tensor are zero-filled
-        const uint32_t dst = a_sm + (grp * R / 128) * kTileBytes + (grp * R % 128) * 128;
-        tma_load_2d(dst, &q_map, 0, row, smem_u32(&ctl->a_full));
-        tma_load_2d(dst + kHalfBytes, &q_map, 64, row, smem_u32(&ctl->a_full));
+        const uint32_t dst = a_sm + (grp * R / 128) * kTileBytes + (grp * R % 128) * 128;   // (rows past the head's last are zero-filled)
+        tma_load_tile(dst, &q_map, 0, i * R, h, b, p.qo.row, p.qo.head, p.qo.outer, smem_u32(&ctl->a_full));
+        tma_load_tile(dst + kHalfBytes, &q_map, 64, i * R, h, b, p.qo.row, p.qo.head, p.qo.outer, smem_u32(&ctl->a_full));
       }
       if (!p.pg.table) {
-        const int krow0 = (b * p.hkv + g) * ns;
         for (int t = 0; t < n_tiles; ++t) {
           const int st = t % kStages;
           if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((t / kStages) & 1) ^ 1, abort_flag, budget)) {
@@ -164,8 +163,8 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
           }
           const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
           mbar_expect_tx(bar, kTileBytes);
-          tma_load_2d(dst, &k_map, 0, krow0 + t * 128, bar);
-          tma_load_2d(dst + kHalfBytes, &k_map, 64, krow0 + t * 128, bar);
+          tma_load_tile(dst, &k_map, 0, t * 128, g, b, p.ko.row, p.ko.head, p.ko.outer, bar);
+          tma_load_tile(dst + kHalfBytes, &k_map, 64, t * 128, g, b, p.ko.row, p.ko.head, p.ko.outer, bar);
           t_issued = t + 1;
         }
       }
@@ -190,9 +189,9 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
         if (lane < parts) {
           int tok = (t * 128 + lane * spp) * p.stride;
           if (tok >= nqb_b * kBlock) tok = 0;      // past the item's length: masked later, any valid page will do
-          const int srow = (int)(kv_row(p.pg, b, p.hkv, g, p.n, tok) / p.stride);
-          tma_load_2d(dst + lane * spp * 128, &k_map, 0, srow, bar);
-          tma_load_2d(dst + kHalfBytes + lane * spp * 128, &k_map, 64, srow, bar);
+          const KvCoord c = kv_coord(p.pg, b, g, tok);        // (a page's first sampled row is a multiple of the stride)
+          tma_load_tile(dst + lane * spp * 128, &k_map, 0, c.row / p.stride, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+          tma_load_tile(dst + kHalfBytes + lane * spp * 128, &k_map, 64, c.row / p.stride, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
         }
         __syncwarp();
         t_issued = t + 1;
@@ -467,35 +466,6 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-// every `stride`-th row of a [rows, 128] bf16 matrix, as boxes of `box_rows` sampled rows x 64 columns
-bool make_strided_map(CUtensorMap* map, const void* basep, uint64_t sampled_rows, int stride, int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)sampled_rows};
-  cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2 * (cuuint64_t)stride};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(basep), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool kap_screen_supported(int rows, int group, int stride, const KvPaging& pg) {
@@ -522,18 +492,26 @@ size_t kap_screen_slot_bytes(int n, int stride) {
   return ((ns + 127) / 128) * kRows * (128 / R) * sizeof(float);
 }
 
-cudaError_t launch_kap_screen(const KapScreenParams& p, cudaStream_t st) {
+cudaError_t launch_kap_screen(const KapScreenParams& p_in, cudaStream_t st) {
+  KapScreenParams p = p_in;
   const int R = 128 / p.stride;
   if (!p.maxima || !p.slot_taken || p.slots <= 0) return cudaErrorInvalidValue;
   cudaError_t e0 = cudaMemsetAsync(p.slot_taken, 0, (size_t)p.slots * sizeof(int32_t), st);
   if (e0 != cudaSuccess) return e0;
   const uint64_t ns = (uint64_t)p.n / p.stride;
   CUtensorMap qm, km;
-  const uint64_t k_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * (p.pg.page_size / p.stride) : (uint64_t)p.batch * p.hkv * ns;
+  // every `stride`-th row of q and k: the row stride of the maps is `stride` rows of the tensor (of the page pool)
   const int k_box = p.pg.table ? ((p.pg.page_size / p.stride) < 128 ? p.pg.page_size / p.stride : 128) : 128;
-  if (!make_strided_map(&qm, p.q, (uint64_t)p.batch * p.hq * ns, p.stride, R) ||
-      !make_strided_map(&km, p.k, k_rows, p.stride, k_box))
-    return cudaErrorInvalidValue;
+  const Strides qs = {p.qs.b, p.qs.h, p.qs.t * p.stride};
+  bool ok = make_tile_map(&qm, &p.qo, p.q, ns, (uint64_t)p.hq, (uint64_t)p.batch, qs, R);
+  if (p.pg.table) {
+    const Strides pool = dense_strides(p.hkv, p.pg.page_size);
+    ok = ok && make_tile_map(&km, &p.ko, p.k, (uint64_t)(p.pg.page_size / p.stride), (uint64_t)p.hkv, (uint64_t)p.pg.num_pages,
+                             Strides{pool.b, pool.h, pool.t * p.stride}, k_box);
+  } else {
+    ok = ok && make_tile_map(&km, &p.ko, p.k, ns, (uint64_t)p.hkv, (uint64_t)p.batch, Strides{p.ks.b, p.ks.h, p.ks.t * p.stride}, k_box);
+  }
+  if (!ok) return cudaErrorInvalidValue;
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;
   const int grid = kap_screen_grid(p.batch, p.hq, p.hkv, p.nqb, p.stride);

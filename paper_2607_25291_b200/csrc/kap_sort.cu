@@ -83,7 +83,7 @@ __device__ void f64_block_maxima(const KapParams& p, const double* Qs, int b, in
       named[u] = j >= 0;
       live[u] = named[u] && (!p.causal || kc <= row0 + r);
       qs[u] = Qs + r * kPad;
-      ks[u] = reinterpret_cast<const uint4*>(p.k + (size_t)kv_row(p.pg, b, p.hkv, g, p.n, (live[u] ? kc : 0) * p.stride) * kHeadDim);
+      ks[u] = reinterpret_cast<const uint4*>(p.k + kv_off(p.pg, p.ks, b, p.hkv, g, (live[u] ? kc : 0) * p.stride));
     }
     double z[2];
     if (e0 - tid + kThreads < items) {
@@ -129,7 +129,7 @@ __device__ void f64_block_maxima_shared_key(const KapParams& p, const double* Qs
     const bool valid = e < items;
     const int set = valid ? e / per_set : 0, ch = (e / R) % chunks, c = e % R;
     const int kc = block_of(set) * R + c;        // sampled key index
-    const uint4* ks = reinterpret_cast<const uint4*>(p.k + (size_t)kv_row(p.pg, b, p.hkv, g, p.n, kc * p.stride) * kHeadDim);
+    const uint4* ks = reinterpret_cast<const uint4*>(p.k + kv_off(p.pg, p.ks, b, p.hkv, g, kc * p.stride));
     const double* q0 = Qs + (size_t)(ch * kRowsPer) * kPad;
     double acc[kRowsPer];
 #pragma unroll
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
     q2 = fmaxf(q2, sp.q2max[row_lo + t]);
     amb |= (unsigned long long)sp.ambmask[row_lo + t] << (t * R);
   }
-  const __nv_bfloat16* qh = p.q + ((size_t)(b * p.hq + h) * p.n) * kHeadDim;
+  const __nv_bfloat16* qh = p.q + elem_off(p.qs, b, h, 0);
 
   // scores of the block = sum over its row tiles (the sum of Eq. 11 splits over the rows), flags = OR; a tile has
   // no score for key blocks wholly after it
@@ -483,7 +483,7 @@ __global__ void __launch_bounds__(kThreads, 6) kap_sort_kernel(KapParams p, KapS
     if (!have_q) {
       for (int e = tid; e < RT * kHeadDim; e += kThreads) {
         const int r = e / kHeadDim, d = e % kHeadDim;
-        Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i_lo * R + r) * p.stride) * kHeadDim + d]);
+        Qs[r * kPad + d] = (double)__bfloat162float(qh[((size_t)(i_lo * R + r) * p.stride) * p.qs.t + d]);
       }
       __syncthreads();
       have_q = true;

@@ -23,8 +23,8 @@ __global__ void __launch_bounds__(256) gather_pages_kernel(const uint4* __restri
     const int bg = (int)(row / rows);
     const int b = bg / hkv, g = bg % hkv;
     if (pg.seq_lens && token >= pg.seq_lens[b]) continue;   // padding: never read as keys
-    const long long src = kv_row(pg, b, hkv, g, n, token);
-    dense[((long long)bg * n + token) * kChunks + c] = pool[src * kChunks + c];
+    const long long src = kv_off(pg, Strides{0, 0, 0}, b, hkv, g, token) / 8;   // (pools only: 16-byte chunks)
+    dense[((long long)bg * n + token) * kChunks + c] = pool[src + c];
   }
 }
 

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
   // this thread's query row as packed bf16 pairs
   uint32_t qreg[kHeadDim / 2];
   {
-    const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)(b * p.hq + h) * p.n) + (size_t)i * kBlock + t) * kHeadDim);
+    const uint4* src = reinterpret_cast<const uint4*>(p.q + elem_off(p.qs, b, h, i * kBlock + t));
 #pragma unroll
     for (int c = 0; c < kHeadDim / 8; ++c) {
       uint4 w = src[c];
@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
     __syncthreads();
     for (int e = t; e < kBlock * kHeadDim / 8; e += kRows) {
       // row e / 16 of the block, 16-byte chunk e % 16 of that row, through the page table if there is one
-      const size_t src = (size_t)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock + e / (kHeadDim / 8)) * (kHeadDim / 8) + e % (kHeadDim / 8);
+      const size_t src = (size_t)kv_off(p.pg, p.ks, b, p.hkv, g, j * kBlock + e / (kHeadDim / 8)) / 8 + e % (kHeadDim / 8);
       reinterpret_cast<uint4*>(Ksm)[e] = kbase[src];
       reinterpret_cast<uint4*>(Vsm)[e] = vbase[src];
     }
@@ -119,7 +119,7 @@ __global__ void __launch_bounds__(kRows) osk_check_kernel(OskParams p) {
     ++computed;
   }
   const float inv = l > 0.f ? 1.f / l : 0.f;  // l > 0 whenever count >= 1
-  __nv_bfloat16* dst = p.out + (((size_t)(b * p.hq + h) * p.n) + (size_t)i * kBlock + t) * kHeadDim;
+  __nv_bfloat16* dst = p.out + elem_off(p.os, b, h, i * kBlock + t);
 #pragma unroll
   for (int d = 0; d < kHeadDim; d += 2) {
     __nv_bfloat162 o2 = __floats2bfloat162_rn(O[d] * inv, O[d + 1] * inv);

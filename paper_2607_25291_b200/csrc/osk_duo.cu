@@ -78,10 +78,10 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 // the page holds whole blocks (pools with smaller pages reach this kernel as dense staging tensors).
 __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensorMap* map, uint32_t dst, int b, int g, int j,
                                               uint32_t bar) {
-  const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock);
+  const KvCoord c = kv_coord(p.pg, b, g, j * kBlock);
   mbar_expect_tx(bar, kTileBytes);
-  tma_load_2d(dst, map, 0, row, bar);
-  tma_load_2d(dst + kHalfBytes, map, 64, row, bar);
+  tma_load_tile(dst, map, 0, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+  tma_load_tile(dst + kHalfBytes, map, 64, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
 }
 
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk)
@@ -124,7 +124,7 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
   if (kMask) walk.init(p, row, J);
   const int cnt = (!valid || i >= nqb_b) ? 0 : (kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride)));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
-  const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N, d] view
+  const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N] view of lse
   const long long budget = p.wait_budget;
 
   const bool issuer = warp < 2 && lane == 0;
@@ -154,8 +154,8 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
     if (pois == 0 && cnt > 0) {
       const uint32_t qb = smem_u32(&ctl->q_full[t]);
       mbar_expect_tx(qb, kTileBytes);
-      tma_load_2d(q_sm, &q_map, 0, q_row0, qb);
-      tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, qb);
+      tma_load_tile(q_sm, &q_map, 0, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, qb);
+      tma_load_tile(q_sm + kHalfBytes, &q_map, 64, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, qb);
       load_kv_block(p, &k_map, x_sm, b, g, min(max(j0, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][0]));
       if (cnt > 1) load_kv_block(p, &k_map, x_sm + kTileBytes, b, g, min(max(j1, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][1]));
     }
@@ -261,7 +261,7 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
       // an empty list (not produced by KAP) or padding past the item's length: zero output, nothing visited
       if (valid) {
         uint4 z = make_uint4(0, 0, 0, 0);
-        uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)q_row0 + r) * kHeadDim);
+        uint4* dst = reinterpret_cast<uint4*>(p.out + elem_off(p.os, b, h, i * kBlock + r));
         for (int c = 0; c < kHeadDim / 8; ++c) dst[c] = z;
         if (p.lse) p.lse[(size_t)q_row0 + r] = -INFINITY;
         if (leader) {
@@ -427,8 +427,8 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
         bar_sync(bar_id, kBlock);
         if (p.lse) p.lse[(size_t)q_row0 + r] = (n > 0 && l > 0.f) ? (m_run + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (leader) {
-          tma_store_2d(&o_map, 0, q_row0, x_sm);
-          tma_store_2d(&o_map, 64, q_row0, x_sm + kHalfBytes);
+          tma_store_tile(&o_map, 0, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, x_sm);
+          tma_store_tile(&o_map, 64, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, x_sm + kHalfBytes);
           tma_store_commit_and_wait_read();
           if (p.visited) p.visited[row] = n;
           if (p.scored) p.scored[row] = k_end + 1;
@@ -445,13 +445,15 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
 
 }  // namespace
 
-cudaError_t launch_osk_duo(const OskParams& p, cudaStream_t st) {
+cudaError_t launch_osk_duo(const OskParams& p_in, cudaStream_t st) {
   CUtensorMap qm, km, vm, om;
+  OskParams p = p_in;
+  TileOrder vo;
   // K and V: the dense tensors, or page pools whose pages hold whole key blocks
-  const uint64_t kv_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * p.pg.page_size : (uint64_t)p.batch * p.hkv * p.n;
   if (p.pg.table && p.pg.page_size < kBlock) return cudaErrorInvalidValue;   // staged as dense tensors by the caller of this launcher
-  if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, kv_rows) ||
-      !make_tile_map(&vm, p.v, kv_rows) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
+  if (!make_tile_map(&qm, &p.qo, p.q, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.qs) ||
+      !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n) || !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n) ||
+      !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
   auto kernel = p.mask ? osk_duo_kernel<true> : osk_duo_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

@@ -97,9 +97,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensorMap* map, uint32_t dst, int b, int g, int j,
                                               uint32_t bar) {
   // a page holds whole key blocks (pools with smaller pages reach this kernel as dense staging tensors)
-  const int row = (int)kv_row(p.pg, b, p.hkv, g, p.n, j * kBlock);
-  tma_load_2d(dst, map, 0, row, bar);
-  tma_load_2d(dst + kHalfBytes, map, 64, row, bar);
+  const KvCoord c = kv_coord(p.pg, b, g, j * kBlock);
+  tma_load_tile(dst, map, 0, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+  tma_load_tile(dst + kHalfBytes, map, 64, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
 }
 
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
@@ -139,7 +139,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   if (kMask) walk.init(p, row, J);
   const int cnt = i >= nqb_b ? 0 : (kMask ? min(walk.kept(), p.order_stride) : max(0, min(p.count[row], p.order_stride)));
   const int cap = p.stage2 ? min(cnt, budget_count_fx(p.cap_fx, J)) : cnt;
-  const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N, d] view
+  const int q_row0 = (b * p.hq + h) * p.n + i * kBlock;   // row of the [B*Hq*N] view of lse
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -181,8 +181,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     mbar_fence_init();
     fence_proxy_async_smem();
     mbar_expect_tx(smem_u32(&ctl->q_stage), kTileBytes);
-    tma_load_2d(q_sm, &q_map, 0, q_row0, smem_u32(&ctl->q_stage));
-    tma_load_2d(q_sm + kHalfBytes, &q_map, 64, q_row0, smem_u32(&ctl->q_stage));
+    tma_load_tile(q_sm, &q_map, 0, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, smem_u32(&ctl->q_stage));
+    tma_load_tile(q_sm + kHalfBytes, &q_map, 64, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, smem_u32(&ctl->q_stage));
     // once some CTA has reported a timeout the rest of the grid returns at once
     ctl->poisoned = poisoned_early;
     ctl->n_needed = min(cnt, cap);
@@ -407,7 +407,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     if (warp < 8) {
       const int r = (warp & 3) * 32 + lane;
       uint4 z = make_uint4(0, 0, 0, 0);
-      uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)q_row0 + r) * kHeadDim);
+      uint4* dst = reinterpret_cast<uint4*>(p.out + elem_off(p.os, b, h, i * kBlock + r));
       for (int c = 0; c < kHeadDim / 8; ++c) dst[c] = z;
       if (p.lse) p.lse[(size_t)q_row0 + r] = -INFINITY;
       if (threadIdx.x == 128) {
@@ -601,8 +601,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           if (p.lse) p.lse[(size_t)q_row0 + r] = (mf + log2f(lt)) * 0.6931471805599453f;
           if (r == 0) {
             if (mbar_wait(smem_u32(&ctl->out_bar), 0, abort_flag, budget)) {
-              tma_store_2d(&o_map, 0, q_row0, k_sm);
-              tma_store_2d(&o_map, 64, q_row0, k_sm + kHalfBytes);
+              tma_store_tile(&o_map, 0, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, k_sm);
+              tma_store_tile(&o_map, 64, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, k_sm + kHalfBytes);
               tma_store_commit_and_wait_read();
             } else if (!*abort_flag) {
               report_timeout(ctl, status);
@@ -625,14 +625,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
 
 }  // namespace
 
-cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st) {
+cudaError_t launch_osk_tc(const OskParams& p_in, cudaStream_t st) {
   CUtensorMap qm, km, vm, om;
+  OskParams p = p_in;
+  TileOrder vo;
   // K and V: the dense tensors, or page pools whose pages hold whole key blocks
-  const uint64_t kv_rows = p.pg.table ? (uint64_t)p.pg.num_pages * p.hkv * p.pg.page_size : (uint64_t)p.batch * p.hkv * p.n;
   if (p.pg.table && p.pg.page_size < kBlock) return cudaErrorInvalidValue;   // staged as dense tensors by the caller of this launcher
-  const int kv_box = kBlock;
-  if (!make_tile_map(&qm, p.q, (uint64_t)p.batch * p.hq * p.n) || !make_tile_map(&km, p.k, kv_rows, kv_box) ||
-      !make_tile_map(&vm, p.v, kv_rows, kv_box) || !make_tile_map(&om, p.out, (uint64_t)p.batch * p.hq * p.n))
+  if (!make_tile_map(&qm, &p.qo, p.q, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.qs) ||
+      !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n) || !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n) ||
+      !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
   auto kernel = p.mask ? osk_tc_kernel<true> : osk_tc_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);

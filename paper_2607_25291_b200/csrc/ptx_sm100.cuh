@@ -92,6 +92,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(dst),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+      : "memory");
+}
+// (c0, c1, c2: the tile's row, head and outer index in the order the tensor map lists those dimensions)
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, int x, int row, int head, int outer, int slot_row,
+                                              int slot_head, int slot_outer, uint32_t bar) {
+  const int c0 = slot_row == 0 ? row : (slot_head == 0 ? head : outer);
+  const int c1 = slot_row == 1 ? row : (slot_head == 1 ? head : outer);
+  const int c2 = slot_row == 2 ? row : (slot_head == 2 ? head : outer);
+  tma_load_4d(dst, map, x, c0, c1, c2, bar);
+}
 // contiguous global bytes -> shared memory (both 16-byte aligned, size a multiple of 16), with an L2 eviction policy
 __device__ __forceinline__ void bulk_load_hint(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
   asm volatile(
@@ -107,6 +121,19 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int 
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(reinterpret_cast<uint64_t>(map)),
                "r"(x), "r"(y), "r"(src)
                : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, int x, int y, int z, int w, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                   reinterpret_cast<uint64_t>(map)),
+               "r"(x), "r"(y), "r"(z), "r"(w), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_tile(const CUtensorMap* map, int x, int row, int head, int outer, int slot_row, int slot_head,
+                                               int slot_outer, uint32_t src) {
+  const int c0 = slot_row == 0 ? row : (slot_head == 0 ? head : outer);
+  const int c1 = slot_row == 1 ? row : (slot_head == 1 ? head : outer);
+  const int c2 = slot_row == 2 ? row : (slot_head == 2 ? head : outer);
+  tma_store_4d(map, x, c0, c1, c2, src);
 }
 __device__ __forceinline__ void tma_store_commit_and_wait_read() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");

@@ -1,5 +1,7 @@
-// Host-side construction of the TMA tensor maps the OSK kernels use: a [rows, 128] bf16 row-major view fetched as
-// boxes of box_rows x 64 columns with the 128-byte swizzle (the layout the tcgen05 shared-memory descriptors read).
+// Host-side construction of the TMA tensor maps of the tensor-core kernels: a bf16 tensor [outer, heads, rows, 128]
+// with arbitrary (outer, head, row) strides and contiguous rows of 128 elements, fetched as boxes of box_rows x 64
+// columns with the 128-byte swizzle (the layout the tcgen05 shared-memory descriptors read).  Dense q / k / v / out
+// tensors are [B, H, N, d] in whatever strides the caller gives; page pools are [P, Hkv, b_p, d], contiguous.
 #pragma once
 
 #include <cuda.h>
@@ -27,17 +29,49 @@ inline EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-inline bool make_tile_map(CUtensorMap* map, const void* basep, uint64_t rows, int box_rows = kBlock) {
+// `s` in elements; `rows`, `heads`, `outer` the extents.  The map lists the three dimensions by ascending stride (a
+// token-major tensor has its head stride below its row stride) and *order says where each went; boxes are box_rows
+// rows of one head of one outer index.  False if the strides cannot be mapped (not multiples of 16 bytes, or equal).
+inline bool make_tile_map(CUtensorMap* map, TileOrder* order, const void* basep, uint64_t rows, uint64_t heads, uint64_t outer,
+                          const Strides& s, int box_rows = kBlock) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(basep), dims, strides, box, estr,
+  struct Dim { long long stride; uint64_t extent; int what; } d[3] = {{s.t, rows, 0}, {s.h, heads, 1}, {s.b, outer, 2}};
+  long long span = kHeadDim;                                      // elements the dimensions that do move reach over
+  for (int a = 0; a < 3; ++a) {
+    if (d[a].extent == 1) continue;
+    if (d[a].stride <= 0 || d[a].stride % 8 != 0) return false;
+    if (d[a].stride * (long long)d[a].extent > span) span = d[a].stride * (long long)d[a].extent;
+  }
+  for (int a = 0; a < 3; ++a)
+    if (d[a].extent == 1) d[a].stride = span;                     // a dimension of extent 1 never moves: it goes outermost
+  for (int a = 0; a < 3; ++a)
+    for (int b = a + 1; b < 3; ++b)
+      if (d[b].stride < d[a].stride) { Dim t = d[a]; d[a] = d[b]; d[b] = t; }
+  cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, 1, 1, 1};
+  cuuint64_t strides[3] = {0, 0, 0};
+  cuuint32_t box[4] = {64, 1, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  int slot[3] = {0, 0, 0};
+  for (int a = 0; a < 3; ++a) {
+    dims[a + 1] = d[a].extent;
+    strides[a] = (cuuint64_t)d[a].stride * 2;
+    slot[d[a].what] = a;
+    if (d[a].what == 0) box[a + 1] = (cuuint32_t)box_rows;
+  }
+  order->row = slot[0]; order->head = slot[1]; order->outer = slot[2];
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(basep), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// k or v of a call: the dense tensor in its strides, or the page pool
+inline bool make_kv_map(CUtensorMap* map, TileOrder* order, const void* basep, const KvPaging& pg, const Strides& s, int batch,
+                        int hkv, int n, int box_rows = kBlock) {
+  if (!pg.table) return make_tile_map(map, order, basep, (uint64_t)n, (uint64_t)hkv, (uint64_t)batch, s, box_rows);
+  return make_tile_map(map, order, basep, (uint64_t)pg.page_size, (uint64_t)hkv, (uint64_t)pg.num_pages,
+                       dense_strides(hkv, pg.page_size), box_rows);
 }
 
 }  // namespace cosa

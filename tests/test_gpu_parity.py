@@ -5,6 +5,7 @@ list positions whose oracle skip margin |gap - theta| / |theta| is below 1e-4 (e
 is then accepted and the comparison follows the GPU's choice there); OSK outputs (bf16 inputs,
 fp32 accumulation) within max-abs 2e-2 and mean-abs 2e-3 of the oracle, LSE within 1e-3.
 """
+import ctypes
 import math
 
 import numpy as np
@@ -769,6 +770,48 @@ def test_batch_with_different_lengths(impl, causal, n, lens):
     paged = run(q2, kpool, vpool, 2, n, seq_lens=seq_lens, kv_page_table=table, kv_page_size=page_size,
                 kv_num_pages=kpool.shape[0])
     check(paged)
+
+
+@pytest.mark.parametrize("impl", OSK_IMPLS)
+def test_token_major_and_fused_qkv_layouts(cfg1, impl):
+    """q, k, v as three views into one token-major buffer [B, N, Hq + 2 Hkv, d] (what a fused QKV projection writes) and
+    out as a view of a token-major [B, N, Hq, d] tensor: passed by their strides, no transpose copy, and every
+    result equals the dense call's bit for bit."""
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    nqb = w.n // 128
+    dense_order, dense_count = run_kap(q, k, w.kap_budget, w.stride, impl=impl)
+    dense = run_osk(q, k, v, dense_order, dense_count, w.osk_budget, w.skip_scale, impl=impl)
+    fused = torch.empty(1, w.n, w.hq + 2 * w.hkv, 128, dtype=torch.bfloat16, device="cuda")
+    fused[:, :, :w.hq] = q.transpose(1, 2)
+    fused[:, :, w.hq:w.hq + w.hkv] = k.transpose(1, 2)
+    fused[:, :, w.hq + w.hkv:] = v.transpose(1, 2)
+    qv = fused[:, :, :w.hq].transpose(1, 2)                   # [B, Hq, N, d] views with token-major strides
+    kv_ = fused[:, :, w.hq:w.hq + w.hkv].transpose(1, 2)
+    vv = fused[:, :, w.hq + w.hkv:].transpose(1, 2)
+    assert not qv.is_contiguous() and qv.stride(2) == (w.hq + 2 * w.hkv) * 128 and qv.stride(1) == 128
+    order, count = alloc_lists(w.hq, nqb)
+    cosa.cosa_kap_select(qv, kv_, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride, impl=impl))
+    assert cosa.cosa_device_status() == 0
+    assert torch.equal(order, dense_order) and torch.equal(count, dense_count)
+    out_tm = torch.zeros(1, w.n, w.hq, 128, dtype=torch.bfloat16, device="cuda")
+    bufs = alloc_outputs(q, nqb)
+    opt = cosa.default_options(skip_scale=w.skip_scale, impl=impl, out_scored=bufs["scored"], out_decisions=bufs["decisions"])
+    cosa.cosa_osk_attention(qv, kv_, vv, order, count, w.osk_budget, out_tm.transpose(1, 2), bufs["lse"], bufs["visited"], opt=opt)
+    assert cosa.cosa_device_status() == 0
+    assert torch.equal(out_tm.transpose(1, 2), dense["out"])
+    for key in ("lse", "visited", "scored", "decisions"):
+        assert torch.equal(bufs[key], dense[key]), key
+    # strides that cannot be mapped are refused, and so are strides together with page pools
+    bad = cosa.default_options()
+    bad.q_strides = (ctypes.c_int64 * 3)(w.hq * w.n * 128, w.n * 128, 100)
+    with pytest.raises(cosa.CosaError) as e:      # (the binding sets strides itself: this goes through the raw call)
+        shape = cosa.make_shape(q, k, True)
+        rc = cosa.library().cosa_kap_select_ex(q.data_ptr(), k.data_ptr(), ctypes.byref(shape), ctypes.c_float(0.25),
+                                               order.data_ptr(), count.data_ptr(), None, ctypes.byref(bad))
+        if rc != 0:
+            raise cosa.CosaError(rc, "cosa_kap_select_ex")
+    assert e.value.status == -1
 
 
 def test_kv_head_shards_concatenate_to_the_unsharded_result(small):
