@@ -69,7 +69,8 @@ __device__ __forceinline__ void screen_timeout(ScreenCtl* c, int32_t* status) {
   atomicMin(status, (int32_t)COSA_ERR_DEVICE_TIMEOUT);
 }
 
-template <int R>
+// kStrict: every multi-lane wait answers per warp (see mbar_wait_warp)
+template <int R, bool kStrict>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                   KapScreenParams p, int32_t* status) {
@@ -142,6 +143,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
   const uint32_t tmem = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort_flag;
   const long long budget = p.wait_budget;
+  constexpr bool strict = kStrict;
 
   if (warp == 0) {
     int t_issued = 0;   // (lane 0) key tiles requested so far
@@ -246,7 +248,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     // each half tile; the swizzle permutes 16-byte chunks inside a row, which a sum of squares does not notice; the
     // chunk order is rotated by the lane so that the rows of a warp hit different banks)
     float q2 = 0.f;
-    bool alive = mbar_wait_warp(smem_u32(&ctl->a_full), 0, abort_flag, budget);
+    bool alive = mbar_wait_warp(smem_u32(&ctl->a_full), 0, abort_flag, budget, strict);
     if (!alive && !*abort_flag) screen_timeout(ctl, status);
     if (alive) {
       const unsigned char* arow = smem + (size_t)rt * kTileBytes + (size_t)(row % 128) * 128;
@@ -267,7 +269,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
     }
     for (int t = 0; t < n_tiles && alive; ++t) {
       const int sb = t % kSteps, st = t % kStages;
-      alive = mbar_wait_warp(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag, budget);   // this tile's MMAs finished
+      alive = mbar_wait_warp(smem_u32(&ctl->k_empty[st]), (t / kStages) & 1, abort_flag, budget, strict);   // this tile's MMAs finished
       if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
       tc_fence_after();
       uint32_t v[kPartCols / 32][32];
@@ -313,7 +315,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       ctl->xt[part][0][row] = top1; ctl->xt[part][1][row] = top2; ctl->xt[part][2][row] = top3;
       ctl->xj[part][0][row] = jstar; ctl->xj[part][1][row] = jstar2;
       mbar_arrive(smem_u32(&ctl->x_bar));
-      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 0, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 0, abort_flag, budget, strict);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
     }
     if (alive) {
@@ -352,7 +354,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
       // every row's M* in shared memory and every parked maximum visible to the whole CTA
       __threadfence_block();
       mbar_arrive(smem_u32(&ctl->x_bar));
-      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 1, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->x_bar), 1, abort_flag, budget, strict);
       if (!alive && !*abort_flag) screen_timeout(ctl, status);
     }
     if (alive) {
@@ -408,7 +410,7 @@ kap_screen_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_consta
             fetch(c + kStages - 1);
           }
         }
-        alive = mbar_wait_warp(smem_u32(&ctl->m_full[st]), (c / kStages) & 1, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->m_full[st]), (c / kStages) & 1, abort_flag, budget, strict);
         if (!alive) { if (!*abort_flag) screen_timeout(ctl, status); break; }
         const int tiles_here = min(kTilesPerChunk, n_tiles - c * kTilesPerChunk);
         const float* stage = reinterpret_cast<const float*>(smem + (size_t)kTileBytes * (kRowTiles + st));
@@ -516,10 +518,13 @@ cudaError_t launch_kap_screen(const KapScreenParams& p_in, cudaStream_t st) {
   if (!status) return cudaErrorInvalidSymbol;
   const int grid = kap_screen_grid(p.batch, p.hq, p.hkv, p.nqb, p.stride);
   cudaError_t e;
-#define COSA_LAUNCH_SCREEN(RR)                                                                                    \
-  e = cudaFuncSetAttribute(kap_screen_kernel<RR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScreenSmem); \
-  if (e != cudaSuccess) return e;                                                                                 \
-  kap_screen_kernel<RR><<<grid, kThreads, kScreenSmem, st>>>(qm, km, p, status);
+#define COSA_LAUNCH_SCREEN(RR)                                                                                              \
+  {                                                                                                                         \
+    auto kernel = wait_budget_is_short(p.wait_budget) ? kap_screen_kernel<RR, true> : kap_screen_kernel<RR, false>;         \
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScreenSmem);                        \
+    if (e != cudaSuccess) return e;                                                                                         \
+    kernel<<<grid, kThreads, kScreenSmem, st>>>(qm, km, p, status);                                                         \
+  }
   if (R == 8) { COSA_LAUNCH_SCREEN(8) }
   else if (R == 16) { COSA_LAUNCH_SCREEN(16) }
   else if (R == 32) { COSA_LAUNCH_SCREEN(32) }

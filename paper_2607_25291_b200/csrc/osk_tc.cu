@@ -8,9 +8,11 @@
 //   warp 1       QK issuer: S = Q K_j^T into one of two TMEM buffers
 //   warp 3       PV issuer: O += P V_j.  Two issuing threads, because a single thread's
 //                instruction stream (descriptors, barrier tests, commits) is what limits how fast
-//                MMAs reach the tensor pipe.  Q K^T takes both operands from shared memory, P V its A
-//                operand from tensor memory, where P has two buffers: the probabilities of the next
-//                computed block are stored while the product of the previous one still runs.
+//                MMAs reach the tensor pipe.  Both products take their A operand (Q, resp. P) from
+//                tensor memory.  (Q read from shared memory instead, which frees the columns for a second
+//                P buffer so that the next block's probabilities are stored while the previous product
+//                still runs, was built and measured 1 % slower at 128K: the product chain is not what
+//                paces the walk.)
 //   warp 2       controller (see below)
 //   warps 4..7   softmax group A: list positions 0, 2, 4, ...   (one thread per query row)
 //   warps 8..11  softmax group B: list positions 1, 3, 5, ...
@@ -24,8 +26,8 @@
 //                the cap on computed blocks, the V tile load of computed blocks, and the
 //                decisions the other warps follow
 // Q, K, V tiles land in shared memory through TMA with the 128-byte swizzle the MMA descriptors
-// expect; the Q tile is fetched by TMA as well and stays in shared memory.
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
+// expect; the Q tile is fetched by TMA as well and copied from shared memory into TMEM by the first group.
+// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P [384,448) Q [448,512).
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds
 // down without writing results.
 #include <math.h>
@@ -52,10 +54,10 @@ constexpr int kSpec = 2;   // K tiles fetched and products issued ahead of the b
 constexpr uint32_t kDecComputed = 1, kDecEnd = 2;  // bits 8.. : computed blocks before this position
 
 struct __align__(8) Control {
-  unsigned long long q_stage, k_full[kKStages], v_full[kVStages];   // q_stage: the Q tile has landed
+  unsigned long long q_stage, q_full, k_full[kKStages], v_full[kVStages];   // Q tile landed / Q copied into TMEM
   unsigned long long k_empty[kKStages];  // QK^T of that stage finished: the stage is free AND its S tile is ready
   unsigned long long s_empty[2];
-  unsigned long long p_full[2];   // P of computed block n is in buffer n & 1
+  unsigned long long p_full[2];   // P of computed block n is stored (barrier n & 1; the one buffer is free again after product n)
   unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1] (P free, O updated, V stage n & 1 free); two
                                   // barriers because a waiter may run two products ahead of the tensor pipe, which one
                                   // barrier's single parity bit cannot tell apart
@@ -104,7 +106,8 @@ __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensor
 
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
 // list-driven kernel carries none of the walk's state
-template <bool kMask>
+// kStrict: every multi-lane wait answers per warp (see mbar_wait_warp)
+template <bool kMask, bool kStrict>
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
@@ -161,7 +164,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   if (threadIdx.x == 0) {
     // barriers first, then the Q tile at once: its address needs nothing from global memory, while the list
     // entries, the count and the status word requested above are still on their way (2 k cycles at the start of a CTA)
-    mbar_init(smem_u32(&ctl->q_stage), 1);
+    mbar_init(smem_u32(&ctl->q_stage), 1); mbar_init(smem_u32(&ctl->q_full), kBlock);
     for (int s = 0; s < kKStages; ++s) { mbar_init(smem_u32(&ctl->k_full[s]), 1); mbar_init(smem_u32(&ctl->k_empty[s]), 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(smem_u32(&ctl->v_full[s]), 1);
@@ -212,9 +215,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
-  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 448u};
+  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 384u};   // one buffer
+  const uint32_t tmem_q = tmem + 448u;
   volatile int* abort_flag = &ctl->abort_flag;
   const long long budget = p.wait_budget;
+  constexpr bool strict = kStrict;
   const float kLog2e = 1.4426950408889634f;
   const float scale2 = p.scale * kLog2e;    // work in base 2: exp(x) = exp2(x * log2 e)
   const float theta2 = (p.use_threshold ? item_theta(p.pg, b, p.theta, p.skip_scale, nqb_b) : 0.f) * kLog2e;
@@ -257,10 +262,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------------ QK issuer
     if (lane == 0) {
-      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] and K_j [N x K], both K-major in shared memory
-      bool alive = mbar_wait(smem_u32(&ctl->q_stage), 0, abort_flag, budget);
+      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);   // Q [M x K] from TMEM, K_j [N x K] K-major
+      bool alive = mbar_wait(smem_u32(&ctl->q_full), 0, abort_flag, budget);
       if (!alive && !*abort_flag) report_timeout(ctl, status);
-      const uint64_t qdesc = smem_desc_sw128(q_sm, 16, 1024);
       const uint64_t kdesc0 = smem_desc_sw128(k_sm, 16, 1024);
       int last_issued = -1;
       int n_certain = 0;        // a copy of n_needed, which only grows: positions below it are certain to be scored
@@ -308,8 +312,8 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         }
         tc_fence_after();
         // 16 elements of d per MMA: 32 bytes along a 128-byte row, the second 64 elements in the other half tile
-        mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
-            tmem_s[sb], qdesc, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk);
+        mma_ts_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+            tmem_s[sb], tmem_q, kdesc0 + (uint64_t)(st * (kTileBytes / 16)), idesc_qk, false);
         mma_commit(smem_u32(&ctl->k_empty[st]));
         last_issued = kk;
       }
@@ -359,7 +363,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     for (int kk = 0; kk < cnt && alive; ++kk) {
       const int par = kk & 1;
       const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
-      alive = mbar_wait_warp(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget, strict);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
       // The statistic is <= 0, so among bit patterns the smallest unsigned word is the largest value.
@@ -425,6 +429,23 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     float m_ref = -INFINITY, l = 0.f;         // this group's partial row sum and the maximum it refers to
     bool alive = true;
     uint32_t s[kBlock];                       // this row's raw logits, then probabilities
+    if (grp == 0) {
+      // Q row: shared memory (TMA box layout, 16-byte chunks swizzled by row) -> TMEM as the A operand of
+      // QK^T: lane = row, two consecutive d per 32-bit column
+      alive = mbar_wait_warp(smem_u32(&ctl->q_stage), 0, abort_flag, budget, strict);
+      if (!alive && !*abort_flag) report_timeout(ctl, status);
+      const unsigned char* qs = smem + (size_t)kTileBytes * (kKStages + kVStages);
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 wv = *reinterpret_cast<const uint4*>(qs + (c >> 3) * kHalfBytes + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+        s[4 * c] = wv.x; s[4 * c + 1] = wv.y; s[4 * c + 2] = wv.z; s[4 * c + 3] = wv.w;
+      }
+      tmem_st32(tmem_q + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_st32(tmem_q + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&ctl->q_full));
+    }
     // only "is this the diagonal block" matters to a group; an ascending mask walk meets it last, if at all.  The list
     // entry of a position is requested one turn ahead: its latency (some 400 cycles) would otherwise sit between a
     // decision and the group's next S tile
@@ -445,9 +466,10 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
             if (*abort_flag || clock64() - t0 > budget) { alive = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           }
         }
-        // one answer per warp: the loads below are executed by all of its lanes or by none
-        ended = __any_sync(0xffffffffu, ended) != 0;
-        alive = __all_sync(0xffffffffu, alive) != 0;
+        if (strict) {   // one answer per warp: the loads below are executed by all of its lanes or by none
+          ended = __any_sync(0xffffffffu, ended) != 0;
+          alive = __all_sync(0xffffffffu, alive) != 0;
+        }
         if (ended || !alive) break;
       }
       tc_fence_after();
@@ -472,15 +494,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
       // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
       //      walk gets here at all (n_needed only grows: an old value merely costs this wait)
-      if (kk >= __shfl_sync(0xffffffffu, ctl->n_needed, 0)) {   // (one reading per warp: the counter grows while it is read)
-        alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
+      if (kk >= (strict ? __shfl_sync(0xffffffffu, ctl->n_needed, 0) : ctl->n_needed)) {   // (one reading per warp when lanes may disagree: the counter grows while it is read)
+        alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget, strict);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         if (ctl->dec[(kk - 1) % kDecRing] & kDecEnd) break;
       }
       // ---- running maximum before this position comes from the other group
       float m_in = -INFINITY;
       if (kk > 0) {
-        alive = mbar_wait_warp(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->m_ready[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget, strict);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         m_in = ctl->mrow[grp ^ 1][r];
       }
@@ -491,7 +513,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       ctl->mrow[grp][r] = m_new;
       mbar_arrive(smem_u32(&ctl->m_ready[grp]));
       // ---- the controller's decision
-      alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget);
+      alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget, strict);
       if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
       const uint32_t d = ctl->dec[kk % kDecRing];
       const bool last = (d & kDecEnd) != 0;
@@ -523,27 +545,23 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       }
 #pragma unroll
       for (int c = 0; c < 64; ++c) s[c] = pack_bf16(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1]));
-      // ---- P has two buffers: the product before last must have finished with this one; O is rescaled only if a row
-      //      maximum moved, and only then must the previous product have finished as well
-      if (n_before > 1) {
-        alive = mbar_wait_warp(smem_u32(&ctl->p_empty[n_before & 1]), ((n_before - 2) >> 1) & 1, abort_flag, budget);
-        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-      }
-      if (n_before > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O
-        alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag, budget);
+      // ---- the previous PV product must have finished: P is free and O may be rescaled
+      if (n_before > 0) {
+        alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_before - 1) & 1]), ((n_before - 1) >> 1) & 1, abort_flag, budget, strict);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         tc_fence_after();
-        uint32_t o[32];
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // O = diag(alpha) O, only if a row maximum moved
+          uint32_t o[32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          tmem_ld32(tmem_o + lane_addr + c * 32, o);
-          tmem_wait_ld();
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_o + lane_addr + c * 32, o);
+            tmem_wait_ld();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-          tmem_st32(tmem_o + lane_addr + c * 32, o);
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+            tmem_st32(tmem_o + lane_addr + c * 32, o);
+          }
         }
       }
-      tc_fence_after();
       tmem_st32(tmem_p[n_before & 1] + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
       tmem_st32(tmem_p[n_before & 1] + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_st();
@@ -560,16 +578,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       mbar_arrive(smem_u32(&ctl->fin_bar));
     } else {
       if (alive) {
-        alive = mbar_wait_warp(smem_u32(&ctl->fin_bar), 0, abort_flag, budget);
+        alive = mbar_wait_warp(smem_u32(&ctl->fin_bar), 0, abort_flag, budget, strict);
         if (!alive && !*abort_flag) report_timeout(ctl, status);
       }
-      if (__all_sync(0xffffffffu, alive && !*abort_flag)) {
+      if (strict ? (__all_sync(0xffffffffu, alive && !*abort_flag) != 0) : (alive && !*abort_flag)) {
         const float mb = ctl->fin_m[r];
         const float mf = fmaxf(m_ref, mb);         // the running maximum is monotone: this is its final value
         const float lt = l * ex2_approx(m_ref - mf) + ctl->fin_l[r] * ex2_approx(mb - mf);
         const int n_comp = ctl->final_computed;
         if (n_comp > 0) {
-          alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag, budget);
+          alive = mbar_wait_warp(smem_u32(&ctl->p_empty[(n_comp - 1) & 1]), ((n_comp - 1) >> 1) & 1, abort_flag, budget, strict);
           if (!alive && !*abort_flag) report_timeout(ctl, status);
         }
         if (alive) {
@@ -615,7 +633,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   }
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (threadIdx.x == 0 && *abort_flag) {
     // copies that nobody has waited for when the walk was given up: the Q tile, a V tile the PV issuer never took
     (void)mbar_wait_noabort(smem_u32(&ctl->q_stage), 0);
     for (int n = ctl->v_taken; n < ctl->v_req; ++n) (void)mbar_wait_noabort(smem_u32(&ctl->v_full[n % kVStages]), (n / kVStages) & 1);
@@ -635,7 +653,9 @@ cudaError_t launch_osk_tc(const OskParams& p_in, cudaStream_t st) {
       !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n) || !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n) ||
       !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
-  auto kernel = p.mask ? osk_tc_kernel<true> : osk_tc_kernel<false>;
+  const bool strict = wait_budget_is_short(p.wait_budget);
+  auto kernel = p.mask ? (strict ? osk_tc_kernel<true, true> : osk_tc_kernel<true, false>)
+                       : (strict ? osk_tc_kernel<false, true> : osk_tc_kernel<false, false>);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
   if (p.decisions) {

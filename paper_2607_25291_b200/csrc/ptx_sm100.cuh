@@ -74,11 +74,19 @@ __device__ __forceinline__ bool mbar_wait_noabort(uint32_t bar, uint32_t parity,
     if (clock64() - t0 > budget) return false;
   }
 }
-// For code all 32 lanes of a warp run together: the same bounded wait, with one answer for the whole warp (lanes that
-// poll on their own can see the budget run out at different moments, and what follows -- tcgen05.ld/st, __syncwarp --
-// must be executed by all lanes or by none)
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
-  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, budget)) != 0;
+// For code all 32 lanes of a warp run together: the same bounded wait, with one answer for the whole warp when
+// `unanimous` is set.  Lanes poll on their own (the cheapest way to wait), so they can see the budget run out at
+// different moments, and what follows -- tcgen05.ld/st, __syncwarp -- must be executed by all lanes or by none.  With
+// the regular budget (about a second) the lanes of a warp, which start their waits within a few cycles of each other,
+// cannot disagree unless the barrier completes in the very cycles in which a second of waiting ends; the vote costs 2 %
+// of the OSK kernel (and a run-time switch more: the kernel is sensitive to its code size), so the kernels exist in
+// two instantiations and the one with the votes is launched when the caller has set a short budget
+// (wait_budget_is_short), where lanes disagreeing is the expected case.
+__host__ __device__ inline bool wait_budget_is_short(long long budget) { return budget < (1LL << 24); }
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget,
+                                               bool unanimous) {
+  const bool ok = mbar_wait(bar, parity, abort_flag, budget);
+  return unanimous ? (__all_sync(0xffffffffu, ok) != 0) : ok;
 }
 // named barrier among `nthreads` threads of the CTA (ids 1..15; 0 is __syncthreads)
 __device__ __forceinline__ void bar_sync(int id, int nthreads) {
