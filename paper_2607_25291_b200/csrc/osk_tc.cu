@@ -32,6 +32,8 @@
 // down without writing results.
 #include <math.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx_sm100.cuh"
 #include "tile_maps.cuh"
@@ -107,7 +109,10 @@ __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensor
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
 // list-driven kernel carries none of the walk's state
 // kStrict: every multi-lane wait answers per warp (see mbar_wait_warp)
-template <bool kMask, bool kStrict>
+// kStage2: false = Stage 2 off (tightened_budget >= 1: Eq. 4, attention over the listed blocks; the library's dense
+//          path).  Every listed block is computed, so nothing waits for a decision: the groups go from the row maxima
+//          straight to the exponentials, and the controller only fetches V tiles, as far ahead as its two stages allow.
+template <bool kMask, bool kStrict, bool kStage2>
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
@@ -176,9 +181,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     mbar_init(smem_u32(&ctl->out_bar), kBlock);
     mbar_init(smem_u32(&ctl->fin_bar), kBlock);
     ctl->n_dec = 0;
-    ctl->end_kk = -1;
+    ctl->end_kk = kStage2 ? -1 : cnt - 1;          // Stage 2 off: the walk ends with the list
     ctl->k_loaded = -1;
-    ctl->final_computed = 0;
+    ctl->final_computed = kStage2 ? 0 : cnt;
     ctl->v_req = 0; ctl->v_taken = 0;
     ctl->abort_flag = 0;
     mbar_fence_init();
@@ -242,7 +247,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           if (*abort_flag || clock64() - t0 > budget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           __nanosleep(32);
         }
-        if (!ok || ctl->end_kk >= 0) break;
+        if (!ok || (kStage2 && ctl->end_kk >= 0)) break;
         const int st = kk % kKStages;
         if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag, budget)) {
           if (!*abort_flag) report_timeout(ctl, status);
@@ -360,7 +365,26 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
-    for (int kk = 0; kk < cnt && alive; ++kk) {
+    if (!kStage2) {
+      // every block is computed: V_j as soon as the product before last has released the stage
+      if (lane == 0) {
+        for (int kk = 0; kk < cnt && alive; ++kk) {
+          const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
+          const int vs = kk % kVStages;
+          alive = mbar_wait(smem_u32(&ctl->p_empty[vs]), ((kk >> 1) & 1) ^ 1, abort_flag, budget);   // PV kk-2 read this stage
+          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+          const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
+          mbar_expect_tx(bar, kTileBytes);
+          load_kv_block(p, &v_map, dst, b, g, j, bar);
+          ctl->v_req = kk + 1;
+        }
+        if (alive && p.decisions)
+          for (int wd = 0; wd * 32 < cnt; ++wd) p.decisions[row * dec_words + wd] = cnt - wd * 32 >= 32 ? 0xffffffffu : ((1u << (cnt - wd * 32)) - 1u);
+      }
+      computed = cnt; scored = cnt;
+      alive = __shfl_sync(0xffffffffu, alive ? 1 : 0, 0) != 0;
+    }
+    for (int kk = 0; kStage2 && kk < cnt && alive; ++kk) {
       const int par = kk & 1;
       const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
       alive = mbar_wait_warp(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget, strict);
@@ -494,7 +518,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const float m_loc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale2;   // scale > 0 commutes with max
       // ---- a product issued ahead of the certain blocks: the decision on the position before tells whether the
       //      walk gets here at all (n_needed only grows: an old value merely costs this wait)
-      if (kk >= (strict ? __shfl_sync(0xffffffffu, ctl->n_needed, 0) : ctl->n_needed)) {   // (one reading per warp when lanes may disagree: the counter grows while it is read)
+      if (kStage2 && kk >= (strict ? __shfl_sync(0xffffffffu, ctl->n_needed, 0) : ctl->n_needed)) {   // (one reading per warp when lanes may disagree: the counter grows while it is read)
         alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp ^ 1]), ((kk - 1) >> 1) & 1, abort_flag, budget, strict);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         if (ctl->dec[(kk - 1) % kDecRing] & kDecEnd) break;
@@ -512,10 +536,13 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       if (lane == 0) ctl->gapw[grp][sub] = gbits;
       ctl->mrow[grp][r] = m_new;
       mbar_arrive(smem_u32(&ctl->m_ready[grp]));
-      // ---- the controller's decision
-      alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget, strict);
-      if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-      const uint32_t d = ctl->dec[kk % kDecRing];
+      // ---- the controller's decision (Stage 2 off: computed, as the kk-th computed block, the last one ends the walk)
+      uint32_t d = kDecComputed | (kk == cnt - 1 ? kDecEnd : 0u) | ((uint32_t)kk << 8);
+      if (kStage2) {
+        alive = mbar_wait_warp(smem_u32(&ctl->dec_bar[grp]), (kk >> 1) & 1, abort_flag, budget, strict);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        d = ctl->dec[kk % kDecRing];
+      }
       const bool last = (d & kDecEnd) != 0;
       if (!(d & kDecComputed)) {                  // skipped: nothing is added to l or O
         if (last) break;
@@ -654,8 +681,12 @@ cudaError_t launch_osk_tc(const OskParams& p_in, cudaStream_t st) {
       !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
   const bool strict = wait_budget_is_short(p.wait_budget);
-  auto kernel = p.mask ? (strict ? osk_tc_kernel<true, true> : osk_tc_kernel<true, false>)
-                       : (strict ? osk_tc_kernel<false, true> : osk_tc_kernel<false, false>);
+  auto pick = [&](auto mask_c, auto strict_c) {
+    return p.stage2 ? osk_tc_kernel<decltype(mask_c)::value, decltype(strict_c)::value, true>
+                    : osk_tc_kernel<decltype(mask_c)::value, decltype(strict_c)::value, false>;
+  };
+  using T = std::true_type; using F = std::false_type;
+  auto kernel = p.mask ? (strict ? pick(T{}, T{}) : pick(T{}, F{})) : (strict ? pick(F{}, T{}) : pick(F{}, F{}));
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
   if (p.decisions) {
