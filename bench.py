@@ -51,6 +51,8 @@ def parse():
     ap.add_argument("--shard", default="layer", choices=["layer", "kv_head"],
                     help="with --gpus N: 'layer' gives every rank a layer of its own (weak scaling, the default); 'kv_head' splits "
                          "ONE layer by KV-head group, rank r running KAP + OSK on its heads only (strong scaling; N <= KV heads)")
+    ap.add_argument("--pages-in-place", action="store_true",
+                    help="with --page-size below 128: OSK reads the pages in place (cosa_options.kv_pages_in_place), no staging copy")
     ap.add_argument("--osk-impl", type=int, default=0, choices=[0, 4],
                     help="4: the OSK kernel that walks two work items per CTA (cosa_options.impl = 4); not the headline config")
     ap.add_argument("--top-p", type=float, default=0.0,
@@ -254,6 +256,7 @@ def main():
         page_table = torch.from_numpy(table).to(dev)[None].contiguous()
         opt.kv_page_table = page_table.data_ptr()
         opt.kv_page_size = args.page_size
+        opt.kv_pages_in_place = 1 if args.pages_in_place else 0
         opt.kv_num_pages = kpool.shape[0]
 
     def step():

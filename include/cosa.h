@@ -120,6 +120,12 @@ typedef struct {
                               row): cosa_workspace_bytes() then includes B*Hkv*N*d*2 bytes for K, and
                               the same again for V in cosa_osk_attention                             */
   int32_t kv_num_pages;    /* pages in the pools                                                     */
+  int32_t kv_pages_in_place; /* cosa_osk_attention only, pools with pages smaller than a key block.  0 (default): the
+                              staging copy described above.  1: no copy and no scratch (cosa_workspace_bytes(1, ...)
+                              is 0): every tile is assembled from the pages themselves, one pair of boxes per page,
+                              issued side by side by the lanes of a warp after their table look-ups.  Same results;
+                              slower the smaller the pages are, since the copy engine works box by box (128K tokens:
+                              8.7 ms dense, 8.9 staged, 9.5 in place at 64-token pages, 11.7 at 16)           */
   const int32_t* seq_lens; /* Non-NULL: device array [B]; batch item b holds seq_lens[b] tokens, a multiple
                               of 128 in [128, N] (a batch of prompts of different lengths, padded to N;
                               Sec. C.1 runs inside a paged serving engine, where this is the rule).  Rows

@@ -43,7 +43,7 @@ class CosaOptions(Structure):
                 ("order_stride", c_int32), ("out_scored", c_void_p), ("out_decisions", c_void_p),
                 ("kap_scores", c_void_p), ("kap_flags", c_void_p), ("workspace", c_void_p),
                 ("workspace_bytes", c_size_t), ("impl", c_int32), ("top_p", c_float), ("logical_mask", c_void_p), ("kv_page_table", c_void_p),
-                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("seq_lens", c_void_p), ("q_strides", ctypes.c_int64 * 3), ("kv_strides", ctypes.c_int64 * 3),
+                ("kv_page_size", c_int32), ("kv_num_pages", c_int32), ("kv_pages_in_place", c_int32), ("seq_lens", c_void_p), ("q_strides", ctypes.c_int64 * 3), ("kv_strides", ctypes.c_int64 * 3),
                 ("out_strides", ctypes.c_int64 * 3), ("wait_cycles", ctypes.c_int64)]
 
 

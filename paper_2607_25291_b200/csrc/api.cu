@@ -147,9 +147,13 @@ static KapScratch kap_scratch_layout(const cosa_shape* s, const cosa_options& o)
   return L;
 }
 static size_t kap_scratch_bytes(const cosa_shape* s, const cosa_options& o) { return kap_scratch_layout(s, o).total; }
-// OSK fetches a key block as one pair of TMA boxes per page: pools whose pages are smaller than a block are copied
-// into dense staging tensors (K, then V) first
-static bool osk_gathers(const cosa_options& o) { return o.kv_page_table && o.impl != 1 && o.kv_page_size < kBlock; }
+// Pools whose pages are smaller than a block are copied into dense staging tensors (K, then V) first by the kernel that
+// fetches a key block as one pair of TMA boxes
+// (with kv_pages_in_place the default kernel assembles a tile from one pair of boxes per page instead, issued by the lanes
+// of a warp side by side, and needs no scratch)
+static bool osk_gathers(const cosa_options& o) {
+  return o.kv_page_table && o.impl != 1 && o.kv_page_size < kBlock && (o.impl == 4 || !o.kv_pages_in_place);
+}
 static size_t osk_scratch_bytes(const cosa_shape* s, const cosa_options& o) {
   return osk_gathers(o) ? 2 * align_up((size_t)s->batch * s->hkv * s->n * s->d * 2, 256) : 0;
 }

@@ -106,13 +106,36 @@ __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensor
   tma_load_tile(dst + kHalfBytes, map, 64, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
 }
 
+// The part of key block j that page `part` of the block holds (pages smaller than a block): one pair of boxes of
+// page_size rows, placed where the rows belong in the tile.  The caller has armed the barrier for the whole tile.
+__device__ __forceinline__ void load_kv_block_part(const OskParams& p, const CUtensorMap* map, uint32_t dst, int b, int g, int j,
+                                                   int part, uint32_t bar) {
+  const int ps = p.pg.page_size;
+  const KvCoord c = kv_coord(p.pg, b, g, j * kBlock + part * ps);
+  tma_load_tile(dst + part * ps * 128, map, 0, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+  tma_load_tile(dst + kHalfBytes + part * ps * 128, map, 64, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+}
+// the same with the page already looked up (the look-up is a global load: done ahead of a wait, it costs nothing)
+__device__ __forceinline__ void load_kv_block_part_at(const OskParams& p, const CUtensorMap* map, uint32_t dst, const KvCoord& c,
+                                                      int part, uint32_t bar) {
+  const int ps = p.pg.page_size;
+  tma_load_tile(dst + part * ps * 128, map, 0, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+  tma_load_tile(dst + kHalfBytes + part * ps * 128, map, 64, c.row, c.head, c.outer, p.ko.row, p.ko.head, p.ko.outer, bar);
+}
+
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk); a compile-time switch so that the
 // list-driven kernel carries none of the walk's state
 // kStrict: every multi-lane wait answers per warp (see mbar_wait_warp)
 // kStage2: false = Stage 2 off (tightened_budget >= 1: Eq. 4, attention over the listed blocks; the library's dense
 //          path).  Every listed block is computed, so nothing waits for a decision: the groups go from the row maxima
 //          straight to the exponentials, and the controller only fetches V tiles, as far ahead as its two stages allow.
-template <bool kMask, bool kStrict, bool kStage2>
+// kSmallPages: K and V are page pools whose pages are smaller than a key block (Sec. C.1: a logical block resolved
+//          through several physical pages).  A tile is then assembled from one pair of boxes per page, which the lanes
+//          of the loader warp (K) and of the controller warp (V) issue side by side, each after its own table look-up;
+//          one thread issuing them all in turn made the walk 1.8 times slower at 16-token pages.  Boxes land on
+//          1024-byte boundaries of the tile (pages of at least 8 tokens), where the 128-byte swizzle, a function of
+//          the shared-memory address, gives the layout of the one-piece tile.
+template <bool kMask, bool kStrict, bool kStage2, bool kSmallPages>
 __global__ void __launch_bounds__(kThreads, 1)
 osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
               const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
@@ -196,7 +219,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     ctl->n_needed = min(cnt, cap);
     if (poisoned_early == 0 && cnt > 0) {
       // the first K tiles, before the rest of the CTA has even finished setting up
-      const int n_first = min(min(cnt, cap), kKStages);
+      const int n_first = kSmallPages ? 0 : min(min(cnt, cap), kKStages);   // (small pages: left to the loader warp's lanes)
       for (int kk = 0; kk < n_first; ++kk) {
         const int j = min(max(first_ids[kk], 0), p.nqb - 1);
         const uint32_t dst = k_sm + kk * kTileBytes, bar = smem_u32(&ctl->k_full[kk]);
@@ -237,9 +260,14 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   if (cnt == 0) {
   } else if (warp == 0) {
     // ------------------------------------------------------------------ K loader
-    if (lane == 0) {
-      int last_issued = min(min(cnt, cap), kKStages) - 1;
-      for (int kk = last_issued + 1; kk < cnt; ++kk) {   // the first tiles were requested in the prologue
+    // lane 0 decides when the next tile may be requested; with small pages every lane then fetches one page's part
+    const int ppb = kSmallPages ? kBlock / p.pg.page_size : 1;       // pages per key block
+    int last_issued = kSmallPages ? -1 : min(min(cnt, cap), kKStages) - 1;   // (without small pages the first tiles were requested in the prologue)
+    for (int kk = last_issued + 1; kk < cnt; ++kk) {
+      int go = 1, j = 0;
+      const int st = kk % kKStages;
+      const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
+      if (lane == 0) {
         const long long t0 = clock64();
         bool ok = true;
         while (kk >= ctl->n_needed + kSpec) {  // at most kSpec tiles beyond the blocks that are certain to be scored
@@ -247,18 +275,27 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           if (*abort_flag || clock64() - t0 > budget) { ok = false; if (!*abort_flag) report_timeout(ctl, status); break; }
           __nanosleep(32);
         }
-        if (!ok || (kStage2 && ctl->end_kk >= 0)) break;
-        const int st = kk % kKStages;
-        if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag, budget)) {
+        if (!ok || (kStage2 && ctl->end_kk >= 0)) {
+          go = 0;
+        } else if (!mbar_wait(smem_u32(&ctl->k_empty[st]), ((kk / kKStages) & 1) ^ 1, abort_flag, budget)) {
           if (!*abort_flag) report_timeout(ctl, status);
-          break;
+          go = 0;
+        } else {
+          j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
+          mbar_expect_tx(bar, kTileBytes);
+          if (!kSmallPages) load_kv_block(p, &k_map, dst, b, g, j, bar);
         }
-        const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
-        const uint32_t dst = k_sm + st * kTileBytes, bar = smem_u32(&ctl->k_full[st]);
-        mbar_expect_tx(bar, kTileBytes);
-        load_kv_block(p, &k_map, dst, b, g, j, bar);
-        last_issued = kk;
       }
+      if (kSmallPages) {
+        go = __shfl_sync(0xffffffffu, go, 0);
+        j = __shfl_sync(0xffffffffu, j, 0);
+        if (go && lane < ppb) load_kv_block_part(p, &k_map, dst, b, g, j, lane, bar);
+        __syncwarp();
+      }
+      if (!go) break;
+      last_issued = kk;
+    }
+    if (lane == 0) {
       ctl->k_loaded = last_issued + 1;       // the QK issuer must not wait for a tile beyond these
       // tiles fetched ahead may never be multiplied: their copies must have landed before the CTA retires
       for (int kk = max(0, last_issued - (kKStages - 1)); kk <= last_issued; ++kk)
@@ -365,28 +402,39 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
+    const int ppb = kSmallPages ? kBlock / p.pg.page_size : 1;       // pages per key block
     if (!kStage2) {
-      // every block is computed: V_j as soon as the product before last has released the stage
-      if (lane == 0) {
-        for (int kk = 0; kk < cnt && alive; ++kk) {
-          const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
-          const int vs = kk % kVStages;
-          alive = mbar_wait(smem_u32(&ctl->p_empty[vs]), ((kk >> 1) & 1) ^ 1, abort_flag, budget);   // PV kk-2 read this stage
-          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-          const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
-          mbar_expect_tx(bar, kTileBytes);
-          load_kv_block(p, &v_map, dst, b, g, j, bar);
-          ctl->v_req = kk + 1;
+      // every block is computed: V_j as soon as the product before last has released the stage (lane 0 waits and arms
+      // the barrier; with small pages every lane then fetches one page's part)
+      for (int kk = 0; kk < cnt && alive; ++kk) {
+        const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);
+        const int vs = kk % kVStages;
+        const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
+        int ok = 1;
+        if (lane == 0) {
+          ok = mbar_wait(smem_u32(&ctl->p_empty[vs]), ((kk >> 1) & 1) ^ 1, abort_flag, budget) ? 1 : 0;   // PV kk-2 read this stage
+          if (!ok) {
+            if (!*abort_flag) report_timeout(ctl, status);
+          } else {
+            mbar_expect_tx(bar, kTileBytes);
+            if (!kSmallPages) load_kv_block(p, &v_map, dst, b, g, j, bar);
+            ctl->v_req = kk + 1;
+          }
         }
-        if (alive && p.decisions)
-          for (int wd = 0; wd * 32 < cnt; ++wd) p.decisions[row * dec_words + wd] = cnt - wd * 32 >= 32 ? 0xffffffffu : ((1u << (cnt - wd * 32)) - 1u);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (kSmallPages && ok && lane < ppb) load_kv_block_part(p, &v_map, dst, b, g, j, lane, bar);
+        __syncwarp();
+        alive = ok != 0;
       }
+      if (lane == 0 && alive && p.decisions)
+        for (int wd = 0; wd * 32 < cnt; ++wd) p.decisions[row * dec_words + wd] = cnt - wd * 32 >= 32 ? 0xffffffffu : ((1u << (cnt - wd * 32)) - 1u);
       computed = cnt; scored = cnt;
-      alive = __shfl_sync(0xffffffffu, alive ? 1 : 0, 0) != 0;
     }
     for (int kk = 0; kStage2 && kk < cnt && alive; ++kk) {
       const int par = kk & 1;
       const int j = kMask ? walk.at(kk) : min(max(list[kk], 0), p.nqb - 1);     // issued before the wait: latency hidden
+      KvCoord vc = KvCoord{0, 0, 0};
+      if (kSmallPages && lane < ppb) vc = kv_coord(p.pg, b, g, j * kBlock + lane * p.pg.page_size);   // ... and so is this lane's page
       alive = mbar_wait_warp(smem_u32(&ctl->m_ready[par]), (kk >> 1) & 1, abort_flag, budget, strict);
       if (!alive) { if (!*abort_flag && lane == 0) report_timeout(ctl, status); break; }
       // Eq. (5): skip iff max over the 128 rows of (m_loc - m) < ln(Delta/N), m including this block.
@@ -398,6 +446,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       const int n_before = computed;
       if (compute) ++computed; else n_needed = min(cnt, n_needed + 1);
       const bool last = (computed == cap) || (kk == cnt - 1);
+      int v_go = 0;
       if (lane == 0) {
         ctl->n_needed = n_needed;
         ctl->dec[kk % kDecRing] = (compute ? kDecComputed : 0u) | (last ? kDecEnd : 0u) | ((uint32_t)n_before << 8);
@@ -413,12 +462,18 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           } else {
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
             mbar_expect_tx(bar, kTileBytes);
-            load_kv_block(p, &v_map, dst, b, g, j, bar);
+            if (!kSmallPages) load_kv_block(p, &v_map, dst, b, g, j, bar);
             ctl->v_req = n_before + 1;
+            v_go = 1;
           }
           dec_word |= 1u << (kk & 31);
         }
         if (p.decisions && ((kk & 31) == 31 || last)) { p.decisions[row * dec_words + (kk >> 5)] = dec_word; dec_word = 0; }
+      }
+      if (kSmallPages && compute) {              // every lane fetches one page's part of V_j
+        v_go = __shfl_sync(0xffffffffu, v_go, 0);
+        const int vs = n_before % kVStages;
+        if (v_go && lane < ppb) load_kv_block_part_at(p, &v_map, v_sm + vs * kTileBytes, vc, lane, smem_u32(&ctl->v_full[vs]));
       }
       __syncwarp();
       if (last) break;
@@ -675,15 +730,19 @@ cudaError_t launch_osk_tc(const OskParams& p_in, cudaStream_t st) {
   OskParams p = p_in;
   TileOrder vo;
   // K and V: the dense tensors, or page pools whose pages hold whole key blocks
-  if (p.pg.table && p.pg.page_size < kBlock) return cudaErrorInvalidValue;   // staged as dense tensors by the caller of this launcher
+  if (p.pg.table && p.pg.page_size < 8) return cudaErrorInvalidValue;
+  const int kv_box = (p.pg.table && p.pg.page_size < kBlock) ? p.pg.page_size : kBlock;   // small pages: one box per page
   if (!make_tile_map(&qm, &p.qo, p.q, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.qs) ||
-      !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n) || !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n) ||
+      !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n, kv_box) ||
+      !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n, kv_box) ||
       !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
   const bool strict = wait_budget_is_short(p.wait_budget);
+  const bool small_pages = p.pg.table && p.pg.page_size < kBlock;
   auto pick = [&](auto mask_c, auto strict_c) {
-    return p.stage2 ? osk_tc_kernel<decltype(mask_c)::value, decltype(strict_c)::value, true>
-                    : osk_tc_kernel<decltype(mask_c)::value, decltype(strict_c)::value, false>;
+    constexpr bool M = decltype(mask_c)::value, S = decltype(strict_c)::value;
+    return p.stage2 ? (small_pages ? osk_tc_kernel<M, S, true, true> : osk_tc_kernel<M, S, true, false>)
+                    : (small_pages ? osk_tc_kernel<M, S, false, true> : osk_tc_kernel<M, S, false, false>);
   };
   using T = std::true_type; using F = std::false_type;
   auto kernel = p.mask ? (strict ? pick(T{}, T{}) : pick(T{}, F{})) : (strict ? pick(F{}, T{}) : pick(F{}, F{}));

@@ -587,16 +587,20 @@ def test_paged_kv_small(small, impl, page_size):
         assert cosa.cosa_device_status() == 0
         ref_order, ref_count = O.kap_select(qf, kf, s=stride, budget=0.6, order_stride=nqb)
         assert np.array_equal(_np(count), ref_count) and np.array_equal(_np(order), ref_order)
-    for tb, skip_scale in ((1.0, 200.0), (0.4, 150.0)):
-        bufs = alloc_outputs(q, nqb)
-        opt = cosa.default_options(skip_scale=skip_scale, impl=impl, out_scored=bufs["scored"],
-                                   out_decisions=bufs["decisions"], **paging)
-        cosa.cosa_osk_attention(q, kpool, vpool, order, count, tb, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
-        assert cosa.cosa_device_status() == 0
-        check_osk_against_oracle(qf, kf, vf, ref_order, ref_count, bufs, tb, skip_scale, range(q.shape[1]), range(nqb))
-        dense = run_osk(q, k, v, order, count, tb, skip_scale, impl)
-        assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
-        assert torch.equal(dense["lse"], bufs["lse"])
+    # pages smaller than a block: staged as dense tensors (default), or read in place, tile by tile (no scratch)
+    for in_place in ((0, 1) if (impl == 0 and page_size < 128) else (0,)):
+        for tb, skip_scale in ((1.0, 200.0), (0.4, 150.0)):
+            bufs = alloc_outputs(q, nqb)
+            opt = cosa.default_options(skip_scale=skip_scale, impl=impl, out_scored=bufs["scored"],
+                                       out_decisions=bufs["decisions"], kv_pages_in_place=in_place, **paging)
+            if in_place:
+                assert cosa.cosa_workspace_bytes(1, cosa.make_shape(q, k), opt) == 0
+            cosa.cosa_osk_attention(q, kpool, vpool, order, count, tb, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+            assert cosa.cosa_device_status() == 0
+            check_osk_against_oracle(qf, kf, vf, ref_order, ref_count, bufs, tb, skip_scale, range(q.shape[1]), range(nqb))
+            dense = run_osk(q, k, v, order, count, tb, skip_scale, impl)
+            assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
+            assert torch.equal(dense["lse"], bufs["lse"])
 
 
 def test_paged_kv_4k(cfg1):
@@ -631,7 +635,7 @@ def test_paged_kv_rejects_bad_arguments(small):
 
 def test_paged_kv_small_pages_with_caller_workspace(small):
     """Pages smaller than a key block are staged as dense tensors in the scratch: a caller-owned workspace of the size
-    the library asks for gives the dense results, a smaller one is refused."""
+    the library asks for gives the dense results, a smaller one is refused; with kv_pages_in_place OSK needs none."""
     q, k, v = small["dev"]
     nqb = q.shape[2] // 128
     kpool, vpool, table, n_pages = _pools(small["w"], 16)
@@ -641,6 +645,7 @@ def test_paged_kv_small_pages_with_caller_workspace(small):
     need = cosa.cosa_workspace_bytes(2, shape, cosa.default_options(**paging))
     assert need >= 2 * kv_bytes
     assert cosa.cosa_workspace_bytes(1, shape, cosa.default_options(**paging)) >= 2 * kv_bytes
+    assert cosa.cosa_workspace_bytes(1, shape, cosa.default_options(kv_pages_in_place=1, **paging)) == 0
     assert cosa.cosa_workspace_bytes(1, shape, cosa.default_options()) == 0
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
     order, count = alloc_lists(q.shape[1], nqb)
@@ -648,12 +653,13 @@ def test_paged_kv_small_pages_with_caller_workspace(small):
     cosa.cosa_kap_select(q, kpool, 0.6, order, count, opt=opt)
     d_order, d_count = run_kap(q, k, 0.6)
     assert torch.equal(order, d_order) and torch.equal(count, d_count)
-    bufs = alloc_outputs(q, nqb)
-    cosa.cosa_osk_attention(q, kpool, vpool, order, count, 0.4, bufs["out"], bufs["lse"], bufs["visited"],
-                            opt=cosa.default_options(skip_scale=150.0, workspace=ws, workspace_bytes=need, **paging))
-    assert cosa.cosa_device_status() == 0
     dense = run_osk(q, k, v, order, count, 0.4, 150.0)
-    assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
+    for extra in (dict(workspace=ws, workspace_bytes=need), dict(kv_pages_in_place=1)):
+        bufs = alloc_outputs(q, nqb)
+        cosa.cosa_osk_attention(q, kpool, vpool, order, count, 0.4, bufs["out"], bufs["lse"], bufs["visited"],
+                                opt=cosa.default_options(skip_scale=150.0, **extra, **paging))
+        assert cosa.cosa_device_status() == 0
+        assert torch.equal(dense["out"], bufs["out"]) and torch.equal(dense["visited"], bufs["visited"])
     small_opt = cosa.default_options(workspace=ws, workspace_bytes=kv_bytes, **paging)
     with pytest.raises(cosa.CosaError):
         cosa.cosa_kap_select(q, kpool, 0.6, order, count, opt=small_opt)
@@ -661,7 +667,6 @@ def test_paged_kv_small_pages_with_caller_workspace(small):
         cosa.cosa_osk_attention(q, kpool, vpool, order, count, 0.4, bufs["out"], bufs["lse"], bufs["visited"], opt=small_opt)
 
 
-# ---------------------------------------------------------------------------------- batch > 1
 @pytest.mark.parametrize("impl", OSK_IMPLS)
 def test_batch_of_two_equals_single_items(impl):
     """Two different sequences in one call give exactly the results of two calls (dense and paged)."""
