@@ -161,6 +161,12 @@ void cosa_default_options(cosa_options* opt);
  * the dense staging tensors; otherwise OSK needs none. */
 size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options* opt);
 
+/* Sizes the library's own per-device scratch (the one calls without opt->workspace use) to at least `bytes` on the
+ * current device, now: allocates, and synchronises the device if a smaller scratch has to be freed first.  After
+ * cosa_reserve_scratch(cosa_workspace_bytes(2, shape, opt)) at start-up, plain calls of that shape or smaller allocate
+ * nothing and do not synchronise.  The scratch is never shrunk; it is released when the process ends. */
+int cosa_reserve_scratch(size_t bytes);
+
 /* Number of blocks kept out of `candidates` under a budget fraction: ceil(budget*candidates)
  * evaluated as (floor(budget_f32 * 2^20) * candidates + 2^20 - 1) >> 20, clamped to
  * [1, candidates].  This is how K_i = B_stage1 x J (Eq. 14) and the Stage-2 cap are rounded. */

@@ -23,6 +23,8 @@ Two tables, both produced with the library's own kernels only:
     python -m paper_2607_25291_b200.ablation sweep        (the 64K budget sweep)
 """
 import argparse
+import json
+import os
 
 import numpy as np
 import torch
@@ -144,9 +146,36 @@ def micro_table(workloads, budgets=MICRO_BUDGETS, with_sdpa=True):
     return rows
 
 
-def stack_table(workload, dense_every=6):
+class Journal:
+    """Rows of a long table kept as JSON lines, so that a run that was cut short resumes where it stopped: rows already
+    in the file are returned by `get` and not measured again."""
+
+    def __init__(self, path):
+        self.path, self.rows = path, {}
+        if path and os.path.exists(path):
+            with open(path) as f:
+                for line in f:
+                    line = line.strip()
+                    if line:
+                        row = json.loads(line)
+                        self.rows[row["key"]] = row
+
+    def get(self, key):
+        return self.rows.get(key)
+
+    def put(self, key, row):
+        row = dict(row, key=key)
+        self.rows[key] = row
+        if self.path:
+            with open(self.path, "a") as f:
+                f.write(json.dumps(row) + "\n")
+        return row
+
+
+def stack_table(workload, dense_every=6, journal=None):
     """One row per layer: KAP ms, OSK ms, blocks computed; the dense references are timed on every dense_every-th
-    layer (their time does not depend on the data) and averaged."""
+    layer (their time does not depend on the data) and averaged.  With a journal, layers it already holds are not run."""
+    journal = journal or Journal(None)
     rows, dense_ms, sdpa_ms = [], [], []
     nqb, hq = workload.n_blocks, workload.hq
     pitch = (cosa.cosa_budget_count(workload.kap_budget, nqb) + 7) // 8 * 8
@@ -156,14 +185,23 @@ def stack_table(workload, dense_every=6):
     opt = cosa.default_options(stride=workload.stride, skip_scale=workload.skip_scale, order_stride=pitch)
     out = None
     for layer in range(workload.layers):
+        need_dense = layer % dense_every == 0
+        have = journal.get(f"{workload.name}/layer{layer}")
+        have_dense = journal.get(f"{workload.name}/dense{layer}") if need_dense else None
+        if have is not None and (not need_dense or have_dense is not None):
+            rows.append(have)
+            if need_dense:
+                dense_ms.append(have_dense["dense_ms"]); sdpa_ms.append(have_dense["sdpa_ms"])
+            continue
         qb, kb, vb, _ = workload.make(layer=layer)
         q, k, v = _dev(qb), _dev(kb), _dev(vb)
         if out is None:
             out = torch.empty_like(q)
         kap = _time(lambda: cosa.cosa_kap_select(q, k, workload.kap_budget, order, count, opt=opt), reps=2)
         osk = _time(lambda: cosa.cosa_osk_attention(q, k, v, order, count, workload.osk_budget, out, None, visited, opt=opt), reps=2)
-        rows.append(dict(layer=layer, kap_ms=kap, osk_ms=osk, listed=int(count.sum()), computed=int(visited.sum())))
-        if layer % dense_every == 0:
+        rows.append(journal.put(f"{workload.name}/layer{layer}",
+                                dict(layer=layer, kap_ms=kap, osk_ms=osk, listed=int(count.sum()), computed=int(visited.sum()))))
+        if need_dense:
             tri = torch.arange(nqb, device="cuda", dtype=torch.int32)
             full = torch.where(tri[None, :] <= tri[:, None], tri[None, :].expand(nqb, nqb),
                                torch.full((), -1, dtype=torch.int32, device="cuda")).expand(1, hq, nqb, nqb).contiguous()
@@ -171,6 +209,7 @@ def stack_table(workload, dense_every=6):
             dopt = cosa.default_options(order_stride=nqb)
             dense_ms.append(_time(lambda: cosa.cosa_osk_attention(q, k, v, full, fcount, 1.0, out, None, None, opt=dopt), reps=1))
             sdpa_ms.append(_time(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v, is_causal=True, enable_gqa=True), reps=1))
+            journal.put(f"{workload.name}/dense{layer}", dict(dense_ms=dense_ms[-1], sdpa_ms=sdpa_ms[-1]))
             del full
         del q, k, v
     return rows, float(np.mean(dense_ms)), float(np.mean(sdpa_ms))
@@ -248,13 +287,15 @@ def main():
     ap.add_argument("--dense-every", type=int, default=6)
     ap.add_argument("--workload", default="qwen3_32k")
     ap.add_argument("--lengths", default="32k,64k,128k")
+    ap.add_argument("--jsonl", default=None,
+                    help="stack: keep the per-layer rows in this file (JSON lines) and resume from it if it exists")
     args = ap.parse_args()
     if args.table == "sweep":
         from synth.configs import SWEEP_STAGE1, SWEEP_STAGE2_MULT
         _print_sweep(sweep_table(WORKLOADS["llama31_64k_sweep"], SWEEP_STAGE1, SWEEP_STAGE2_MULT))
     elif args.table == "stack":
         wl = WORKLOADS[args.workload if args.workload != "qwen3_32k" else "qwen3_128k_x36"]
-        _print_stack(*stack_table(wl, args.dense_every))
+        _print_stack(*stack_table(wl, args.dense_every, Journal(args.jsonl)))
     elif args.table == "remap":
         _print_remap(remap_table(WORKLOADS[args.workload]))
     else:

@@ -26,7 +26,7 @@ COSA_ERR_DEVICE_TIMEOUT = -5
 COSA_ERR_BAD_ORDER = -6
 
 EXPORTS = (
-    "cosa_default_options", "cosa_workspace_bytes", "cosa_budget_count", "cosa_kap_select",
+    "cosa_default_options", "cosa_workspace_bytes", "cosa_reserve_scratch", "cosa_budget_count", "cosa_kap_select",
     "cosa_kap_select_ex", "cosa_kap_select_static", "cosa_kap_select_static_max_bytes", "cosa_osk_attention", "cosa_osk_attention_ex", "cosa_reorder_lists", "cosa_lists_to_mask", "cosa_validate_order",
     "cosa_host_call_workspace_bytes", "cosa_prefill_host", "cosa_device_status", "cosa_debug_set_device_status", "cosa_options_bytes", "cosa_shape_bytes",
     "cosa_last_cuda_error", "cosa_status_string", "cosa_version",
@@ -76,6 +76,8 @@ def _load():
     lib.cosa_default_options.restype = None
     lib.cosa_workspace_bytes.argtypes = [c_int, POINTER(CosaShape), POINTER(CosaOptions)]
     lib.cosa_workspace_bytes.restype = c_size_t
+    lib.cosa_reserve_scratch.argtypes = [c_size_t]
+    lib.cosa_reserve_scratch.restype = c_int
     lib.cosa_budget_count.argtypes = [c_float, c_int32]
     lib.cosa_budget_count.restype = c_int32
     lib.cosa_kap_select.argtypes = [c_void_p, c_void_p, POINTER(CosaShape), c_float, c_void_p, c_void_p, c_void_p]
@@ -180,6 +182,10 @@ def _set_strides(opt, q=None, k=None, v=None, out=None):
 
 def cosa_budget_count(budget: float, candidates: int) -> int:
     return int(_load().cosa_budget_count(budget, candidates))
+
+
+def cosa_reserve_scratch(nbytes: int) -> None:
+    _check(_load().cosa_reserve_scratch(int(nbytes)), "cosa_reserve_scratch")
 
 
 def cosa_workspace_bytes(op: int, shape: CosaShape, opt: CosaOptions | None = None) -> int:

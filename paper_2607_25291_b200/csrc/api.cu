@@ -6,6 +6,8 @@
 
 #include <mutex>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace cosa {
@@ -56,6 +58,12 @@ int own_scratch(size_t need, void** out) {
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// A named range around a call's enqueue work, for timelines of a profiler that follows NVTX (free when none is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
 
 // wide_q_ok: the caller accepts query blocks of 256 rows (KAP's shared-ranking variant)
 int check_shape(const cosa_shape* s, bool wide_q_ok = false) {
@@ -186,6 +194,7 @@ size_t cosa_workspace_bytes(int op, const cosa_shape* shape, const cosa_options*
 
 int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, float budget, int32_t* out_order,
                        int32_t* out_count, void* stream, const cosa_options* opt) {
+  NvtxRange range("cosa_kap_select");
   int rc = check_shape(shape, true);
   if (rc != COSA_OK) return rc;
   if (!q || !k || !out_order || !out_count) return COSA_ERR_INVALID_ARG;
@@ -284,6 +293,11 @@ int cosa_kap_select_ex(const void* q, const void* k, const cosa_shape* shape, fl
   return COSA_OK;
 }
 
+int cosa_reserve_scratch(size_t bytes) {
+  void* unused = nullptr;
+  return own_scratch(bytes, &unused);
+}
+
 int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape, float budget, int32_t* out_order,
                     int32_t* out_count, void* stream) {
   return cosa_kap_select_ex(q, k, shape, budget, out_order, out_count, stream, nullptr);
@@ -292,6 +306,7 @@ int cosa_kap_select(const void* q, const void* k, const cosa_shape* shape, float
 int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cosa_shape* shape, const int32_t* order,
                           const int32_t* count, float tightened_budget, void* out, float* out_lse,
                           int32_t* out_visited, void* stream, const cosa_options* opt) {
+  NvtxRange range("cosa_osk_attention");
   int rc = check_shape(shape);
   if (rc != COSA_OK) return rc;
   if (!q || !k || !v || !out) return COSA_ERR_INVALID_ARG;

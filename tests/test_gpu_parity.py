@@ -840,6 +840,26 @@ def test_kv_head_shards_concatenate_to_the_unsharded_result(small):
             assert torch.equal(torch.cat([p[2][key] for p in parts], 1), whole[key]), key
 
 
+def test_reserved_scratch_makes_plain_calls_allocation_free(cfg1):
+    """cosa_reserve_scratch sizes the library's own scratch ahead of time: the plain calls that follow allocate
+    nothing (the free memory of the device does not move)."""
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    nqb = w.n // 128
+    cosa.cosa_reserve_scratch(cosa.cosa_workspace_bytes(2, cosa.make_shape(q, k)))
+    order, count = alloc_lists(w.hq, nqb)
+    bufs = alloc_outputs(q, nqb)
+    def both():
+        cosa.cosa_kap_select(q, k, w.kap_budget, order, count)
+        cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, bufs["out"], bufs["lse"], bufs["visited"])
+        torch.cuda.synchronize()
+    both()                                               # (first use loads the kernels' code)
+    free = torch.cuda.mem_get_info()[0]
+    both()
+    assert torch.cuda.mem_get_info()[0] == free
+    assert cosa.cosa_device_status() == 0
+
+
 def test_osk_is_deterministic(cfg1):
     w = cfg1["w"]
     q, k, v = cfg1["dev"]
