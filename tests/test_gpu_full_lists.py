@@ -96,6 +96,77 @@ def compare_every_list(w, qb, kb, budget, score_heads=()):
     return dict(lists=w.hq * nqb, screen_rel_err=worst_err, min_rel_score_gap=min_gap, min_row_top2_gap=min_top2)
 
 
+def _osk_head(h):
+    """OSK of query head h on the chosen query blocks: decisions, counters, outputs against the oracle."""
+    try:
+        from threadpoolctl import threadpool_limits
+        limiter = threadpool_limits(1)
+    except Exception:
+        limiter = None
+    from tests.test_gpu_parity import check_osk_against_oracle
+    g = _G
+    G = g["qb"].shape[0] // g["kb"].shape[0]
+    qf = bf16_bits_to_f64(g["qb"][h])[None]
+    kf = bf16_bits_to_f64(g["kb"][h // G])[None]
+    vf = bf16_bits_to_f64(g["vb"][h // G])[None]
+    one = {k_: torch.from_numpy(a[h:h + 1])[None] for k_, a in g["bufs"].items()}
+    stats = check_osk_against_oracle(qf, kf, vf, g["order"][h:h + 1], g["count"][h:h + 1], one, g["osk_budget"], g["skip_scale"],
+                                     [0], g["blocks"])
+    del limiter
+    return h, stats
+
+
+def compare_every_work_item(w, qb, kb, vb, kap_budget, osk_budget):
+    """KAP then OSK on the whole workload; every (head, query block) of Stage 2 against the oracle."""
+    q, k, v = to_dev(qb), to_dev(kb), to_dev(vb)
+    nqb = w.n_blocks
+    pitch = (cosa.cosa_budget_count(kap_budget, nqb) + 7) // 8 * 8
+    order = torch.empty(1, w.hq, nqb, pitch, dtype=torch.int32, device="cuda")
+    count = torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda")
+    bufs = dict(out=torch.empty_like(q), lse=torch.empty(1, w.hq, w.n, dtype=torch.float32, device="cuda"),
+                visited=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                scored=torch.empty(1, w.hq, nqb, dtype=torch.int32, device="cuda"),
+                decisions=torch.zeros(1, w.hq, nqb, (pitch + 31) // 32, dtype=torch.int32, device="cuda"))
+    opt = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, out_scored=bufs["scored"],
+                               out_decisions=bufs["decisions"])
+    cosa.cosa_kap_select(q, k, kap_budget, order, count, opt=opt)
+    cosa.cosa_osk_attention(q, k, v, order, count, osk_budget, bufs["out"], bufs["lse"], bufs["visited"], opt=opt)
+    assert cosa.cosa_device_status() == 0
+    _G.clear()
+    _G.update(qb=qb, kb=kb, vb=vb, order=order[0].cpu().numpy(), count=count[0].cpu().numpy(), blocks=list(range(nqb)),
+              osk_budget=osk_budget, skip_scale=w.skip_scale,
+              bufs={k_: (t[0].float().cpu().numpy() if t.dtype == torch.bfloat16 else t[0].cpu().numpy()) for k_, t in bufs.items()})
+    del q, k, v, order, count, bufs
+    with mp.get_context("fork").Pool(max(1, min(w.hq, os.cpu_count() or 2))) as pool:
+        results = pool.map(_osk_head, range(w.hq), chunksize=1)
+    _G.clear()
+    return dict(items=w.hq * nqb, max_abs=float(max(s["max_abs"] for _, s in results)),
+                mean_abs=float(np.mean([s["mean_abs"] for _, s in results])), lse=float(max(s["lse"] for _, s in results)),
+                near_margin=sum(s["near_margin"] for _, s in results))
+
+
+def test_qwen3_128k_osk_on_every_work_item():
+    """Stage 2 at the benchmark's size on all 32,768 work items (every head x every query block): decision bits and
+    counters exact outside the oracle's 1e-4 margin, outputs and LSE within the bars, one head per worker process."""
+    w = WORKLOADS["qwen3_128k"]
+    qb, kb, vb, _ = w.make()
+    print("128k OSK", compare_every_work_item(w, qb, kb, vb, w.kap_budget, w.osk_budget))
+
+
+def test_llama31_64k_osk_on_every_work_item_of_two_sweep_cells():
+    """The 64K budget sweep: the 25 % Stage-1 column with Stage 2 at half of it, and with Stage 2 off."""
+    w = WORKLOADS["llama31_64k_sweep"]
+    qb, kb, vb, _ = w.make()
+    print("64k OSK 25%/12.5%", compare_every_work_item(w, qb, kb, vb, 0.25, 0.125))
+    print("64k OSK 12.5%/off", compare_every_work_item(w, qb, kb, vb, 0.125, 1.0))
+
+
+def test_qwen3_128k_stack_layer_osk_on_every_work_item():
+    w = WORKLOADS["qwen3_128k_x36"]
+    qb, kb, vb, _ = w.make(layer=4)                            # the layer with the densest needles
+    print("128k stack layer 4 OSK", compare_every_work_item(w, qb, kb, vb, w.kap_budget, w.osk_budget))
+
+
 def test_qwen3_128k_every_list_and_screen_error():
     w = WORKLOADS["qwen3_128k"]
     qb, kb, _, _ = w.make()

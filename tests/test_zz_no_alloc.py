@@ -76,3 +76,36 @@ def test_static_scratch_size_limit_at_the_sizes_the_header_names():
     assert e.value.status == -3
     torch.cuda.synchronize()
     assert int(count[0, 0, 0]) == -7 and int((order == -7).sum()) == order.numel()
+
+
+def test_static_scratch_entry_point_in_a_fresh_process_touches_no_allocator():
+    """In a process of its own, before any other entry point of the library has run: were the call to fall back on
+    the library's cudaMalloc'ed scratch, the free memory of the device would drop across it."""
+    import subprocess
+    import sys
+    code = r'''
+import sys, torch
+sys.path.insert(0, ".")
+import paper_2607_25291_b200 as cosa
+from synth.configs import tiny
+from tests.helpers import alloc_lists, to_dev
+qb, kb, _, _ = tiny(seed=31, hq=4, hkv=2, n=2048, needles=3).make()
+q, k = to_dev(qb), to_dev(kb)
+order, count = alloc_lists(4, 16)
+torch.cuda.synchronize()
+before = torch.cuda.mem_get_info()[0]
+cosa.cosa_kap_select_static(q, k, 0.3, order, count, opt=cosa.default_options())
+torch.cuda.synchronize()
+mid = torch.cuda.mem_get_info()[0]          # (the first launch loads the kernels' code: allowed to cost memory once)
+cosa.cosa_kap_select_static(q, k, 0.3, order, count, opt=cosa.default_options())
+torch.cuda.synchronize()
+after = torch.cuda.mem_get_info()[0]
+assert cosa.cosa_device_status() == 0 and int(count.min()) >= 1
+assert after == mid, (before, mid, after)
+assert before - mid < (64 << 20), (before, mid)   # (code loading only)
+print("ok", before - mid)
+'''
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    res = subprocess.run([sys.executable, "-c", code], cwd=root, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0 and "ok" in res.stdout, res.stdout + res.stderr
