@@ -412,7 +412,7 @@ def main():
                            "skip_scale": w.skip_scale,
                            "parallelism": (f"one layer, KV heads split over {world} ranks" if args.shard == "kv_head"
                                            else f"layer-per-rank x{world}"),
-                           "l2": "inputs (2.7 GB) exceed L2; no flush", "blocks_listed": n_listed,
+                           "l2": "inputs (%.1f GB) exceed L2; no flush" % ((q.numel() + k.numel() + v.numel()) * 2 / 1e9), "blocks_listed": n_listed,
                            "blocks_scored": n_scored, "blocks_computed": n_computed,
                            "causal_block_pairs": pairs, "input_generation_s": round(t_gen, 1)},
                 "latency_ms": {"kap": kap_ms, "osk": osk_ms, "kap_plus_osk": ms_per_step},

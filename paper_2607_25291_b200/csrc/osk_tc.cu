@@ -59,7 +59,7 @@ struct __align__(8) Control {
   unsigned long long q_stage, q_full, k_full[kKStages], v_full[kVStages];   // Q tile landed / Q copied into TMEM
   unsigned long long k_empty[kKStages];  // QK^T of that stage finished: the stage is free AND its S tile is ready
   unsigned long long s_empty[2];
-  unsigned long long p_full[2];   // P of computed block n is stored (barrier n & 1; the one buffer is free again after product n)
+  unsigned long long p_full;      // P of the next computed block is stored
   unsigned long long p_empty[2];  // PV product n signals p_empty[n & 1] (P free, O updated, V stage n & 1 free); two
                                   // barriers because a waiter may run two products ahead of the tensor pipe, which one
                                   // barrier's single parity bit cannot tell apart
@@ -73,7 +73,7 @@ struct __align__(8) Control {
   volatile int end_kk;            // last scored position, -1 until known
   volatile int k_loaded;          // K tiles the loader requested; -1 until it has stopped requesting
   volatile int final_computed;
-  volatile int v_req, v_taken;    // V tiles requested by the controller / whose arrival the PV issuer has waited for
+  volatile int v_req;             // V tiles the controller has requested (written once, when it leaves its loop)
   volatile int abort_flag;
   int poisoned;
   volatile uint32_t dec[kDecRing];
@@ -199,15 +199,15 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       mbar_init(smem_u32(&ctl->s_empty[s]), kBlock);
       mbar_init(smem_u32(&ctl->m_ready[s]), kBlock); mbar_init(smem_u32(&ctl->dec_bar[s]), 1);
       mbar_init(smem_u32(&ctl->p_empty[s]), 1);
-      mbar_init(smem_u32(&ctl->p_full[s]), kBlock);
     }
     mbar_init(smem_u32(&ctl->out_bar), kBlock);
+    mbar_init(smem_u32(&ctl->p_full), kBlock);
     mbar_init(smem_u32(&ctl->fin_bar), kBlock);
     ctl->n_dec = 0;
     ctl->end_kk = kStage2 ? -1 : cnt - 1;          // Stage 2 off: the walk ends with the list
     ctl->k_loaded = -1;
     ctl->final_computed = kStage2 ? 0 : cnt;
-    ctl->v_req = 0; ctl->v_taken = 0;
+    ctl->v_req = 0;
     ctl->abort_flag = 0;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -243,7 +243,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   const uint32_t tmem = ctl->tmem_base;
   const uint32_t tmem_s[2] = {tmem, tmem + 128u};
   const uint32_t tmem_o = tmem + 256u;
-  const uint32_t tmem_p[2] = {tmem + 384u, tmem + 384u};   // one buffer
+  const uint32_t tmem_p = tmem + 384u;
   const uint32_t tmem_q = tmem + 448u;
   volatile int* abort_flag = &ctl->abort_flag;
   const long long budget = p.wait_budget;
@@ -373,7 +373,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       int n_issued = 0;
       for (int n = 0; alive; ++n) {
         // the next computed block's P, or the end of the walk
-        const uint32_t bar = smem_u32(&ctl->p_full[n & 1]), par = (n >> 1) & 1;
+        const uint32_t bar = smem_u32(&ctl->p_full), par = n & 1;
         bool done = false;
         if (!mbar_try_wait(bar, par)) {
           const long long t0 = clock64();
@@ -386,10 +386,9 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
         const int vs = n % kVStages;
         alive = mbar_wait(smem_u32(&ctl->v_full[vs]), (n / kVStages) & 1, abort_flag, budget);
         if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
-        ctl->v_taken = n + 1;
         tc_fence_after();
         // 16 keys per MMA: 8 TMEM columns of P, 2 KiB (two 8-key groups) of the V tile
-        mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p[n & 1], vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
+        mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem_o, tmem_p, vdesc0 + (uint64_t)(vs * (kTileBytes / 16)), idesc_pv, n > 0);
         mma_commit(smem_u32(&ctl->p_empty[n & 1]));
         n_issued = n + 1;
       }
@@ -399,6 +398,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else if (warp == 2) {
     // ------------------------------------------------------------------ controller
     int computed = 0, n_needed = min(cnt, cap), scored = 0;
+    int n_vreq = 0;                  // (lane 0) V tiles requested so far
     uint32_t dec_word = 0;
     const int dec_words = (p.order_stride + 31) / 32;
     bool alive = true;
@@ -418,7 +418,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           } else {
             mbar_expect_tx(bar, kTileBytes);
             if (!kSmallPages) load_kv_block(p, &v_map, dst, b, g, j, bar);
-            ctl->v_req = kk + 1;
+            n_vreq = kk + 1;
           }
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -463,7 +463,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
             const uint32_t dst = v_sm + vs * kTileBytes, bar = smem_u32(&ctl->v_full[vs]);
             mbar_expect_tx(bar, kTileBytes);
             if (!kSmallPages) load_kv_block(p, &v_map, dst, b, g, j, bar);
-            ctl->v_req = n_before + 1;
+            n_vreq = n_before + 1;
             v_go = 1;
           }
           dec_word |= 1u << (kk & 31);
@@ -478,6 +478,7 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
       __syncwarp();
       if (last) break;
     }
+    if (lane == 0) ctl->v_req = n_vreq;
     if (lane == 0 && alive && !*abort_flag) {
       if (p.visited) p.visited[row] = computed;
       if (p.scored) p.scored[row] = scored;
@@ -644,11 +645,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           }
         }
       }
-      tmem_st32(tmem_p[n_before & 1] + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
-      tmem_st32(tmem_p[n_before & 1] + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
+      tmem_st32(tmem_p + lane_addr, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+      tmem_st32(tmem_p + lane_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(smem_u32(&ctl->p_full[n_before & 1]));
+      mbar_arrive(smem_u32(&ctl->p_full));
       l = l * ex2_approx(m_ref - m_new) + ((rs[0] + rs[1]) + (rs[2] + rs[3]));
       m_ref = m_new;
       if (last) break;
@@ -716,9 +717,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) {
-    // copies that nobody has waited for when the walk was given up: the Q tile, a V tile the PV issuer never took
+    // copies that nobody may have waited for when the walk was given up: the Q tile, and the last V tiles the controller
+    // requested (a tile the PV issuer did take has completed its barrier phase: the wait returns at once)
     (void)mbar_wait_noabort(smem_u32(&ctl->q_stage), 0);
-    for (int n = ctl->v_taken; n < ctl->v_req; ++n) (void)mbar_wait_noabort(smem_u32(&ctl->v_full[n % kVStages]), (n / kVStages) & 1);
+    const int nv = ctl->v_req;
+    for (int n = max(0, nv - kVStages); n < nv; ++n) (void)mbar_wait_noabort(smem_u32(&ctl->v_full[n % kVStages]), (n / kVStages) & 1);
   }
   if (warp == 1) tmem_dealloc(tmem, kTmemCols);
 }
