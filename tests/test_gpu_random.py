@@ -144,3 +144,59 @@ def test_random_paged_and_ragged_batches_equal_dense():
                 ln = lens[b] if use_lens else n
                 rows = ln // 128 if name in ("order", "count", "visited") else ln
                 assert torch.equal(ref[name][b, :, :rows], got[name][b, :, :rows]), (name, b, what)
+
+
+def _relayout(t, layout, pad):
+    """The [B,H,N,d] tensor `t` as a view with other strides holding the same values: token-major [B,N,H,d], batch
+    innermost of the outer three [N,H,B,d]... or the dense layout with padded row and head pitches."""
+    B, H, N, d = t.shape
+    if layout == "dense":
+        return t
+    if layout == "token_major":
+        return t.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    if layout == "head_major_batch_inner":                      # memory order [H, N, B, d]
+        return t.permute(1, 2, 0, 3).contiguous().permute(2, 0, 1, 3)
+    if layout == "padded":                                      # rows 8 or 16 elements apart more than they need, heads with slack
+        buf = torch.zeros(B, H, N + 3, d + pad, dtype=t.dtype, device=t.device)
+        buf[:, :, :N, :d] = t
+        return buf[:, :, :N, :d]
+    raise ValueError(layout)
+
+
+def test_random_layouts_agree_with_the_dense_layout():
+    """q, k, v and out in randomly drawn layouts (token-major, batch innermost, padded pitches; one batch item or two):
+    lists, outputs, LSE and counters equal those of the dense layout bit for bit, on the tensor-core kernels and the
+    check kernels alike."""
+    rng = np.random.default_rng(20260801)
+    layouts = ("dense", "token_major", "head_major_batch_inner", "padded")
+    for _ in range(16):
+        hq, hkv = _draw_heads(rng)
+        B = int(rng.choice([1, 2]))
+        n = int(rng.choice([512, 1024, 2048]))
+        impl = int(rng.choice([0, 0, 1, 4]))
+        budget, tb = float(rng.choice([0.3, 0.6, 1.0])), float(rng.choice([0.2, 0.5, 1.0]))
+        qs, ks, vs = [], [], []
+        for b in range(B):
+            qb, kb, vb, _ = tiny(seed=int(rng.integers(1, 10**6)), hq=hq, hkv=hkv, n=n, needles=int(rng.integers(0, 5))).make()
+            qs.append(_dev(qb)); ks.append(_dev(kb)); vs.append(_dev(vb))
+        q, k, v = torch.stack(qs), torch.stack(ks), torch.stack(vs)
+        nqb = n // 128
+        def run(qq, kk, vv, out):
+            order = torch.full((B, hq, nqb, nqb), -5, dtype=torch.int32, device="cuda")
+            count = torch.full((B, hq, nqb), -5, dtype=torch.int32, device="cuda")
+            lse = torch.empty(B, hq, n, dtype=torch.float32, device="cuda")
+            vis = torch.empty(B, hq, nqb, dtype=torch.int32, device="cuda")
+            cosa.cosa_kap_select(qq, kk, budget, order, count, opt=cosa.default_options(impl=impl))
+            cosa.cosa_osk_attention(qq, kk, vv, order, count, tb, out, lse, vis, opt=cosa.default_options(skip_scale=150.0, impl=impl))
+            assert cosa.cosa_device_status() == 0
+            return order, count, lse, vis
+        ref_out = torch.empty_like(q)
+        ref = run(q, k, v, ref_out)
+        lq, lkv, lo = (str(rng.choice(layouts)) for _ in range(3))
+        pq, pkv, po = (int(rng.choice([8, 16, 64])) for _ in range(3))
+        out_buf = _relayout(torch.zeros_like(q), lo, po)
+        got = run(_relayout(q, lq, pq), _relayout(k, lkv, pkv), _relayout(v, lkv, pkv), out_buf)
+        what = dict(B=B, hq=hq, hkv=hkv, n=n, impl=impl, budget=budget, tb=tb, layouts=(lq, lkv, lo))
+        for a, b_ in zip(ref, got):
+            assert torch.equal(a, b_), what
+        assert torch.equal(out_buf, ref_out), what
