@@ -92,7 +92,7 @@ def test_random_paged_and_ragged_batches_equal_dense():
     """Page pools of any page size (8..512 tokens), with and without per-item lengths, give bit for bit the lists and
     outputs of the dense tensors they hold."""
     rng = np.random.default_rng(20260727)
-    for _ in range(24):
+    for _ in range(36):
         hq, hkv = _draw_heads(rng)
         n = int(rng.choice([1024, 2048]))
         B = int(rng.choice([1, 2]))
@@ -136,9 +136,10 @@ def test_random_paged_and_ragged_batches_equal_dense():
             return dict(order=order, count=count, out=out, lse=lse, visited=vis)
 
         ref = run(k, v)
-        got = run(kpool, vpool, kv_page_table=table, kv_page_size=ps, kv_num_pages=kpool.shape[0])
+        in_place = int(ps < 128 and rng.random() < 0.6)     # small pages: staged (default) or read in place
+        got = run(kpool, vpool, kv_page_table=table, kv_page_size=ps, kv_num_pages=kpool.shape[0], kv_pages_in_place=in_place)
         what = dict(hq=hq, hkv=hkv, n=n, B=B, ps=ps, lens=lens if use_lens else None, budget=budget, tb=tb, causal=causal,
-                    stride=stride, skip=skip)
+                    stride=stride, skip=skip, in_place=in_place)
         for name in ref:
             for b in range(B):
                 ln = lens[b] if use_lens else n
