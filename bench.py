@@ -53,11 +53,15 @@ def parse():
                          "ONE layer by KV-head group, rank r running KAP + OSK on its heads only (strong scaling; N <= KV heads)")
     ap.add_argument("--pages-in-place", action="store_true",
                     help="with --page-size below 128: OSK reads the pages in place (cosa_options.kv_pages_in_place), no staging copy")
-    ap.add_argument("--osk-impl", type=int, default=0, choices=[0, 4],
-                    help="4: the OSK kernel that walks two work items per CTA (cosa_options.impl = 4); not the headline config")
+    ap.add_argument("--osk-impl", type=int, default=0, choices=[0, 4, 5],
+                    help="4: the OSK kernel that walks two work items per CTA (cosa_options.impl = 4); 5: the same kernel on the two row "
+                         "tiles of a 256-row query block, every fetched K/V tile serving both (needs --block-q 256); not the headline config")
     ap.add_argument("--top-p", type=float, default=0.0,
                     help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
-    return ap.parse_args()
+    args = ap.parse_args()
+    if args.osk_impl == 5 and args.block_q != 256:
+        ap.error("--osk-impl 5 walks the lists of --block-q 256")
+    return args
 
 
 def measured_peaks():
@@ -361,7 +365,7 @@ def main():
         r.update(extra)
         return r
 
-    roof_osk = tensor_roof("osk_duo_kernel" if args.osk_impl == 4 else "osk_tc_kernel", osk_tflops, {"traffic": (traffic or {}).get("osk_tc_kernel")})
+    roof_osk = tensor_roof("osk_duo_kernel" if args.osk_impl in (4, 5) else "osk_tc_kernel", osk_tflops, {"traffic": (traffic or {}).get("osk_tc_kernel")})
     # KAP: the screen kernel forms the sampled logits on the tensor cores (one pass over the key tiles; whole tiles,
     # so somewhat more than the causal pairs), the sort kernel is ALU work; the algorithmic FLOPs (causal pairs only)
     # are set against the tensor peak, and the algorithmic bytes (sampled rows read once, lists written once)
@@ -408,7 +412,7 @@ def main():
                 "scaling": "strong" if args.shard == "kv_head" else "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                 "config": {"workload": w.name, "hq": w.hq, "hkv": w.hkv, "seq_len": w.n, "head_dim": 128, "block": 128,
-                           "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "kap_block_q": args.block_q, "osk_kernel": "osk_duo_kernel" if args.osk_impl == 4 else "osk_tc_kernel", "osk_budget": w.osk_budget, "stride": w.stride,
+                           "kap_budget": kap_budget, "top_p": args.top_p or None, "kv_page_size": args.page_size or None, "kap_block_q": args.block_q, "osk_kernel": "osk_duo_kernel" if args.osk_impl in (4, 5) else "osk_tc_kernel", "osk_budget": w.osk_budget, "stride": w.stride,
                            "skip_scale": w.skip_scale,
                            "parallelism": (f"one layer, KV heads split over {world} ranks" if args.shard == "kv_head"
                                            else f"layer-per-rank x{world}"),

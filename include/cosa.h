@@ -49,7 +49,8 @@ typedef enum {
   COSA_ERR_WORKSPACE = -3,     /* workspace missing or too small                                 */
   COSA_ERR_CUDA = -4,          /* a CUDA runtime call failed (see cosa_last_cuda_error)          */
   COSA_ERR_DEVICE_TIMEOUT = -5,/* a bounded device-side wait ran out (from cosa_device_status)   */
-  COSA_ERR_BAD_ORDER = -6      /* an order list holds an id outside its legal range              */
+  COSA_ERR_BAD_ORDER = -6      /* an order list holds an id outside its legal range (or, with
+                                  impl = 5, the lists of a 256-row block are not nested)          */
 } cosa_status;
 
 /* Problem shape shared by both stages. */
@@ -95,7 +96,15 @@ typedef struct {
                               runs the kernel that walks two work items per CTA, each with a softmax
                               group, an S and an O accumulator of its own (the arrangement a 256-row
                               query block with one vote per 128-row tile takes; measured slower than
-                              one work item per CTA, kept for comparison)                          */
+                              one work item per CTA, kept for comparison); 5 = as 4, and the two work
+                              items of a CTA are the two 128-row tiles of one 256-row query block
+                              (Sec. C.1), which walk one ranking together so that every K and V tile
+                              the CTA fetches serves both: for the lists cosa_kap_select writes with
+                              block_q = 256 (the first tile's list a subsequence of the second's;
+                              anything else is reported as COSA_ERR_BAD_ORDER through
+                              cosa_device_status and the call's results are then unspecified); N a
+                              multiple of 256, no logical_mask, no seq_lens; slower again (the tiles
+                              advance in lock-step), kept as the shared-fetch form of that variant   */
   float   top_p;           /* KAP only.  > 0: Top-p retention (Sec. 4.2, text after Eq. 13; p = 0.95
                               in Sec. C.1): K_i = length of the shortest prefix of the order whose
                               scores sum to >= top_p * (sum over all candidates), never more than

@@ -160,7 +160,7 @@ static size_t kap_scratch_bytes(const cosa_shape* s, const cosa_options& o) { re
 // (with kv_pages_in_place the default kernel assembles a tile from one pair of boxes per page instead, issued by the lanes
 // of a warp side by side, and needs no scratch)
 static bool osk_gathers(const cosa_options& o) {
-  return o.kv_page_table && o.impl != 1 && o.kv_page_size < kBlock && (o.impl == 4 || !o.kv_pages_in_place);
+  return o.kv_page_table && o.impl != 1 && o.kv_page_size < kBlock && (o.impl == 4 || o.impl == 5 || !o.kv_pages_in_place);
 }
 static size_t osk_scratch_bytes(const cosa_shape* s, const cosa_options& o) {
   return osk_gathers(o) ? 2 * align_up((size_t)s->batch * s->hkv * s->n * s->d * 2, 256) : 0;
@@ -341,6 +341,8 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   p.theta = p.use_threshold ? (float)log((double)o.skip_scale / (double)shape->n) : 0.f;
   p.skip_scale = o.skip_scale;
   p.scale = o.softmax_scale > 0.f ? o.softmax_scale : (float)(1.0 / sqrt((double)shape->d));
+  // impl = 5 walks the two row tiles of a 256-row query block together: list-driven, whole blocks of 256 rows
+  if (o.impl == 5 && (o.logical_mask || o.seq_lens || shape->n % (2 * kBlock) != 0)) return COSA_ERR_UNSUPPORTED;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (osk_gathers(o)) {
     const size_t need = osk_scratch_bytes(shape, o), one = need / 2;
@@ -365,7 +367,7 @@ int cosa_osk_attention_ex(const void* q, const void* k, const void* v, const cos
   }
   if (!p.pg.table && !strides_given(o.kv_strides)) p.ks = dense_strides(p.hkv, p.n);
   p.wait_budget = o.wait_cycles > 0 ? (long long)o.wait_cycles : (1LL << 31);
-  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : (o.impl == 4 ? launch_osk_duo(p, st) : launch_osk_tc(p, st));
+  cudaError_t e = (o.impl == 1) ? launch_osk_check(p, st) : ((o.impl == 4 || o.impl == 5) ? launch_osk_duo(p, o.impl == 5, st) : launch_osk_tc(p, st));
   if (e != cudaSuccess) return cuda_fail(e, "osk launch");
   return COSA_OK;
 }

@@ -225,7 +225,7 @@ cudaError_t launch_gather_pages(const __nv_bfloat16* pool, __nv_bfloat16* dense,
                                 int every, cudaStream_t st);   // (pools are contiguous; the staging tensor is dense)
 cudaError_t launch_osk_check(const OskParams& p, cudaStream_t st);
 cudaError_t launch_osk_tc(const OskParams& p, cudaStream_t st);
-cudaError_t launch_osk_duo(const OskParams& p, cudaStream_t st);
+cudaError_t launch_osk_duo(const OskParams& p, bool shared, cudaStream_t st);
 cudaError_t launch_reorder_lists(int32_t* order, const int32_t* count, int total_qb, int order_stride, int descending,
                                  cudaStream_t st);
 cudaError_t launch_lists_to_mask(const int32_t* order, const int32_t* count, int total_qb, int order_stride, int nkb,

@@ -20,6 +20,15 @@
 // Only listed blocks are ever fetched ("physical jumping"); at most one K tile per item is fetched beyond the
 // walk's end.
 // TMEM columns: S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512).
+//
+// kShared: the two work items are the two 128-row tiles of one 256-row query block (Sec. C.1: blocks of 256 query rows
+// with the skip test still taken per 128 rows), whose lists come from one ranking: the second tile's list is the
+// ranking, the first tile's is the ranking without the key blocks that lie wholly after it.  The CTA then walks the
+// ranking once and every K and V tile it fetches serves both tiles: one thread requests the tiles (a ring of three K
+// slots, requested two positions ahead, and one V slot) and issues the products of both items; at each position an
+// item takes part if the ranking's entry is the next entry of its own list; each group votes, skips or computes and
+// ends on its own cap as before; V_j is requested once if either item computes block j.  A first list that is not a
+// subsequence of the second cannot be walked this way: the CTA reports COSA_ERR_BAD_ORDER and writes nothing.
 // Every wait is bounded; a wait that runs out sets the device status word and the CTA winds down without
 // writing results, after the copies and products it has in flight have finished.
 #include <math.h>
@@ -37,7 +46,8 @@ constexpr int kTileBytes = kBlock * kHeadDim * 2;  // 32 KiB: one 128 x 128 bf16
 constexpr int kHalfBytes = kTileBytes / 2;         // one TMA box: 128 rows x 64 columns
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
-constexpr int kTiles = 6;                          // Q_0 Q_1, two slots per item
+constexpr int kTiles = 6;                          // Q_0 Q_1, two slots per item (kShared: three K slots and one V slot)
+constexpr int kKRing = 3;                          // kShared: K slots
 constexpr uint32_t kOutCompute = 1, kOutEnd = 2;
 
 struct __align__(8) DuoControl {
@@ -59,6 +69,8 @@ struct __align__(8) DuoControl {
   volatile int v_taken[2];           // V tiles whose arrival the issuer has waited for
   volatile uint32_t out_w[2][2];     // [item][k & 1]
   unsigned vote[2][2][4];            // [item][k & 1][warp]: bits of max over the warp's rows of (m_loc - m), <= 0
+  unsigned long long kr_full[kKRing];// kShared: the K tile of ranking position k has landed in slot k % 3
+  unsigned long long vs_full;        // kShared: the V tile requested last has landed
 };
 
 constexpr size_t kSmemBytes = (size_t)kTileBytes * kTiles + sizeof(DuoControl);
@@ -85,7 +97,8 @@ __device__ __forceinline__ void load_kv_block(const OskParams& p, const CUtensor
 }
 
 // kMask: walk a binary block mask instead of the order lists (see BlockWalk)
-template <bool kMask>
+// kShared: the items are the two row tiles of a 256-row query block and share every fetched tile (see above; lists only)
+template <bool kMask, bool kShared>
 __global__ void __launch_bounds__(kThreads, 1)
 osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                const __grid_constant__ CUtensorMap v_map, const __grid_constant__ CUtensorMap o_map, OskParams p,
@@ -101,20 +114,26 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int t = warp < 4 ? (warp & 1) : ((warp - 4) >> 2);   // the item this thread works for
   const uint32_t q_sm = base + t * kTileBytes;
-  const uint32_t x_sm = base + (2 + 2 * t) * kTileBytes;     // the item's two tile slots
+  const uint32_t x_sm = base + (2 + 2 * t) * kTileBytes;     // the item's two tile slots (not kShared)
+  const uint32_t kr_sm = base + 2 * kTileBytes;              // kShared: the K ring, then the V slot
+  const uint32_t vs_sm = base + (2 + kKRing) * kTileBytes;
 
   // work items in the order: KV head major, then query blocks from the longest list down, the group's query heads
   // innermost; a CTA takes two neighbours, which have lists of similar length and read much the same K/V pages
+  // (kShared: the same order over 256-row blocks; the CTA takes the block's two row tiles)
   const int total = p.batch * p.hq * p.nqb;
   const int w_raw = 2 * blockIdx.x + t;
-  const bool valid = w_raw < total;
+  const bool valid = kShared || w_raw < total;
   const int w = valid ? w_raw : total - 1;
   const int G = p.hq / p.hkv;
-  const int per_kv = G * p.nqb;
-  const int b = w / (p.hkv * per_kv);
-  const int wk = w % (p.hkv * per_kv);
+  const int nqb_u = kShared ? p.nqb / 2 : p.nqb;             // query blocks in units of the CTA's assignment
+  const int per_kv = G * nqb_u;
+  const int wu = kShared ? (int)blockIdx.x : w;
+  const int b = wu / (p.hkv * per_kv);
+  const int wk = wu % (p.hkv * per_kv);
   const int g = wk / per_kv;
-  const int i = p.nqb - 1 - (wk % per_kv) / G;
+  const int iu = nqb_u - 1 - (wk % per_kv) / G;
+  const int i = kShared ? 2 * iu + t : iu;
   const int h = g * G + (wk % per_kv) % G;
   const size_t row = (size_t)(b * p.hq + h) * p.nqb + i;
   const int nqb_b = item_blocks(p.pg, b, p.nqb);   // the item's own length in blocks; query blocks past it are padding
@@ -149,6 +168,10 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
     ctl->poisoned[t] = pois;       // once some CTA has reported a timeout the rest of the grid returns at once
     ctl->grp_bad[t][0] = 0; ctl->grp_bad[t][1] = 0; ctl->fin_bad[t] = 0; ctl->v_req[t] = 0; ctl->v_taken[t] = 0;
     if (t == 0) ctl->abort_flag = 0;
+    if (kShared && t == 1) {
+      for (int sl = 0; sl < kKRing; ++sl) mbar_init(smem_u32(&ctl->kr_full[sl]), 1);
+      mbar_init(smem_u32(&ctl->vs_full), 1);
+    }
     mbar_fence_init();
     fence_proxy_async_smem();
     if (pois == 0 && cnt > 0) {
@@ -156,8 +179,15 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
       mbar_expect_tx(qb, kTileBytes);
       tma_load_tile(q_sm, &q_map, 0, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, qb);
       tma_load_tile(q_sm + kHalfBytes, &q_map, 64, i * kBlock, h, b, p.qo.row, p.qo.head, p.qo.outer, qb);
-      load_kv_block(p, &k_map, x_sm, b, g, min(max(j0, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][0]));
-      if (cnt > 1) load_kv_block(p, &k_map, x_sm + kTileBytes, b, g, min(max(j1, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][1]));
+      if (!kShared) {
+        load_kv_block(p, &k_map, x_sm, b, g, min(max(j0, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][0]));
+        if (cnt > 1) load_kv_block(p, &k_map, x_sm + kTileBytes, b, g, min(max(j1, 0), p.nqb - 1), smem_u32(&ctl->k_full[t][1]));
+      } else if (t == 1) {
+        // the second tile's list is the ranking the CTA walks: its first tiles (this thread has initialised their barriers)
+        load_kv_block(p, &k_map, kr_sm, b, g, min(max(j0, 0), p.nqb - 1), smem_u32(&ctl->kr_full[0]));
+        if (cnt > 1) load_kv_block(p, &k_map, kr_sm + kTileBytes, b, g, min(max(j1, 0), p.nqb - 1), smem_u32(&ctl->kr_full[1]));
+        if (cnt > 2) load_kv_block(p, &k_map, kr_sm + 2 * kTileBytes, b, g, min(max(list[2], 0), p.nqb - 1), smem_u32(&ctl->kr_full[2]));
+      }
     }
   }
   if (warp == 2) {
@@ -171,8 +201,12 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
   if ((ctl->poisoned[0] | ctl->poisoned[1]) != 0) {   // nothing was requested by an issuer that saw the word set; the other one's copies must land
     if (issuer && ctl->poisoned[t] == 0 && cnt > 0) {
       (void)mbar_wait_noabort(smem_u32(&ctl->q_full[t]), 0);
-      (void)mbar_wait_noabort(smem_u32(&ctl->k_full[t][0]), 0);
-      if (cnt > 1) (void)mbar_wait_noabort(smem_u32(&ctl->k_full[t][1]), 0);
+      if (!kShared) {
+        (void)mbar_wait_noabort(smem_u32(&ctl->k_full[t][0]), 0);
+        if (cnt > 1) (void)mbar_wait_noabort(smem_u32(&ctl->k_full[t][1]), 0);
+      } else if (t == 1) {
+        for (int sl = 0; sl < min(cnt, kKRing); ++sl) (void)mbar_wait_noabort(smem_u32(&ctl->kr_full[sl]), 0);
+      }
     }
     __syncthreads();
     if (warp == 2) tmem_dealloc(tmem, kTmemCols);
@@ -189,7 +223,123 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
 
   if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-    if (issuer) {
+    if (kShared && issuer && t == 1) {
+      // ------------------------------------------------------------------ one issuer for both tiles: walks the ranking
+      const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);     // Q [M x K] and K_j [N x K], both K-major
+      const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);   // P [M x K] from TMEM, V_j [K x N] N-major
+      const int32_t* list0 = p.order + (row - 1) * p.order_stride;    // the first tile's own list
+      const int cnt1 = cnt;
+      const int cnt0 = max(0, min(p.count[row - 1], p.order_stride));
+      auto rank_at = [&](int k) { return (k < cnt1 && k < p.order_stride) ? min(max(list[k], 0), p.nqb - 1) : 0; };
+      auto own_at = [&](int k) { return (k < cnt0 && k < p.order_stride) ? min(max(list0[k], 0), p.nqb - 1) : -1; };
+      int r0 = rank_at(0), r1 = rank_at(1), r2 = rank_at(2), r3 = rank_at(3);   // ranking entries k .. k + 3
+      int a0 = own_at(0), a1 = own_at(1);                                      // the first tile's next two entries
+      int kl[2] = {0, 0};           // positions each item has taken part in
+      int nn[2] = {0, 0};           // blocks each item has computed
+      bool act[2] = {cnt0 > 0, cnt1 > 0};
+      int k_req = min(cnt1, kKRing), k_taken = 0, v_req = 0, v_taken = 0;
+      uint32_t pend_bar[2] = {0, 0}, pend_par[2] = {0, 0};   // per item: the last commit, while nobody is known to have seen it
+      bool alive = true;
+      for (int tt = 0; tt < 2 && alive; ++tt)
+        if (act[tt]) {
+          alive = mbar_wait(smem_u32(&ctl->q_full[tt]), 0, abort_flag, budget);
+          if (!alive && !*abort_flag) report_timeout(ctl, status);
+        }
+      for (int k = 0; k < cnt1 && alive && (act[0] || act[1]); ++k) {
+        const int j = r0;
+        const uint32_t slot_sm = kr_sm + (k % kKRing) * kTileBytes;
+        // K(k+2) goes where K(k-1) was: both items are done with that one (their outcomes have been seen)
+        if (k >= 1 && k + 2 < cnt1) {
+          load_kv_block(p, &k_map, kr_sm + ((k + 2) % kKRing) * kTileBytes, b, g, r2, smem_u32(&ctl->kr_full[(k + 2) % kKRing]));
+          k_req = k + 3;
+        }
+        const bool part[2] = {act[0] && a0 == j, act[1]};
+        alive = mbar_wait(smem_u32(&ctl->kr_full[k % kKRing]), (k / kKRing) & 1, abort_flag, budget);
+        if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+        k_taken = k + 1;
+        tc_fence_after();
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt)
+          if (part[tt]) {
+            mma_ss_x8<2, 4, 6, kHalfBytes / 16, kHalfBytes / 16 + 2, kHalfBytes / 16 + 4, kHalfBytes / 16 + 6>(
+                tmem + tt * 128u, smem_desc_sw128(base + tt * kTileBytes, 16, 1024), smem_desc_sw128(slot_sm, 16, 1024), idesc_qk);
+            mma_commit(smem_u32(&ctl->s_full[tt]));
+            pend_bar[tt] = smem_u32(&ctl->s_full[tt]); pend_par[tt] = kl[tt] & 1;
+          }
+        // the list entries further on, on their way while the groups decide
+        r0 = r1; r1 = r2; r2 = r3; r3 = rank_at(k + 4);
+        if (part[0]) { a0 = a1; a1 = own_at(kl[0] + 2); }
+        uint32_t ow[2] = {0, 0};
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt)
+          if (part[tt] && alive) {
+            alive = mbar_wait(smem_u32(&ctl->outcome[tt]), kl[tt] & 1, abort_flag, budget);
+            if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+            pend_bar[tt] = 0;                     // the group has S: the product is over
+            ow[tt] = ctl->out_w[tt][kl[tt] & 1];
+          }
+        if (!alive) break;
+        bool need[2] = {(ow[0] & kOutCompute) != 0, (ow[1] & kOutCompute) != 0};
+        if (need[0] || need[1]) {
+          // V_j once for both (the slot is free: every earlier P V product was waited for below)
+          load_kv_block(p, &v_map, vs_sm, b, g, j, smem_u32(&ctl->vs_full));
+          ++v_req;
+          const bool comp[2] = {need[0], need[1]};
+          const long long t0 = clock64();
+          while (need[0] || need[1]) {            // whichever group has its P ready first
+#pragma unroll
+            for (int tt = 0; tt < 2; ++tt)
+              if (need[tt] && mbar_try_wait(smem_u32(&ctl->p_full[tt]), nn[tt] & 1)) {
+                if (v_taken < v_req) {
+                  alive = mbar_wait(smem_u32(&ctl->vs_full), (v_req - 1) & 1, abort_flag, budget);
+                  if (!alive) break;
+                  v_taken = v_req;
+                }
+                tc_fence_after();
+                mma_ts_x8<128, 256, 384, 512, 640, 768, 896>(tmem + 256u + tt * 128u, tmem + tt * 128u,
+                                                             smem_desc_sw128(vs_sm, kHalfBytes, 1024), idesc_pv, nn[tt] > 0);
+                mma_commit(smem_u32(&ctl->pv_done[tt]));
+                pend_bar[tt] = smem_u32(&ctl->pv_done[tt]); pend_par[tt] = nn[tt] & 1;
+                need[tt] = false;
+              }
+            if (!alive || *abort_flag || clock64() - t0 > budget) { alive = false; break; }
+          }
+          if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+          // P lies over S, and the next block's V tile goes into the same slot: the products must be over
+#pragma unroll
+          for (int tt = 0; tt < 2; ++tt)
+            if (comp[tt] && alive) {
+              alive = mbar_wait(smem_u32(&ctl->pv_done[tt]), nn[tt] & 1, abort_flag, budget);
+              if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
+              pend_bar[tt] = 0;
+              ++nn[tt];
+            }
+          if (!alive) break;
+        }
+#pragma unroll
+        for (int tt = 0; tt < 2; ++tt)
+          if (part[tt]) {
+            ++kl[tt];
+            if (ow[tt] & kOutEnd) {
+              act[tt] = false;
+              mbar_arrive(smem_u32(&ctl->fin[tt]));   // nothing of the item is in flight any more: its group may finish
+            }
+          }
+      }
+      if (alive && act[0]) {
+        // the ranking is exhausted and the first tile still has entries: its list is no subsequence of the second's
+        ctl->abort_flag = 1;
+        atomicMin(status, (int32_t)COSA_ERR_BAD_ORDER);
+      }
+      // whatever is still in flight finishes on its own and must have done so before the CTA retires
+      if (cnt0 > 0) (void)mbar_wait_noabort(smem_u32(&ctl->q_full[0]), 0);
+      if (cnt1 > 0) (void)mbar_wait_noabort(smem_u32(&ctl->q_full[1]), 0);
+      for (int tt = 0; tt < 2; ++tt)
+        if (pend_bar[tt] != 0 && !mbar_wait_noabort(pend_bar[tt], pend_par[tt]) && !*abort_flag) report_timeout(ctl, status);
+      for (int kk = k_taken; kk < k_req; ++kk)
+        if (!mbar_wait_noabort(smem_u32(&ctl->kr_full[kk % kKRing]), (kk / kKRing) & 1) && !*abort_flag) report_timeout(ctl, status);
+      if (v_taken < v_req && !mbar_wait_noabort(smem_u32(&ctl->vs_full), (v_req - 1) & 1) && !*abort_flag) report_timeout(ctl, status);
+    } else if (!kShared && issuer) {
       // ------------------------------------------------------------------ issuer of item t
       const uint32_t idesc_qk = idesc_bf16(kBlock, kBlock, 0, 0);     // Q [M x K] and K_j [N x K], both K-major
       const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);   // P [M x K] from TMEM, V_j [K x N] N-major
@@ -330,8 +480,10 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
         k_end = k;
         if (leader) {
           if (compute) {                              // fetch V_j now that the block is known to be computed: into the
-            ctl->v_req[t] = n;                        // slot of K_j, which the finished product has released
-            load_kv_block(p, &v_map, x_sm + (k & 1) * kTileBytes, b, g, min(max(jv, 0), p.nqb - 1), smem_u32(&ctl->v_full[t]));
+            if (!kShared) {                           // slot of K_j, which the finished product has released
+              ctl->v_req[t] = n;                      // (kShared: the issuer requests it, once for both tiles)
+              load_kv_block(p, &v_map, x_sm + (k & 1) * kTileBytes, b, g, min(max(jv, 0), p.nqb - 1), smem_u32(&ctl->v_full[t]));
+            }
             dec_word |= 1u << (k & 31);
           }
           ctl->out_w[t][k & 1] = (compute ? kOutCompute : 0u) | (last ? kOutEnd : 0u);
@@ -407,7 +559,9 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
 #pragma unroll
           for (int c = 0; c < kBlock; ++c) s[c] = 0u;
         }
-        unsigned char* stage0 = smem + (size_t)(2 + 2 * t) * kTileBytes;
+        // (kShared: in the item's Q tile, which no product reads any more; the K ring may still serve the other tile)
+        unsigned char* stage0 = smem + (size_t)(kShared ? t : 2 + 2 * t) * kTileBytes;
+        const uint32_t stage_sm = kShared ? q_sm : x_sm;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           const uint32_t* o = &s[c * 32];
@@ -427,8 +581,8 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
         bar_sync(bar_id, kBlock);
         if (p.lse) p.lse[(size_t)q_row0 + r] = (n > 0 && l > 0.f) ? (m_run + log2f(l)) * 0.6931471805599453f : -INFINITY;
         if (leader) {
-          tma_store_tile(&o_map, 0, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, x_sm);
-          tma_store_tile(&o_map, 64, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, x_sm + kHalfBytes);
+          tma_store_tile(&o_map, 0, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, stage_sm);
+          tma_store_tile(&o_map, 64, i * kBlock, h, b, p.oo.row, p.oo.head, p.oo.outer, stage_sm + kHalfBytes);
           tma_store_commit_and_wait_read();
           if (p.visited) p.visited[row] = n;
           if (p.scored) p.scored[row] = k_end + 1;
@@ -445,17 +599,19 @@ osk_duo_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant_
 
 }  // namespace
 
-cudaError_t launch_osk_duo(const OskParams& p_in, cudaStream_t st) {
+// shared: the work items of a CTA are the two row tiles of a 256-row query block and share every fetched tile
+cudaError_t launch_osk_duo(const OskParams& p_in, bool shared, cudaStream_t st) {
   CUtensorMap qm, km, vm, om;
   OskParams p = p_in;
   TileOrder vo;
   // K and V: the dense tensors, or page pools whose pages hold whole key blocks
   if (p.pg.table && p.pg.page_size < kBlock) return cudaErrorInvalidValue;   // staged as dense tensors by the caller of this launcher
+  if (shared && (p.mask || p.pg.seq_lens || p.nqb % 2 != 0)) return cudaErrorInvalidValue;
   if (!make_tile_map(&qm, &p.qo, p.q, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.qs) ||
       !make_kv_map(&km, &p.ko, p.k, p.pg, p.ks, p.batch, p.hkv, p.n) || !make_kv_map(&vm, &vo, p.v, p.pg, p.ks, p.batch, p.hkv, p.n) ||
       !make_tile_map(&om, &p.oo, p.out, (uint64_t)p.n, (uint64_t)p.hq, (uint64_t)p.batch, p.os))
     return cudaErrorInvalidValue;
-  auto kernel = p.mask ? osk_duo_kernel<true> : osk_duo_kernel<false>;
+  auto kernel = shared ? osk_duo_kernel<false, true> : (p.mask ? osk_duo_kernel<true, false> : osk_duo_kernel<false, false>);
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (e != cudaSuccess) return e;
   if (p.decisions) {

@@ -561,6 +561,76 @@ def test_kap_wide_query_blocks_4k(cfg1, impl):
             assert o[h, 2 * big, :c[h, 2 * big]].tolist() == [j for j in hi if j != 2 * big + 1]
 
 
+def _wide_lists(q, k, budget, causal=True, stride=8):
+    order, count = alloc_lists(q.shape[1], q.shape[2] // 128)
+    cosa.cosa_kap_select(q, k, budget, order, count, causal=causal, opt=cosa.default_options(stride=stride), block_q=256)
+    assert cosa.cosa_device_status() == 0
+    return order, count
+
+
+@pytest.mark.parametrize("budget,tb,skip_scale", [(0.3, 0.4, 150.0), (0.6, 0.5, 400.0), (1.0, 0.3, 150.0), (0.6, 0.5, -1.0),
+                                                  (0.6, 1.0, -1.0), (1.0, 1.0, -1.0)])
+def test_osk_two_row_tiles_of_a_wide_block_share_each_fetched_tile(small, budget, tb, skip_scale):
+    """impl = 5: one CTA walks the ranking of a 256-row query block once for both of its 128-row tiles (Sec. C.1: the
+    skip test stays per 128 rows).  Each tile must come out as if it had walked its own list alone: decisions,
+    counters, outputs and LSE against the oracle on every tile, and the same decisions and counters as the
+    one-item kernel on the same lists."""
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    nqb = q.shape[2] // 128
+    order, count = _wide_lists(q, k, budget)
+    bufs = run_osk(q, k, v, order, count, tb, skip_scale, impl=5)
+    check_osk_against_oracle(qf, kf, vf, _np(order), _np(count), bufs, tb, skip_scale, range(q.shape[1]), range(nqb))
+    one = run_osk(q, k, v, order, count, tb, skip_scale, impl=0)
+    for key in ("visited", "scored", "decisions"):
+        assert torch.equal(bufs[key], one[key]), key
+    assert (bufs["out"].float() - one["out"].float()).abs().max() < OUT_MAX
+
+
+def test_osk_wide_blocks_noncausal_and_4k(small, cfg1):
+    q, k, v = small["dev"]
+    qf, kf, vf = small["f64"]
+    nqb = q.shape[2] // 128
+    order, count = _wide_lists(q, k, 0.5, causal=False)
+    bufs = run_osk(q, k, v, order, count, 0.5, 150.0, impl=5, causal=False)
+    check_osk_against_oracle(qf, kf, vf, _np(order), _np(count), bufs, 0.5, 150.0, range(q.shape[1]), range(nqb), causal=False)
+    w = cfg1["w"]
+    q, k, v = cfg1["dev"]
+    qf, kf, vf = cfg1["f64"]
+    order, count = _wide_lists(q, k, w.kap_budget, stride=w.stride)
+    bufs = run_osk(q, k, v, order, count, w.osk_budget, w.skip_scale, impl=5)
+    check_osk_against_oracle(qf, kf, vf, _np(order), _np(count), bufs, w.osk_budget, w.skip_scale, range(w.hq),
+                             [0, 1, 2, 3, 14, 15, 30, 31])
+
+
+def test_osk_wide_blocks_refuse_lists_that_are_not_nested(small):
+    """The first tile's list must be a subsequence of the second's (what block_q = 256 selection writes); ordinary
+    per-tile lists are not, in general, and the kernel reports that instead of walking something else."""
+    q, k, v = small["dev"]
+    nqb = q.shape[2] // 128
+    order, count = alloc_lists(q.shape[1], nqb)
+    order.fill_(-1)
+    order[..., 0] = 0
+    count.fill_(1)
+    order[:, :, 1::2, 0] = 1          # second tiles list block 1 only, first tiles block 0 only
+    bufs = alloc_outputs(q, nqb)
+    cosa.cosa_osk_attention(q, k, v, order, count, 0.5, bufs["out"], bufs["lse"], bufs["visited"],
+                            opt=cosa.default_options(skip_scale=150.0, impl=5))
+    assert cosa.cosa_device_status() == -6
+    assert cosa.cosa_device_status() == 0
+    # the same lists nested by hand (block 0 for both) are fine, and masks, lengths and odd block counts are refused up front
+    order[..., 0] = 0
+    cosa.cosa_osk_attention(q, k, v, order, count, 0.5, bufs["out"], bufs["lse"], bufs["visited"],
+                            opt=cosa.default_options(skip_scale=150.0, impl=5))
+    assert cosa.cosa_device_status() == 0
+    assert int(bufs["visited"].min()) == 1 and int(bufs["visited"].max()) == 1
+    with pytest.raises((cosa.CosaError, ValueError)):
+        cosa.cosa_osk_attention(q[:, :, :896].contiguous(), k[:, :, :896].contiguous(), v[:, :, :896].contiguous(),
+                                order[:, :, :7].contiguous(), count[:, :, :7].contiguous(), 0.5, bufs["out"][:, :, :896].contiguous(),
+                                bufs["lse"][:, :, :896].contiguous(), bufs["visited"][:, :, :7].contiguous(),
+                                opt=cosa.default_options(skip_scale=150.0, impl=5, order_stride=nqb))
+
+
 # ---------------------------------------------------------------------------------- paged K/V
 def _pools(w, page_size):
     """K and V of the workload as page pools that share one seeded page table."""

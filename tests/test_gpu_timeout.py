@@ -43,12 +43,13 @@ def test_kap_wait_budget_of_one_cycle_reports_a_timeout_and_the_next_call_is_cle
     assert torch.equal(order, ref_order) and torch.equal(count, ref_count)
 
 
-@pytest.mark.parametrize("impl", [0, 4])        # one work item per CTA, two work items per CTA
+@pytest.mark.parametrize("impl", [0, 4, 5])     # one work item per CTA, two work items per CTA, the two row tiles of a 256-row block per CTA
 def test_osk_wait_budget_of_one_cycle_reports_a_timeout_and_the_next_call_is_clean(cfg1, impl):
     w, (q, k, v) = cfg1["w"], cfg1["dev"]
     nqb = w.n // 128
     order, count = alloc_lists(w.hq, nqb)
-    cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride))
+    cosa.cosa_kap_select(q, k, w.kap_budget, order, count, opt=cosa.default_options(stride=w.stride),
+                         block_q=256 if impl == 5 else 128)
     ref = alloc_outputs(q, nqb)
     cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, ref["out"], ref["lse"], ref["visited"],
                             opt=cosa.default_options(skip_scale=w.skip_scale, impl=impl))
