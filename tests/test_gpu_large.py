@@ -214,6 +214,17 @@ def test_qwen3_32k_wide_query_blocks_sampled():
             assert ref_count[0, i] == count_np[h, i] and np.array_equal(ref_order[0, i], order_np[h, i]), (h, i)
         one = {k_: t[:, h:h + 1] for k_, t in bufs.items()}
         check_osk_against_oracle(qf, kf, vf, order_np[h:h + 1], count_np[h:h + 1], one, w.osk_budget, w.skip_scale, [0], tiles[::3])
+    # the same lists walked by one CTA per 256-row block, every fetched K/V tile serving both row tiles (impl = 5): every
+    # decision and counter of the layer as above, outputs within rounding of them
+    shared = {k_: torch.zeros_like(t) for k_, t in bufs.items()}
+    opt5 = cosa.default_options(stride=w.stride, skip_scale=w.skip_scale, order_stride=pitch, impl=5,
+                                out_scored=shared["scored"], out_decisions=shared["decisions"])
+    cosa.cosa_osk_attention(q, k, v, order, count, w.osk_budget, shared["out"], shared["lse"], shared["visited"], opt=opt5)
+    assert cosa.cosa_device_status() == 0
+    for key in ("visited", "scored", "decisions"):
+        assert torch.equal(shared[key], bufs[key]), key
+    assert float((shared["out"].float() - bufs["out"].float()).abs().max()) < 2e-2
+    assert float((shared["lse"] - bufs["lse"]).abs().max()) < 1e-3
 
 
 def test_llama31_64k_budget_sweep_sampled():
