@@ -56,6 +56,7 @@ def parse():
     ap.add_argument("--osk-impl", type=int, default=0, choices=[0, 4, 5],
                     help="4: the OSK kernel that walks two work items per CTA (cosa_options.impl = 4); 5: the same kernel on the two row "
                          "tiles of a 256-row query block, every fetched K/V tile serving both (needs --block-q 256); not the headline config")
+    ap.add_argument("--no-burst", action="store_true", help="skip the five spaced single steps reported beside the timed region")
     ap.add_argument("--top-p", type=float, default=0.0,
                     help="Stage 1 by Top-p instead of the workload's budget fraction (Sec. C.1: 0.95); not the headline config")
     args = ap.parse_args()
@@ -333,6 +334,26 @@ def main():
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": ke}
         del ws
 
+    # ---- the same step as a burst: five launches 50 ms apart, best of five.  The K back-to-back steps above pull the SM
+    # clock down within some twenty launches (sw_power_cap; 1965 -> about 1750 MHz), while the burst GEMM peak the
+    # roofline is set against was taken as a best-of-ten of single products at the full clock; this is the step measured
+    # the same way, reported beside the timed region's figures, never in place of them.
+    burst_run = None
+    if rank == 0 and world == 1 and not args.no_burst:
+        bk, bo = [], []
+        for _ in range(5):
+            torch.cuda.synchronize()
+            time.sleep(0.05)
+            e3 = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e3[0].record(stream)
+            cosa.cosa_kap_select(q, k_in, kap_budget, order, count, opt=opt, stream=stream, block_q=args.block_q)
+            e3[1].record(stream)
+            cosa.cosa_osk_attention(q, k_in, v_in, order, count, w.osk_budget, out, lse, visited, opt=opt, stream=stream)
+            e3[2].record(stream)
+            torch.cuda.synchronize()
+            bk.append(e3[0].elapsed_time(e3[1])); bo.append(e3[1].elapsed_time(e3[2]))
+        burst_run = {"kap_ms": min(bk), "osk_ms": min(bo), "how": "best of 5 single steps 50 ms apart (SM clock at its maximum)"}
+
     # ---- rooflines (fractions "of measured" unless the peaks file is absent)
     peaks = measured_peaks()
     # Which measured GEMM figure a kernel is set against follows the length of the timed region: the burst figure
@@ -366,6 +387,10 @@ def main():
         return r
 
     roof_osk = tensor_roof("osk_duo_kernel" if args.osk_impl in (4, 5) else "osk_tc_kernel", osk_tflops, {"traffic": (traffic or {}).get("osk_tc_kernel")})
+    if burst_run:
+        b_tflops = flops_step / (burst_run["osk_ms"] * 1e-3) / 1e12
+        roof_osk["as_a_burst"] = {"ms": burst_run["osk_ms"], "achieved": b_tflops, "frac_of_burst": b_tflops / peaks["bf16_tflops"],
+                                  "how": burst_run["how"]}
     # KAP: the screen kernel forms the sampled logits on the tensor cores (one pass over the key tiles; whole tiles,
     # so somewhat more than the causal pairs), the sort kernel is ALU work; the algorithmic FLOPs (causal pairs only)
     # are set against the tensor peak, and the algorithmic bytes (sampled rows read once, lists written once)
@@ -420,6 +445,7 @@ def main():
                            "blocks_scored": n_scored, "blocks_computed": n_computed,
                            "causal_block_pairs": pairs, "input_generation_s": round(t_gen, 1)},
                 "latency_ms": {"kap": kap_ms, "osk": osk_ms, "kap_plus_osk": ms_per_step},
+                "latency_ms_as_a_burst": ({"kap": burst_run["kap_ms"], "osk": burst_run["osk_ms"], "how": burst_run["how"]} if burst_run else None),
                 "e2e": e2e, "gpu_launches": 4 * args.steps, "clocks": clocks, "roofline": roofline,
                 "roofline_osk": roof_osk, "roofline_kap": roof_kap, "cpu_baseline": cpu, "comparators": extras,
                 "wall_s_timed_region": t_wall}

@@ -139,6 +139,7 @@ struct OskParams {
   float theta;           // ln(Delta / N)
   float skip_scale;      // Delta (for items whose own length replaces N, see item_theta)
   float scale;           // softmax scale
+  int wave;              // (set by the tensor-core launcher) CTAs resident at a time; a CTA prefetches list lines for the work item that many further on
   long long wait_budget; // clock cycles a device-side wait may take before the kernel gives up
   Strides qs, ks, os;    // strides of q, of k and v (dense; pools are contiguous), of out
   TileOrder qo, ko, oo;  // coordinate order of the tensor maps over q, over k and v, over out (set by the launcher)

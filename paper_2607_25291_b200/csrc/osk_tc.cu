@@ -345,9 +345,11 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
           if (!alive) { if (!*abort_flag) report_timeout(ctl, status); break; }
         }
         // Issuing a product keeps this thread busy for about as long as the product runs, so whatever is checked
-        // between two products leaves the tensor pipe idle: look at the next position now, without waiting.
+        // between two products leaves the tensor pipe idle: look at the next position now, without waiting.  Only with
+        // Stage 2 off, where products follow one another closely; in a sparse walk the next S buffer is rarely free
+        // yet, and the two tests then only delay the product at hand (1 % of the kernel at 128K).
         verified = false;
-        if (kk + 1 < n_certain) {
+        if (!kStage2 && kk + 1 < n_certain) {
           const int k1 = kk + 1;
           verified = mbar_test_wait(smem_u32(&ctl->k_full[k1 % kKStages]), (k1 / kKStages) & 1) &&
                      mbar_test_wait(smem_u32(&ctl->s_empty[k1 & 1]), ((k1 >> 1) & 1) ^ 1);
@@ -367,6 +369,16 @@ osk_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__
   } else if (warp == 3) {
     // ------------------------------------------------------------------ PV issuer
     if (lane == 0) {
+      // The count and the head of the list of the work item one wave of CTAs further on: the tiles streamed since KAP
+      // wrote them have pushed these lines out of L2, and that CTA's first loads would wait for HBM (0.3 % of the kernel)
+      if (!kMask && w + (int)p.wave < (int)gridDim.x) {
+        const int w2 = w + (int)p.wave;
+        const int b2 = w2 / (p.hkv * per_kv), wk2 = w2 % (p.hkv * per_kv);
+        const int g2 = wk2 / per_kv, i2 = p.nqb - 1 - (wk2 % per_kv) / G, h2 = g2 * G + (wk2 % per_kv) % G;
+        const size_t row2 = (size_t)(b2 * p.hq + h2) * p.nqb + i2;
+        prefetch_l2(p.order + row2 * p.order_stride);
+        prefetch_l2(p.count + row2);
+      }
       const uint32_t idesc_pv = idesc_bf16(kBlock, kHeadDim, 0, 1);  // P [M x K] from TMEM, V_j [K x N] N-major
       const uint64_t vdesc0 = smem_desc_sw128(v_sm, kHalfBytes, 1024);
       bool alive = true;
@@ -758,6 +770,10 @@ cudaError_t launch_osk_tc(const OskParams& p_in, cudaStream_t st) {
   }
   int32_t* status = device_status_word();
   if (!status) return cudaErrorInvalidSymbol;
+  int dev = 0, n_sm = 0;
+  p.wave = 1 << 30;   // (no prefetch if the SM count cannot be read)
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n_sm > 0)
+    p.wave = n_sm;    // one CTA per SM
   kernel<<<p.batch * p.hq * p.nqb, kThreads, kSmemBytes, st>>>(qm, km, vm, om, p, status);
   return cudaGetLastError();
 }
